@@ -1,0 +1,150 @@
+/*
+ * patconv — pattern-based sparse 3x3 convolution for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The operations follow "An Image Enhancing Pattern-based Sparsity for Real-time Inference on
+ * Mobile Devices" (arXiv 2001.07710):
+ *   - pattern pruning: every 3x3 kernel is multiplied element-wise by one binary mask taken from
+ *     a small pattern library; every mask keeps exactly four entries (Section 4.1, Section 5.1);
+ *   - connectivity pruning: whole kernels are removed according to their L2 norm (Section 6.1);
+ *   - filter / kernel re-ordering and compact weight storage for execution (Section 6.2).
+ *
+ * Conventions used by every entry point
+ *   kernel position (r,s): r = row 0..2 (top to bottom), s = column 0..2 (left to right);
+ *   mask bit b = 3*r + s; a pattern is a 9-bit integer with exactly four bits set.
+ *   weights      [F][C][3][3] fp32, F = filters (output channels), C = input channels.
+ *   activations  NHWC, fp32 or fp16; outputs NHWC in the ORIGINAL filter order.
+ *   convolution  cross-correlation (no kernel flip), zero padding 1, stride 1 or 2, no bias:
+ *                Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1.
+ *
+ * Memory and execution
+ *   "dev" pointers are device memory owned by the caller; "host" pointers are host memory.
+ *   The library allocates no device memory unless an entry point says otherwise.  All device
+ *   work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *   and the calls return without synchronising.  Arguments are validated on the host before
+ *   anything is launched.
+ *
+ * Errors
+ *   Every function that returns int returns PAT_OK (0) or a PAT_ERR_* code; nothing is launched
+ *   when a code other than PAT_OK / PAT_ERR_CUDA is returned.  pat_last_error() gives a
+ *   thread-local message for the last failing call on the calling thread.
+ */
+#ifndef PATCONV_H_
+#define PATCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PAT_OK               0
+#define PAT_ERR_INVALID_ARG  1   /* null pointer, negative size, value out of range          */
+#define PAT_ERR_SHAPE        2   /* unsupported tensor shape                                  */
+#define PAT_ERR_LIBRARY      3   /* pattern library: mask without 4 bits, duplicate, K range  */
+#define PAT_ERR_DTYPE        4   /* dtype is neither PAT_F32 nor PAT_F16                      */
+#define PAT_ERR_ALIGN        5   /* pointer alignment                                         */
+#define PAT_ERR_BLOB         6   /* packed blob does not match the arguments                  */
+#define PAT_ERR_CUDA         7   /* a CUDA runtime call failed                                */
+#define PAT_ERR_WORKSPACE    8   /* workspace or blob buffer too small                        */
+
+#define PAT_F32 0                /* fp32 storage, fp32 accumulation                           */
+#define PAT_F16 1                /* fp16 storage (weights, activations), fp32 accumulation    */
+
+#define PAT_PRUNED 0xFF          /* pattern id of a kernel removed by connectivity pruning    */
+
+const char *pat_strerror(int code);
+const char *pat_last_error(void);
+
+/* Built-in pattern libraries (Section 4.2 derives the eight patterns; Section 7.1 uses libraries
+ * of 12, 8 and 4 patterns).  K = 4: centre + three of the four arms (missing arm: down, up, left,
+ * right).  K = 8: those plus the four 2x2 blocks containing the centre (top-left, top-right,
+ * bottom-left, bottom-right).  K = 12: those plus {centre, up, down, top-left corner} and its
+ * three clockwise quarter-turn rotations (a convention of this library: the paper shows the
+ * additional four patterns only in a figure).
+ * masks_out: host, K entries.  Returns PAT_ERR_LIBRARY for any other K. */
+int pat_library_builtin(int K, uint16_t *masks_out);
+
+/* Bytes of device workspace pat_project needs for an F x C layer (0 on invalid sizes). */
+size_t pat_project_workspace(int F, int C);
+
+/* Pattern selection + connectivity pruning of one layer (Sections 4.1, 5.1, 6.1).
+ * For every kernel (f,c) the mask of the library that keeps the largest sum of squares is chosen
+ * (squares and sums in float64, bits in ascending order; lowest pattern id on ties).  The n_keep
+ * kernels with the largest kept sum of squares survive (lower f*C+c on ties); the others are
+ * removed.  Results are exact and deterministic.
+ *   w           dev, [F][C][3][3] fp32
+ *   masks       host, K distinct 9-bit masks with four bits each, 1 <= K <= 255
+ *   n_keep      0 .. F*C
+ *   pattern_id  dev out, [F*C] bytes: chosen pattern id, PAT_PRUNED for removed kernels
+ *   w_masked    dev out, [F][C][3][3] fp32: kept entries bit-identical to w, all others +0.0;
+ *               may be the same buffer as w
+ *   workspace   dev, at least pat_project_workspace(F, C) bytes, 256-byte aligned; contents are
+ *               scratch (no need to clear); concurrent calls must use different workspaces */
+int pat_project(const float *w, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+                uint8_t *pattern_id, float *w_masked, void *workspace, size_t workspace_bytes,
+                void *stream);
+
+/* Size in bytes of the packed blob of a layer (0 on invalid arguments).  A pure function of its
+ * arguments, so no device-to-host transfer is ever needed to size a buffer. */
+size_t pat_pack_size(int F, int C, int K, int64_t n_keep, int dtype);
+
+/* Compressed, re-ordered weight storage (Section 6.2: filters with similar kernels are grouped,
+ * and inside each filter the kernels of identical pattern are grouped).
+ * Canonical section of the blob (host-readable layout given by pat_blob_layout):
+ *   perm[F]       i32  new position -> original filter; filters sorted by kept-kernel count
+ *                      (descending), then per-pattern count vector (lexicographically
+ *                      descending), then original index (ascending)
+ *   fptr[F+1]     i32  first kernel of each re-ordered filter; fptr[F] = n_keep
+ *   pptr[F][K+1]  i32  first kernel of each pattern segment of the filter
+ *   chan[n_keep]  u16  input channel of each kernel; kernels ordered by (pattern id, channel)
+ *   w4[n_keep][4]      the four kept entries in ascending bit order, fp32, or fp16 rounded to
+ *                      nearest-even when dtype = PAT_F16
+ * followed by an execution section (kernels re-sorted by blocks of 16 input channels) that only
+ * pat_conv3x3 reads.
+ *   w_masked, pattern_id  dev, as written by pat_project; exactly n_keep kernels must be kept
+ *   blob        dev out, at least pat_pack_size(...) bytes, 256-byte aligned */
+int pat_pack(const float *w_masked, const uint8_t *pattern_id, int F, int C,
+             const uint16_t *masks, int K, int64_t n_keep, int dtype,
+             void *blob, size_t blob_bytes, void *stream);
+
+/* Byte offsets of the canonical arrays inside a blob (host-side helper; offsets[0..4] =
+ * perm, fptr, pptr, chan, w4).  Returns PAT_ERR_* on invalid arguments. */
+int pat_blob_layout(int F, int C, int K, int64_t n_keep, int dtype, size_t offsets[5]);
+
+/* Expand a blob back to dense masked weights [F][C][3][3] fp32 (fp16 entries are widened
+ * exactly).  Inverse of pat_pack: for dtype PAT_F32 the result is bit-identical to w_masked. */
+int pat_unpack(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+               int dtype, float *w_dense_out, void *stream);
+
+/* The sparse convolution (the execution side of Section 6.2: per-pattern access code with the
+ * four tap positions fixed at compile time, no per-weight index decoding, pattern-grouped
+ * kernels, filters grouped by load).
+ *   Y[n][y][x][f] = sum over kept kernels (f,c) and their four taps (r,s) of
+ *                   w[f][c][r][s] * X[n][y*stride + r - 1][x*stride + s - 1][c]
+ * Products and sums are fp32 (fp16 inputs are widened exactly); the result is stored in the
+ * blob's dtype (fp16: round to nearest even).
+ *   blob     dev, written by pat_pack with the same (F, C, masks, K, n_keep, dtype)
+ *   masks    host, the library the blob was packed with (selects the compiled tap code)
+ *   x        dev, NHWC [N][H][W][C], 16-byte aligned
+ *   y        dev out, NHWC [N][Ho][Wo][F], 16-byte aligned, must not overlap x
+ * Restrictions: C a multiple of 8, F a multiple of 8 (PAT_ERR_SHAPE otherwise). */
+int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+                int dtype, const void *x, void *y, int N, int H, int W, int stride, void *stream);
+
+/* Dense 3x3 convolution for layers that are not pruned (the first layer of VGG-16, C = 3).
+ *   w   dev, [F][C][3][3] fp32 (converted to the activation type on the fly)
+ *   x   dev NHWC [N][H][W][C]; y dev NHWC [N][Ho][Wo][F]; dtype of x and y = `dtype`
+ * Restrictions: C <= 16, F a multiple of 8, F <= 512. */
+int pat_conv3x3_dense(const float *w, int F, int C, int dtype, const void *x, void *y,
+                      int N, int H, int W, int stride, void *stream);
+
+/* Synchronises `stream` and returns the device-side status word: PAT_OK, or PAT_ERR_BLOB when a
+ * kernel found a blob header that did not match its arguments (the kernel then wrote nothing).
+ * The word is cleared by the call. */
+int pat_query_status(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PATCONV_H_ */

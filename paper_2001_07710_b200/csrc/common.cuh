@@ -1,0 +1,80 @@
+// Shared host/device definitions of the patconv library: error reporting, blob layout, launch helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/patconv.h"
+
+namespace pat {
+
+constexpr uint32_t kBlobMagic = 0x50415443u;  // "PATC"
+constexpr uint32_t kBlobVersion = 1u;
+constexpr int kChanTile = 16;                 // granularity (input channels) of the execution section
+constexpr int kMaxK = 255;
+
+// First 256 bytes of every blob.
+struct BlobHeader {
+  uint32_t magic, version;
+  int32_t F, C, K, dtype;
+  int64_t n_keep;
+  uint64_t total_bytes;
+  uint16_t masks[kMaxK + 1];  // library the blob was packed with (entries >= K are 0)
+};
+static_assert(sizeof(BlobHeader) <= 768, "header must fit its slot");
+constexpr size_t kHeaderBytes = 768;
+
+// Byte offsets of every array in a blob; a pure function of (F, C, K, n_keep, dtype).
+struct BlobLayout {
+  size_t perm, fptr, pptr, chan, w4;   // canonical section
+  size_t tptr, tmeta, tw4;             // execution section
+  size_t scratch;                      // pack-time temporaries: hist[F][K], count[F], inverse permutation[F]
+  size_t total;
+  int nct;                             // number of 16-channel tiles = ceil(C / 16)
+};
+
+__host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+__host__ __device__ inline int elem_bytes(int dtype) { return dtype == PAT_F16 ? 2 : 4; }
+
+__host__ __device__ inline BlobLayout blob_layout(int F, int C, int K, int64_t n_keep, int dtype) {
+  BlobLayout L;
+  const size_t e = (size_t)elem_bytes(dtype);
+  const size_t nk = (size_t)n_keep;
+  L.nct = (C + kChanTile - 1) / kChanTile;
+  size_t o = kHeaderBytes;
+  L.perm = o;  o = align256(o + sizeof(int32_t) * (size_t)F);
+  L.fptr = o;  o = align256(o + sizeof(int32_t) * ((size_t)F + 1));
+  L.pptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 1));
+  L.chan = o;  o = align256(o + sizeof(uint16_t) * nk);
+  L.w4 = o;    o = align256(o + 4 * e * nk);
+  L.tptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)L.nct + 1));
+  L.tmeta = o; o = align256(o + sizeof(uint32_t) * nk);
+  L.tw4 = o;   o = align256(o + 4 * e * nk);
+  L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 2));
+  L.total = o;
+  return L;
+}
+
+// Library passed by value to kernels.
+struct MaskTable {
+  uint16_t m[kMaxK + 1];
+  int K;
+};
+
+// Device address of the status word shared by all kernels of the library (nullptr on failure).
+int* status_word();
+
+int set_error(int code, const char* fmt, ...);
+int check_library(const uint16_t* masks, int K);
+int check_cuda(cudaError_t e, const char* what);
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Tap positions of a mask: bits in ascending order.
+__host__ __device__ inline void mask_bits(uint32_t m, int bits[4]) {
+  int t = 0;
+  for (int b = 0; b < 9 && t < 4; ++b)
+    if (m & (1u << b)) bits[t++] = b;
+  for (; t < 4; ++t) bits[t] = 4;
+}
+
+}  // namespace pat

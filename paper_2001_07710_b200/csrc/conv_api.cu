@@ -1,0 +1,26 @@
+// pat_conv3x3: argument validation and choice of the kernel for a layer shape.
+#include "common.cuh"
+
+namespace pat {
+int conv_generic(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep, int dtype,
+                 const void* x, void* y, int N, int H, int W, int stride, cudaStream_t st);
+}
+
+using namespace pat;
+
+extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                           int dtype, const void* x, void* y, int N, int H, int W, int stride, void* stream) {
+  if (!blob || !x || !y) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3: null pointer");
+  if (F < 1 || C < 1 || F > 65535 || C > 65535) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: F=%d C=%d outside 1..65535", F, C);
+  if (int rc = check_library(masks, K)) return rc;
+  if (dtype != PAT_F32 && dtype != PAT_F16) return set_error(PAT_ERR_DTYPE, "pat_conv3x3: dtype %d", dtype);
+  if (n_keep < 0 || n_keep > (int64_t)F * C) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3: n_keep outside 0..F*C");
+  if (N < 1 || H < 1 || W < 1) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: N, H, W must be positive");
+  if (stride != 1 && stride != 2) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3: stride %d (1 or 2)", stride);
+  if (!aligned(blob, 256)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3: blob must be 256-byte aligned");
+  if (!aligned(x, 16) || !aligned(y, 16)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3: x and y must be 16-byte aligned");
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  if ((size_t)N * ((Ho + 7) / 8) * ((Wo + 31) / 32) > 0x7FFFFFFFull) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: too many tiles");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  return conv_generic(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, st);
+}

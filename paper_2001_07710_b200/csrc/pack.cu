@@ -1,0 +1,270 @@
+// pat_pack / pat_unpack: compressed, re-ordered weight storage.
+//
+// Section 6.2 re-orders filters so that filters with similar kernels sit together (balanced work per thread
+// group) and groups, inside each filter, the kernels that share a pattern (one code path per group, no
+// branches inside it).  The blob holds a canonical section in exactly that order and an execution section in
+// which each filter's kernels are re-sorted by blocks of 16 input channels (the unit in which the convolution
+// kernels stage activations), then pattern, then channel.
+#include "common.cuh"
+
+namespace pat {
+namespace {
+
+struct BlobPtrs {
+  BlobHeader* hdr;
+  int32_t *perm, *fptr, *pptr;
+  uint16_t* chan;
+  void* w4;
+  int32_t* tptr;
+  uint32_t* tmeta;
+  void* tw4;
+  int32_t *hist, *cnt, *inv;
+};
+
+__host__ __device__ inline BlobPtrs blob_ptrs(void* blob, const BlobLayout& L, int F, int K) {
+  char* b = static_cast<char*>(blob);
+  BlobPtrs p;
+  p.hdr = reinterpret_cast<BlobHeader*>(b);
+  p.perm = reinterpret_cast<int32_t*>(b + L.perm);
+  p.fptr = reinterpret_cast<int32_t*>(b + L.fptr);
+  p.pptr = reinterpret_cast<int32_t*>(b + L.pptr);
+  p.chan = reinterpret_cast<uint16_t*>(b + L.chan);
+  p.w4 = b + L.w4;
+  p.tptr = reinterpret_cast<int32_t*>(b + L.tptr);
+  p.tmeta = reinterpret_cast<uint32_t*>(b + L.tmeta);
+  p.tw4 = b + L.tw4;
+  p.hist = reinterpret_cast<int32_t*>(b + L.scratch);
+  p.cnt = p.hist + (size_t)F * K;
+  p.inv = p.cnt + F;
+  return p;
+}
+
+// One block per original filter: per-pattern counts and kept count.
+__global__ void __launch_bounds__(256) k_pack_count(const uint8_t* __restrict__ pid, int C, int K, BlobPtrs bp, int* status) {
+  extern __shared__ int sh[];   // K counters
+  const int f = blockIdx.x;
+  for (int j = threadIdx.x; j < K; j += blockDim.x) sh[j] = 0;
+  __syncthreads();
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    const int p = pid[(size_t)f * C + c];
+    if (p == PAT_PRUNED) continue;
+    if (p >= K) { atomicExch(status, PAT_ERR_BLOB); continue; }
+    atomicAdd(&sh[p], 1);
+  }
+  __syncthreads();
+  int tot = 0;
+  for (int j = threadIdx.x; j < K; j += blockDim.x) bp.hist[(size_t)f * K + j] = sh[j];
+  if (threadIdx.x == 0) {
+    for (int j = 0; j < K; ++j) tot += sh[j];
+    bp.cnt[f] = tot;
+  }
+}
+
+// One thread per filter: position = number of filters that come before it in the ordering
+// (kept count descending, per-pattern counts lexicographically descending, original index ascending).
+__global__ void k_pack_rank(int F, int K, BlobPtrs bp) {
+  const int f = blockIdx.x * blockDim.x + threadIdx.x;
+  if (f >= F) return;
+  const int nf = bp.cnt[f];
+  const int32_t* hf = bp.hist + (size_t)f * K;
+  int rank = 0;
+  for (int g = 0; g < F; ++g) {
+    if (g == f) continue;
+    const int ng = bp.cnt[g];
+    bool before;
+    if (ng != nf) before = ng > nf;
+    else {
+      const int32_t* hg = bp.hist + (size_t)g * K;
+      int j = 0;
+      while (j < K && hg[j] == hf[j]) ++j;
+      before = (j < K) ? (hg[j] > hf[j]) : (g < f);
+    }
+    rank += before ? 1 : 0;
+  }
+  bp.perm[rank] = f;
+  bp.inv[f] = rank;
+}
+
+// One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
+__global__ void __launch_bounds__(1024) k_pack_ptrs(int F, int C, int K, long long n_keep, int dtype, MaskTable lib,
+                                                    unsigned long long total_bytes, BlobPtrs bp, int* status) {
+  __shared__ int part[1024];
+  __shared__ int carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < F; base += 1024) {
+    const int q = base + threadIdx.x;
+    const int v = (q < F) ? bp.cnt[bp.perm[q]] : 0;
+    part[threadIdx.x] = v;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+      const int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0;
+      __syncthreads();
+      part[threadIdx.x] += a;
+      __syncthreads();
+    }
+    if (q < F) {
+      const int start = carry + part[threadIdx.x] - v;
+      bp.fptr[q] = start;
+      const int32_t* h = bp.hist + (size_t)bp.perm[q] * K;
+      int pos = start;
+      for (int j = 0; j < K; ++j) { bp.pptr[(size_t)q * (K + 1) + j] = pos; pos += h[j]; }
+      bp.pptr[(size_t)q * (K + 1) + K] = pos;
+    }
+    __syncthreads();
+    if (threadIdx.x == 1023) carry += part[1023];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    bp.fptr[F] = carry;
+    const bool ok = (long long)carry == n_keep;
+    if (!ok) atomicExch(status, PAT_ERR_BLOB);
+    BlobHeader* h = bp.hdr;
+    h->magic = ok ? kBlobMagic : 0u;
+    h->version = kBlobVersion;
+    h->F = F; h->C = C; h->K = K; h->dtype = dtype;
+    h->n_keep = n_keep;
+    h->total_bytes = total_bytes;
+    for (int j = 0; j <= kMaxK; ++j) h->masks[j] = lib.m[j];
+  }
+}
+
+template <typename T> __device__ inline T cvt_weight(float v);
+template <> __device__ inline float cvt_weight<float>(float v) { return v; }
+template <> __device__ inline __half cvt_weight<__half>(float v) { return __float2half_rn(v); }
+
+// One block per original filter: place every kept kernel in the canonical and in the execution order.
+template <typename T>
+__global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ wm, const uint8_t* __restrict__ pid,
+                                                      int C, int K, int nct, MaskTable lib, BlobPtrs bp) {
+  extern __shared__ uint8_t spid[];   // C pattern ids of this filter
+  const int f = blockIdx.x;
+  const int q = bp.inv[f];
+  for (int c = threadIdx.x; c < C; c += blockDim.x) spid[c] = pid[(size_t)f * C + c];
+  __syncthreads();
+  const int f0 = bp.fptr[q];
+  // execution-section pointers: kernels of this filter before channel tile t
+  for (int t = threadIdx.x; t <= nct; t += blockDim.x) {
+    int n = 0;
+    const int cend = min(t * kChanTile, C);
+    for (int c = 0; c < cend; ++c) n += (spid[c] != PAT_PRUNED) ? 1 : 0;
+    bp.tptr[(size_t)q * (nct + 1) + t] = f0 + n;
+  }
+  T* w4 = static_cast<T*>(bp.w4);
+  T* tw4 = static_cast<T*>(bp.tw4);
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    const int j = spid[c];
+    if (j == PAT_PRUNED || j >= K) continue;
+    const int tile = c / kChanTile;
+    int same_before = 0;      // kernels of the same pattern on lower channels      (canonical order)
+    int exec_before = 0;      // kernels ordered before (tile, pattern, channel)    (execution order)
+    for (int d = 0; d < C; ++d) {
+      const int pd = spid[d];
+      if (pd == PAT_PRUNED) continue;
+      same_before += (pd == j && d < c) ? 1 : 0;
+      const int td = d / kChanTile;
+      const bool lt = (td < tile) || (td == tile && (pd < j || (pd == j && d < c)));
+      exec_before += lt ? 1 : 0;
+    }
+    const int pos = bp.pptr[(size_t)q * (K + 1) + j] + same_before;
+    const int tpos = f0 + exec_before;
+    bp.chan[pos] = (uint16_t)c;
+    bp.tmeta[tpos] = (uint32_t)c | ((uint32_t)j << 16);
+    int bits[4];
+    mask_bits(lib.m[j], bits);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const T v = cvt_weight<T>(wm[((size_t)f * C + c) * 9 + bits[t]]);
+      w4[(size_t)pos * 4 + t] = v;
+      tw4[(size_t)tpos * 4 + t] = v;
+    }
+  }
+}
+
+__device__ inline bool header_matches(const BlobHeader* h, int F, int C, int K, long long n_keep, int dtype, const MaskTable& lib) {
+  if (h->magic != kBlobMagic || h->version != kBlobVersion) return false;
+  if (h->F != F || h->C != C || h->K != K || h->dtype != dtype || h->n_keep != n_keep) return false;
+  for (int j = 0; j < K; ++j) if (h->masks[j] != lib.m[j]) return false;
+  return true;
+}
+
+// One block per re-ordered filter: write its kept entries into the (pre-zeroed) dense tensor.
+template <typename T>
+__global__ void __launch_bounds__(128) k_unpack(BlobPtrs bp, int F, int C, int K, long long n_keep, int dtype, MaskTable lib,
+                                                float* __restrict__ out, int* status) {
+  if (!header_matches(bp.hdr, F, C, K, n_keep, dtype, lib)) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(status, PAT_ERR_BLOB);
+    return;
+  }
+  const int q = blockIdx.x;
+  const int f = bp.perm[q];
+  const T* w4 = static_cast<const T*>(bp.w4);
+  for (int j = 0; j < K; ++j) {
+    int bits[4];
+    mask_bits(lib.m[j], bits);
+    const int a = bp.pptr[(size_t)q * (K + 1) + j], b = bp.pptr[(size_t)q * (K + 1) + j + 1];
+    for (int k = a + threadIdx.x; k < b; k += blockDim.x) {
+      const int c = bp.chan[k];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) out[((size_t)f * C + c) * 9 + bits[t]] = (float)w4[(size_t)k * 4 + t];
+    }
+  }
+}
+
+int common_checks(const char* who, int F, int C, const uint16_t* masks, int K, int64_t n_keep, int dtype) {
+  if (F < 1 || C < 1 || F > 65535 || C > 65535) return set_error(PAT_ERR_SHAPE, "%s: F=%d C=%d outside 1..65535", who, F, C);
+  if (int rc = check_library(masks, K)) return rc;
+  if (dtype != PAT_F32 && dtype != PAT_F16) return set_error(PAT_ERR_DTYPE, "%s: dtype %d", who, dtype);
+  if (n_keep < 0 || n_keep > (int64_t)F * C) return set_error(PAT_ERR_INVALID_ARG, "%s: n_keep=%lld outside 0..F*C", who, (long long)n_keep);
+  return PAT_OK;
+}
+
+MaskTable make_table(const uint16_t* masks, int K) {
+  MaskTable lib;
+  for (int j = 0; j <= kMaxK; ++j) lib.m[j] = (j < K) ? masks[j] : (uint16_t)0;
+  lib.K = K;
+  return lib;
+}
+
+}  // namespace
+}  // namespace pat
+
+using namespace pat;
+
+extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F, int C,
+                        const uint16_t* masks, int K, int64_t n_keep, int dtype,
+                        void* blob, size_t blob_bytes, void* stream) {
+  if (!w_masked || !pattern_id || !blob) return set_error(PAT_ERR_INVALID_ARG, "pat_pack: null pointer");
+  if (int rc = common_checks("pat_pack", F, C, masks, K, n_keep, dtype)) return rc;
+  if (!aligned(blob, 256)) return set_error(PAT_ERR_ALIGN, "pat_pack: blob must be 256-byte aligned");
+  const BlobLayout L = blob_layout(F, C, K, n_keep, dtype);
+  if (blob_bytes < L.total) return set_error(PAT_ERR_WORKSPACE, "pat_pack: blob has %zu bytes, needs %zu", blob_bytes, L.total);
+  int* status = status_word();
+  if (!status) return set_error(PAT_ERR_CUDA, "pat_pack: cannot resolve the status word");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const MaskTable lib = make_table(masks, K);
+  const BlobPtrs bp = blob_ptrs(blob, L, F, K);
+  k_pack_count<<<F, 256, K * sizeof(int), st>>>(pattern_id, C, K, bp, status);
+  k_pack_rank<<<(F + 127) / 128, 128, 0, st>>>(F, K, bp);
+  k_pack_ptrs<<<1, 1024, 0, st>>>(F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
+  if (dtype == PAT_F16) k_pack_scatter<__half><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+  else k_pack_scatter<float><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+  return check_cuda(cudaGetLastError(), "pat_pack launch");
+}
+
+extern "C" int pat_unpack(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                          int dtype, float* w_dense_out, void* stream) {
+  if (!blob || !w_dense_out) return set_error(PAT_ERR_INVALID_ARG, "pat_unpack: null pointer");
+  if (int rc = common_checks("pat_unpack", F, C, masks, K, n_keep, dtype)) return rc;
+  if (!aligned(blob, 256)) return set_error(PAT_ERR_ALIGN, "pat_unpack: blob must be 256-byte aligned");
+  int* status = status_word();
+  if (!status) return set_error(PAT_ERR_CUDA, "pat_unpack: cannot resolve the status word");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const BlobLayout L = blob_layout(F, C, K, n_keep, dtype);
+  const BlobPtrs bp = blob_ptrs(const_cast<void*>(blob), L, F, K);
+  const MaskTable lib = make_table(masks, K);
+  if (int rc = check_cuda(cudaMemsetAsync(w_dense_out, 0, sizeof(float) * 9 * (size_t)F * C, st), "pat_unpack memset")) return rc;
+  if (dtype == PAT_F16) k_unpack<__half><<<F, 128, 0, st>>>(bp, F, C, K, (long long)n_keep, dtype, lib, w_dense_out, status);
+  else k_unpack<float><<<F, 128, 0, st>>>(bp, F, C, K, (long long)n_keep, dtype, lib, w_dense_out, status);
+  return check_cuda(cudaGetLastError(), "pat_unpack launch");
+}

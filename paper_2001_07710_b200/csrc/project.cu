@@ -1,0 +1,240 @@
+// pat_project: per-kernel pattern selection and per-layer connectivity pruning, exact and deterministic.
+//
+// Pattern pruning multiplies each 3x3 kernel by one mask of the library (Section 4.1); the mask kept is the
+// one that retains the largest squared L2 norm, the one-shot form of the argmax binarisation of Section 5.1.
+// Connectivity pruning ranks kernels by their L2 norm (Section 6.1) and keeps the n_keep strongest of the layer.
+//
+// Exactness: squares of fp32 values are exact in fp64 and are added in ascending bit order, so the energies
+// are the same bits on any IEEE machine.  The n_keep-th largest energy is found with a 4-pass, 16-bit radix
+// select over the (monotone) bit pattern of the non-negative doubles; ties at the threshold are resolved by
+// index with a block scan.
+#include "common.cuh"
+
+namespace pat {
+namespace {
+
+constexpr int kSelBlock = 1024;
+constexpr int kBins = 65536;
+
+struct SelectState {
+  unsigned long long prefix;   // bits of the threshold key decided so far
+  long long remaining;         // how many keys with this prefix (and below-decided digits) are still to be kept
+};
+
+// workspace layout
+struct ProjWs {
+  unsigned long long* key;     // [FC] energy bit patterns
+  unsigned char* pid;          // [FC] best pattern per kernel
+  unsigned int* hist;          // [65536]
+  unsigned int* blk;           // [nblk + 1] tie counts per block, then exclusive offsets
+  SelectState* st;
+  size_t bytes;
+};
+
+inline ProjWs carve(void* base, int64_t FC) {
+  ProjWs w;
+  char* p = static_cast<char*>(base);
+  size_t o = 0;
+  w.key = reinterpret_cast<unsigned long long*>(p + o); o = align256(o + 8 * (size_t)FC);
+  w.pid = reinterpret_cast<unsigned char*>(p + o);      o = align256(o + (size_t)FC);
+  w.hist = reinterpret_cast<unsigned int*>(p + o);      o = align256(o + 4 * (size_t)kBins);
+  const size_t nblk = (size_t)((FC + kSelBlock - 1) / kSelBlock);
+  w.blk = reinterpret_cast<unsigned int*>(p + o);       o = align256(o + 4 * (nblk + 1));
+  w.st = reinterpret_cast<SelectState*>(p + o);         o = align256(o + sizeof(SelectState));
+  w.bytes = o;
+  return w;
+}
+
+// One thread per kernel: energies of all masks, argmax (lowest id on ties).
+__global__ void k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
+                                 unsigned long long* __restrict__ key, unsigned char* __restrict__ pid) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= FC) return;
+  double sq[9];
+#pragma unroll
+  for (int b = 0; b < 9; ++b) {
+    const double v = (double)w[i * 9 + b];
+    sq[b] = v * v;
+  }
+  double best_e = -1.0;
+  int best = 0;
+  for (int j = 0; j < lib.K; ++j) {
+    const unsigned m = lib.m[j];
+    double e = 0.0;
+#pragma unroll
+    for (int b = 0; b < 9; ++b)
+      if (m & (1u << b)) e += sq[b];
+    if (e > best_e) { best_e = e; best = j; }
+  }
+  key[i] = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
+  pid[i] = (unsigned char)best;
+}
+
+__global__ void k_sel_init(SelectState* st, long long n_keep, unsigned int* hist) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
+  if (i < kBins) hist[i] = 0u;
+}
+
+// Histogram of the current 16-bit digit over the keys that match the decided prefix.
+__global__ void k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
+                           const SelectState* __restrict__ st, unsigned int* __restrict__ hist) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= FC) return;
+  const int shift = 48 - 16 * pass;
+  const unsigned long long k = key[i];
+  if (pass > 0 && (k >> (shift + 16)) != st->prefix) return;
+  atomicAdd(&hist[(unsigned)((k >> shift) & 0xFFFFull)], 1u);
+}
+
+// One block: find the digit d with  count(digit > d) < remaining <= count(digit >= d);  clears the histogram.
+__global__ void __launch_bounds__(1024) k_sel_pick(SelectState* st, unsigned int* hist) {
+  __shared__ unsigned long long part[1024];
+  const int t = threadIdx.x;
+  constexpr int per = kBins / 1024;   // 64 bins per thread; thread 0 owns the highest digits
+  const int top = kBins - 1 - t * per;
+  unsigned long long s = 0;
+  for (int q = 0; q < per; ++q) s += hist[top - q];
+  part[t] = s;
+  __syncthreads();
+  // inclusive scan (Hillis-Steele) over threads, highest digits first
+  for (int off = 1; off < 1024; off <<= 1) {
+    unsigned long long v = (t >= off) ? part[t - off] : 0ull;
+    __syncthreads();
+    part[t] += v;
+    __syncthreads();
+  }
+  const unsigned long long before = part[t] - s;   // keys with digits above this thread's range
+  const unsigned long long rem = (unsigned long long)st->remaining;
+  __syncthreads();
+  if (rem > before && rem <= before + s) {
+    unsigned long long above = before;
+    for (int q = 0; q < per; ++q) {
+      const unsigned int h = hist[top - q];
+      if (rem <= above + h) {
+        st->prefix = (st->prefix << 16) | (unsigned long long)(top - q);
+        st->remaining = (long long)(rem - above);
+        break;
+      }
+      above += h;
+    }
+  }
+  __syncthreads();
+  for (int q = 0; q < per; ++q) hist[top - q] = 0u;
+}
+
+// Ties at the threshold: count per block of 1024 consecutive kernels.
+__global__ void __launch_bounds__(kSelBlock) k_tie_count(const unsigned long long* __restrict__ key, int64_t FC,
+                                                         const SelectState* __restrict__ st, unsigned int* __restrict__ blk) {
+  const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
+  const int tie = (i < FC && key[i] == st->prefix) ? 1 : 0;
+  const int n = __syncthreads_count(tie);
+  if (threadIdx.x == 0) blk[blockIdx.x] = (unsigned)n;
+}
+
+// One block: exclusive scan of the per-block tie counts (sequential over chunks of 1024 blocks).
+__global__ void __launch_bounds__(1024) k_tie_scan(unsigned int* blk, int nblk) {
+  __shared__ unsigned int part[1024];
+  __shared__ unsigned int carry;
+  if (threadIdx.x == 0) carry = 0u;
+  __syncthreads();
+  for (int base = 0; base < nblk; base += 1024) {
+    const int i = base + threadIdx.x;
+    const unsigned int v = (i < nblk) ? blk[i] : 0u;
+    part[threadIdx.x] = v;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+      unsigned int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0u;
+      __syncthreads();
+      part[threadIdx.x] += a;
+      __syncthreads();
+    }
+    if (i < nblk) blk[i] = carry + part[threadIdx.x] - v;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry += part[1023];
+    __syncthreads();
+  }
+}
+
+// Decide keep / remove per kernel and write pattern ids and masked weights.
+__global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t FC, MaskTable lib,
+                                                        const unsigned long long* __restrict__ key,
+                                                        const unsigned char* __restrict__ pid_in,
+                                                        const SelectState* __restrict__ st,
+                                                        const unsigned int* __restrict__ blk,
+                                                        unsigned char* __restrict__ pid_out, float* wm, int keep_all_or_none) {
+  __shared__ unsigned int warp_cnt[kSelBlock / 32];
+  const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
+  const bool valid = i < FC;
+  bool keep;
+  if (keep_all_or_none >= 0) {            // n_keep == F*C (1) or n_keep == 0 (0): no threshold needed
+    keep = keep_all_or_none == 1;
+  } else {
+    const unsigned long long thr = st->prefix;
+    const unsigned long long k = valid ? key[i] : 0ull;
+    const bool tie = valid && k == thr;
+    // rank of this tie among all ties in index order
+    const unsigned ballot = __ballot_sync(0xFFFFFFFFu, tie);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) warp_cnt[wid] = __popc(ballot);
+    __syncthreads();
+    unsigned rank = blk[blockIdx.x] + __popc(ballot & ((1u << lane) - 1u));
+    for (int q = 0; q < wid; ++q) rank += warp_cnt[q];
+    keep = valid && (k > thr || (tie && (long long)rank < st->remaining));
+  }
+  if (!valid) return;
+  const unsigned char p = pid_in[i];
+  const unsigned m = keep ? lib.m[p] : 0u;
+  pid_out[i] = keep ? p : (unsigned char)PAT_PRUNED;
+#pragma unroll
+  for (int b = 0; b < 9; ++b) {
+    const float v = w[i * 9 + b];
+    wm[i * 9 + b] = (m & (1u << b)) ? v : 0.0f;
+  }
+}
+
+}  // namespace
+}  // namespace pat
+
+using namespace pat;
+
+extern "C" size_t pat_project_workspace(int F, int C) {
+  if (F < 1 || C < 1 || F > 65535 || C > 65535) return 0;
+  return carve(nullptr, (int64_t)F * C).bytes;
+}
+
+extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                           uint8_t* pattern_id, float* w_masked, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  if (!w || !pattern_id || !w_masked || !workspace) return set_error(PAT_ERR_INVALID_ARG, "pat_project: null pointer");
+  if (F < 1 || C < 1 || F > 65535 || C > 65535) return set_error(PAT_ERR_SHAPE, "pat_project: F=%d C=%d outside 1..65535", F, C);
+  if (int rc = check_library(masks, K)) return rc;
+  const int64_t FC = (int64_t)F * C;
+  if (n_keep < 0 || n_keep > FC) return set_error(PAT_ERR_INVALID_ARG, "pat_project: n_keep=%lld outside 0..%lld", (long long)n_keep, (long long)FC);
+  if (!aligned(w, 4) || !aligned(w_masked, 4)) return set_error(PAT_ERR_ALIGN, "pat_project: weights must be 4-byte aligned");
+  if (!aligned(workspace, 256)) return set_error(PAT_ERR_ALIGN, "pat_project: workspace must be 256-byte aligned");
+  const ProjWs ws = carve(workspace, FC);
+  if (workspace_bytes < ws.bytes) return set_error(PAT_ERR_WORKSPACE, "pat_project: workspace has %zu bytes, needs %zu", workspace_bytes, ws.bytes);
+
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  MaskTable lib;
+  for (int j = 0; j <= kMaxK; ++j) lib.m[j] = (j < K) ? masks[j] : (uint16_t)0;
+  lib.K = K;
+  const int nb256 = (int)((FC + 255) / 256);
+  const int nblk = (int)((FC + kSelBlock - 1) / kSelBlock);
+  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid);
+  int mode = -1;
+  if (n_keep == FC) mode = 1;
+  else if (n_keep == 0) mode = 0;
+  if (mode < 0) {
+    k_sel_init<<<kBins / 256, 256, 0, st>>>(ws.st, (long long)n_keep, ws.hist);
+    for (int pass = 0; pass < 4; ++pass) {
+      k_sel_hist<<<nb256, 256, 0, st>>>(ws.key, FC, pass, ws.st, ws.hist);
+      k_sel_pick<<<1, 1024, 0, st>>>(ws.st, ws.hist);
+    }
+    k_tie_count<<<nblk, kSelBlock, 0, st>>>(ws.key, FC, ws.st, ws.blk);
+    k_tie_scan<<<1, 1024, 0, st>>>(ws.blk, nblk);
+  }
+  k_finalize<<<nblk, kSelBlock, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
+  return check_cuda(cudaGetLastError(), "pat_project launch");
+}

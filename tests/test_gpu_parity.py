@@ -1,0 +1,144 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2001_07710_b200 as pc
+from paper_2001_07710_b200 import workloads
+from helpers import check_close, gpu_project_pack, read_blob, store, stored_weights
+
+pytestmark = pytest.mark.gpu
+
+
+def _weights(seed, F, C):
+    return workloads.make_weights(np.random.default_rng(seed), F, C)
+
+
+# ------------------------------------------------------------------ projection: bit exact
+@pytest.mark.parametrize("F,C,K,num,den", [(8, 8, 8, 3, 10), (64, 64, 8, 3, 10), (37, 53, 12, 1, 8), (128, 64, 4, 1, 4),
+                                            (256, 256, 12, 1, 2), (512, 512, 8, 1, 8), (5, 3, 8, 1, 1), (3, 1100, 8, 1, 3)])
+def test_project_bit_exact(F, C, K, num, den):
+    w = _weights(F * 1000 + C, F, C)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm = pc.pat_project(torch.from_numpy(w).cuda(), pc.pat_library_builtin(K), n_keep)
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    assert np.array_equal(wm.cpu().numpy().view(np.uint32), wm_o.view(np.uint32))
+
+
+def test_project_full_library_and_in_place():
+    masks = np.array([sum(1 << b for b in comb) for comb in itertools.combinations(range(9), 4)], dtype=np.uint16)
+    w = _weights(11, 24, 40)
+    pid_o, wm_o, _ = oracle.project(w, masks, 300)
+    wt = torch.from_numpy(w).cuda()
+    pid, wm = pc.pat_project(wt, masks, 300, w_masked=wt)        # w_masked aliases w
+    assert wm.data_ptr() == wt.data_ptr()
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    assert np.array_equal(wm.cpu().numpy().view(np.uint32), wm_o.view(np.uint32))
+
+
+@pytest.mark.parametrize("n_keep", [0, 1, 7, 40, 41, 100, 2047, 2048])
+def test_project_ties_and_extremes(n_keep):
+    """Many identical kernels (ties at the threshold broken by index), zero kernels, all / none kept."""
+    rng = np.random.default_rng(3)
+    F, C = 32, 64
+    w = np.zeros((F, C, 3, 3), dtype=np.float32)
+    base = rng.standard_normal((5, 3, 3)).astype(np.float32)
+    choice = rng.integers(0, 6, size=(F, C))
+    for i in range(5):
+        w[choice == i] = base[i]                                   # choice == 5 stays all-zero
+    masks = oracle.library(8)
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm = pc.pat_project(torch.from_numpy(w).cuda(), masks, n_keep)
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    assert np.array_equal(wm.cpu().numpy().view(np.uint32), wm_o.view(np.uint32))
+    assert int((pid.cpu().numpy() != 255).sum()) == n_keep
+
+
+# ------------------------------------------------------------------ pack: bit exact, round trip
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("F,C,K,num,den", [(8, 8, 8, 3, 10), (64, 64, 8, 3, 10), (37, 53, 12, 1, 8), (256, 256, 4, 1, 2),
+                                            (512, 512, 8, 1, 8), (16, 48, 8, 1, 1), (16, 16, 8, 0, 1)])
+def test_pack_bit_exact_and_round_trip(F, C, K, num, den, dtype):
+    w = _weights(F * 7 + C, F, C)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.pack(wm_o, pid_o, masks, dtype)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    got = read_blob(blob, F, C, K, n_keep, dtype)
+    for name in ("perm", "fptr", "pptr", "chan", "w4"):
+        assert np.array_equal(got[name], ref[name]), name
+    back = pc.pat_unpack(blob, F, C, masks, n_keep, dtype).cpu().numpy()
+    if dtype == "f32":
+        assert np.array_equal(back.view(np.uint32), wm_o.view(np.uint32))
+    else:
+        assert np.array_equal(back, wm_o.astype(np.float16).astype(np.float32))
+    assert pc.pat_query_status() == 0
+
+
+def test_blob_mismatch_is_reported_not_executed():
+    F, C, K = 16, 16, 8
+    masks = oracle.library(K)
+    w = _weights(5, F, C)
+    pid, wm, blob = gpu_project_pack(w, masks, 64, "f32")
+    x = torch.zeros((1, 8, 8, C), device="cuda")
+    y = torch.full((1, 8, 8, F), 7.0, device="cuda")
+    other = oracle.library(12)[4:12]                                # a different library of the same size
+    pc.pat_conv3x3(blob, F, C, other, 64, "f32", x, y=y)
+    with pytest.raises(pc.PatError) as e:
+        pc.pat_query_status()
+    assert e.value.code == 6
+    assert float(y.min()) == 7.0                                    # nothing was written
+    assert pc.pat_query_status() == 0                               # the word was cleared
+
+
+# ------------------------------------------------------------------ convolution
+CONV_CASES = [
+    # N, H, W, C, F, K, keep num/den, stride
+    (1, 56, 56, 64, 64, 8, 3, 10, 1),      # config 0
+    (2, 20, 37, 24, 40, 8, 1, 4, 1),       # ragged tiles, C and F not multiples of 16/32
+    (3, 9, 33, 16, 8, 12, 1, 2, 1),
+    (1, 1, 1, 8, 8, 4, 1, 1, 1),           # single pixel
+    (2, 14, 14, 128, 96, 8, 1, 8, 1),
+    (2, 28, 28, 64, 64, 4, 1, 1, 1),       # nothing pruned by connectivity
+    (1, 12, 12, 32, 32, 8, 0, 1, 1),       # everything pruned: output is zero
+    (2, 56, 56, 32, 32, 8, 1, 4, 2),       # stride 2, even size
+    (2, 15, 23, 16, 24, 12, 1, 2, 2),      # stride 2, odd sizes
+    (1, 7, 7, 48, 64, 8, 1, 4, 1),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_conv_matches_oracle(case, dtype):
+    N, H, W, C, F, K, num, den, stride = case
+    rng = np.random.default_rng(hash(case) % (2 ** 32))
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, dtype), x, stride)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, torch.from_numpy(x).cuda(), stride)
+    assert pc.pat_query_status() == 0
+    assert tuple(y.shape) == ref.shape
+    check_close(y.float().cpu().numpy(), ref, dtype)
+    if n_keep == 0:
+        assert not y.any()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("N,H,W,C,F,stride", [(2, 40, 70, 3, 64, 1), (1, 9, 9, 1, 8, 1), (2, 17, 33, 3, 40, 2), (1, 16, 16, 16, 32, 1)])
+def test_dense_conv_matches_oracle(N, H, W, C, F, stride, dtype):
+    rng = np.random.default_rng(N * 1000 + H)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    ref = oracle.conv3x3(stored_weights(w, dtype), x, stride)
+    y = pc.pat_conv3x3_dense(torch.from_numpy(w).cuda(), dtype, torch.from_numpy(x).cuda(), stride)
+    check_close(y.float().cpu().numpy(), ref, dtype)
