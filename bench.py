@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Throughput of the pattern-sparse 3x3 convolution path on synthetic VGG-16-shaped layers.
+
+One step = one pass of the whole path over one batch: for each of the 13 VGG-16 conv layers, pattern
+selection + connectivity pruning (pat_project), packing (pat_pack) and the convolution itself
+(pat_conv3x3; the first layer, C = 3, is dense: pat_conv3x3_dense).  Every layer has its own seeded input
+tensor of that layer's shape (batch 64, fp16 storage, fp32 accumulation), all resident in HBM before the
+timed region; the working set (about 3.4 GB) is far larger than L2, so nothing is reused across steps.
+
+Prints one JSON line.  `--impl reference` times the CPU oracle on the host cores instead (a bounded sample).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2001_07710_b200 import workloads  # noqa: E402
+
+METRIC = "pattern-sparse conv images/s"
+UNIT = "images/s"
+SM_COUNT, FMA_LANES, SM_MAX_MHZ = 148, 128, 1965.0
+FMA_PEAK_TFLOPS = 2 * FMA_LANES * SM_COUNT * SM_MAX_MHZ * 1e6 / 1e12     # 74.45: fp32 FMA, no tensor cores
+DEFAULT_CONFIG = 3
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return json.load(open(p)), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm)); out["sm_max_mhz"] = float(max(mx)); out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2001_07710_b200 as pc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    pc.load()
+
+    cfg = workloads.configs()[args.config]
+    N = cfg.N if args.batch is None else args.batch
+    dtype = cfg.dtype
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    elem = 2 if dtype == "f16" else 4
+    masks = {K: pc.pat_library_builtin(K) for K in (4, 8, 12)}
+    stream = torch.cuda.current_stream()
+
+    # ---- seeded host tensors (pinned: they are also the source of the end-to-end copies)
+    layers = []
+    for L in cfg.layers:
+        w_np, x_np = workloads.make_layer_tensors(cfg.number, L, N)
+        hw = torch.from_numpy(w_np).pin_memory()
+        hx = torch.from_numpy(x_np).to(tdt).pin_memory()
+        del x_np
+        hy = torch.empty((N, L.Ho, L.Wo, L.F), dtype=tdt).pin_memory()
+        st = dict(L=L, hw=hw, hx=hx, hy=hy,
+                  w=hw.cuda(), x=hx.cuda(), y=torch.empty((N, L.Ho, L.Wo, L.F), dtype=tdt, device="cuda"))
+        if not L.dense:
+            st["pid"] = torch.empty((L.F, L.C), dtype=torch.uint8, device="cuda")
+            st["wm"] = torch.empty((L.F, L.C, 3, 3), dtype=torch.float32, device="cuda")
+            st["ws"] = torch.empty(pc.pat_project_workspace(L.F, L.C), dtype=torch.uint8, device="cuda")
+            st["blob"] = torch.empty(pc.pat_pack_size(L.F, L.C, L.K, L.n_keep, dtype), dtype=torch.uint8, device="cuda")
+        layers.append(st)
+
+    def step(conv_events=None):
+        for i, st in enumerate(layers):
+            L = st["L"]
+            if L.dense:
+                if conv_events is not None: conv_events[i][0].record(stream)
+                pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
+                if conv_events is not None: conv_events[i][1].record(stream)
+            else:
+                pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
+                pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
+                if conv_events is not None: conv_events[i][0].record(stream)
+                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"])
+                if conv_events is not None: conv_events[i][1].record(stream)
+
+    def step_e2e():
+        for st in layers:
+            L = st["L"]
+            st["w"].copy_(st["hw"], non_blocking=True)
+            st["x"].copy_(st["hx"], non_blocking=True)
+            if L.dense:
+                pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
+            else:
+                pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
+                pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
+                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"])
+            st["hy"].copy_(st["y"], non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- warm-up
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert pc.pat_query_status() == 0
+
+    # ---- timed region: device-resident inputs
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
+          for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    launches0 = pc.pat_launch_count()
+    barrier()
+    sampler.start()
+    e0.record(stream)
+    for k in range(args.steps):
+        step(ev[k])
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = pc.pat_launch_count() - launches0
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_step = ms_total / args.steps
+    value = world * N * args.steps / (ms_total * 1e-3)
+
+    # per-layer convolution times (mean over the timed steps)
+    conv_ms = [float(np.mean([ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)])) for i in range(len(layers))]
+
+    # ---- end to end: host buffers, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, 3))
+    step_e2e()
+    barrier()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_e2e()
+    e1.record(stream)
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+    h2d = sum(st["hw"].numel() * 4 + st["hx"].numel() * elem for st in layers)
+    d2h = sum(st["hy"].numel() * elem for st in layers)
+    assert pc.pat_query_status() == 0
+
+    # ---- roofline of the dominant kernel (the sparse convolution), and per layer
+    peaks, peak_kind = measured_peaks()
+    hbm = peaks["hbm_gbs"]
+    per_layer = []
+    sparse_flop = sparse_ms = 0.0
+    for st, ms in zip(layers, conv_ms):
+        L = st["L"]
+        flop = L.useful_flop(N)
+        byts = L.compulsory_bytes(N, elem)
+        t_roof_us = max(flop / (FMA_PEAK_TFLOPS * 1e12), byts / (hbm * 1e9)) * 1e6
+        per_layer.append({"layer": L.name, "shape": f"{L.H}x{L.W}x{L.C}->{L.F}", "n_keep": L.n_keep,
+                          "conv_us": round(ms * 1e3, 2), "eff_tflops": round(flop / (ms * 1e-3) / 1e12, 3),
+                          "roof_us": round(t_roof_us, 2), "roof_frac": round(t_roof_us / (ms * 1e3), 4)})
+        if not L.dense:
+            sparse_flop += flop; sparse_ms += ms
+    achieved = sparse_flop / (sparse_ms * 1e-3) / 1e12
+    total_flop = sum(st["L"].useful_flop(N) for st in layers)
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 storage, f32 accumulate" if dtype == "f16" else "f32", "data": "synthetic",
+        "config": {"workload": f"config {cfg.number}: {cfg.name}", "batch_per_gpu": N,
+                   "layers": len(layers), "step": "project + pack + conv for every layer",
+                   "l2": "inputs larger than L2 (about 3.4 GB touched per step)", "seed": workloads.BASE_SEED},
+        "effective_gflops": round(total_flop * world * args.steps / (ms_total * 1e-3) / 1e9, 1),
+        "conv_only_images_per_s": round(world * N / (sum(conv_ms) * 1e-3), 2),
+        "roofline": {"bound": "alu", "kernel": "sparse conv (12 launches per step)", "achieved": round(achieved, 3),
+                     "peak": round(FMA_PEAK_TFLOPS, 2), "unit": "TFLOP/s", "frac": round(achieved / FMA_PEAK_TFLOPS, 4),
+                     "peak_kind": "derived: 2 x 128 fp32 lanes x 148 SMs x 1.965 GHz", "traffic": None,
+                     "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
+                     "min_layer_frac": min(p["roof_frac"] for p in per_layer if p["layer"] != "conv1")},
+        "layers": per_layer,
+        "e2e": {"value": round(world * N * e2e_steps / (ms_e2e * 1e-3), 2), "unit": UNIT,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_seconds)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: a seeded fraction of the outputs of one image
+    of every layer, each computed by the oracle's direct float64 definition over the masked weights."""
+
+    def __init__(self, cfg, frac: float):
+        import oracle
+        self.oracle = oracle
+        self.cfg = cfg
+        self.frac = frac
+        self.items = []
+        rng = np.random.default_rng(1234)
+        for L in cfg.layers:
+            w, x = workloads.make_layer_tensors(cfg.number, L, cfg.N, n_limit=1)
+            if cfg.dtype == "f16":
+                x = x.astype(np.float16)
+            if L.dense:
+                wm = w
+            else:
+                _, wm, _ = oracle.project(w, oracle.library(L.K), L.n_keep)
+            if cfg.dtype == "f16":
+                wm = wm.astype(np.float16)
+            total = L.Ho * L.Wo * L.F
+            n = max(1, int(round(total * frac)))
+            flat = rng.choice(total, size=n, replace=False) if n < total else np.arange(total)
+            coords = np.stack([np.zeros(n, dtype=np.int64), flat // (L.Wo * L.F), (flat // L.F) % L.Wo, flat % L.F], axis=1).astype(np.int32)
+            self.items.append((L, wm.astype(np.float64), x, coords))
+
+    def run(self):
+        acc = 0.0
+        for L, wm, x, coords in self.items:
+            acc += float(self.oracle.conv3x3_at(wm, x, coords, L.stride).sum())
+        return acc
+
+
+def _omp_threads() -> int:
+    v = os.environ.get("OMP_NUM_THREADS")
+    if v:
+        return int(v)
+    return len(os.sched_getaffinity(0))
+
+
+def _calibrate(cfg, budget_s: float) -> float:
+    """Fraction of one image's outputs the oracle can compute in about budget_s seconds."""
+    probe = OracleSample(cfg, 0.002)
+    t = time.perf_counter(); probe.run(); dt = time.perf_counter() - t
+    return float(min(1.0, 0.002 * budget_s / max(dt, 1e-6)))
+
+
+def cpu_baseline(cfg, budget_s: float = 20.0):
+    frac = _calibrate(cfg, budget_s)
+    s = OracleSample(cfg, frac)
+    t = time.perf_counter(); s.run(); dt = time.perf_counter() - t
+    reps = 1
+    while dt < 0.5 * budget_s and reps < 16:          # fast hosts: repeat the sample to reach the time budget
+        t = time.perf_counter(); s.run(); dt += time.perf_counter() - t
+        reps += 1
+    return {"value": round(frac * reps / dt, 5), "unit": UNIT, "cores": _omp_threads(), "kind": "oracle",
+            "sample": f"{frac * 100:.2f}% of the outputs of one image of all {len(cfg.layers)} layers, {reps} time(s) "
+                      f"(direct dense float64 convolution of the masked weights), {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = workloads.configs()[args.config]
+    total = args.steps + args.warmup
+    per_step = max(2.0, min(20.0, 150.0 / max(total, 1)))
+    frac = _calibrate(cfg, per_step)
+    s = OracleSample(cfg, frac)
+    for _ in range(args.warmup):
+        s.run()
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        s.run()
+    dt = time.perf_counter() - t
+    value = frac * args.steps / dt
+    sample = (f"{frac * 100:.3f}% of the outputs of one image of all {len(cfg.layers)} layers per step, "
+              f"direct dense float64 convolution of the masked weights")
+    out = {"impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": UNIT,
+           "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": round(dt / args.steps * 1e3, 2), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"config {cfg.number}: {cfg.name}", "sample": sample, "seed": workloads.BASE_SEED},
+           "cpu_baseline": {"value": round(value, 5), "unit": UNIT, "cores": _omp_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": round(value, 5), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="workload number (3 = VGG-16 batch 64 fp16 storage)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch size (profiling small cases)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -144,6 +144,10 @@ int pat_conv3x3_dense(const float *w, int F, int C, int dtype, const void *x, vo
  * The word is cleared by the call. */
 int pat_query_status(void *stream);
 
+/* Number of CUDA kernels this library has launched from the calling process so far (all threads,
+ * all entry points).  Host-side counter; useful to check that work really ran on the GPU. */
+uint64_t pat_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

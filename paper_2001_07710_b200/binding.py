@@ -23,7 +23,7 @@ TORCH_DTYPE = {PAT_F32: torch.float32, PAT_F16: torch.float16}
 
 EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project_workspace", "pat_project",
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
-           "pat_query_status"]
+           "pat_query_status", "pat_launch_count"]
 
 
 class PatError(RuntimeError):
@@ -56,6 +56,7 @@ def load() -> C.CDLL:
     L.pat_conv3x3.argtypes = [vp, i32, i32, vp, i32, i64, i32, vp, vp, i32, i32, i32, i32, vp]
     L.pat_conv3x3_dense.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp]
     L.pat_query_status.argtypes = [vp]
+    L.pat_launch_count.argtypes = []; L.pat_launch_count.restype = C.c_uint64
     _lib = L
     return L
 
@@ -163,3 +164,7 @@ def pat_query_status(stream=None) -> int:
     rc = load().pat_query_status(_stream(stream))
     _check(rc)
     return rc
+
+
+def pat_launch_count() -> int:
+    return int(load().pat_launch_count())

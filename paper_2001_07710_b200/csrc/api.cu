@@ -2,6 +2,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include "common.cuh"
 
 namespace pat {
@@ -24,6 +25,10 @@ int* status_word() {
 }
 
 static thread_local char t_last_error[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+uint64_t launches() { return g_launches.load(std::memory_order_relaxed); }
 
 int set_error(int code, const char* fmt, ...) {
   va_list ap;
@@ -73,6 +78,8 @@ const char* pat_strerror(int code) {
 }
 
 const char* pat_last_error(void) { return t_last_error; }
+
+uint64_t pat_launch_count(void) { return pat::launches(); }
 
 int pat_library_builtin(int K, uint16_t* masks_out) {
   // bit b = 3*r + s.  cross family | 2x2 blocks holding the centre | centre + opposite arms + corner

@@ -64,6 +64,9 @@ struct MaskTable {
 // Device address of the status word shared by all kernels of the library (nullptr on failure).
 int* status_word();
 
+// Host-side count of kernel launches (see pat_launch_count).
+void count_launches(int n);
+
 int set_error(int code, const char* fmt, ...);
 int check_library(const uint16_t* masks, int K);
 int check_cuda(cudaError_t e, const char* what);

@@ -222,6 +222,7 @@ int launch_sparse(const ConvArgs& a, const MaskTable& lib, cudaStream_t st) {
   if (int rc = prepare(k_conv_sparse_generic<T, STRIDE>, smem)) return rc;
   const dim3 grid((unsigned)((size_t)a.N * a.tiles_x * a.tiles_y), (unsigned)((a.F + FG - 1) / FG));
   k_conv_sparse_generic<T, STRIDE><<<grid, NWARP * 32, smem, st>>>(a, lib);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
 }
 
@@ -232,6 +233,7 @@ int launch_dense(const DenseArgs& a, cudaStream_t st) {
   if (int rc = prepare(k_conv_dense_small_c<T, STRIDE>, smem)) return rc;
   const dim3 grid((unsigned)((size_t)a.N * a.tiles_x * a.tiles_y), (unsigned)((a.F + FG - 1) / FG));
   k_conv_dense_small_c<T, STRIDE><<<grid, NWARP * 32, smem, st>>>(a);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_conv3x3_dense launch");
 }
 

@@ -249,6 +249,7 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   k_pack_ptrs<<<1, 1024, 0, st>>>(F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
   if (dtype == PAT_F16) k_pack_scatter<__half><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
   else k_pack_scatter<float><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+  count_launches(4);
   return check_cuda(cudaGetLastError(), "pat_pack launch");
 }
 
@@ -266,5 +267,6 @@ extern "C" int pat_unpack(const void* blob, int F, int C, const uint16_t* masks,
   if (int rc = check_cuda(cudaMemsetAsync(w_dense_out, 0, sizeof(float) * 9 * (size_t)F * C, st), "pat_unpack memset")) return rc;
   if (dtype == PAT_F16) k_unpack<__half><<<F, 128, 0, st>>>(bp, F, C, K, (long long)n_keep, dtype, lib, w_dense_out, status);
   else k_unpack<float><<<F, 128, 0, st>>>(bp, F, C, K, (long long)n_keep, dtype, lib, w_dense_out, status);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_unpack launch");
 }

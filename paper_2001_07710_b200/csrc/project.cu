@@ -236,5 +236,6 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
     k_tie_scan<<<1, 1024, 0, st>>>(ws.blk, nblk);
   }
   k_finalize<<<nblk, kSelBlock, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
+  count_launches(mode < 0 ? 13 : 2);
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
