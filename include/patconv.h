@@ -47,6 +47,7 @@ extern "C" {
 #define PAT_ERR_BLOB         6   /* packed blob does not match the arguments                  */
 #define PAT_ERR_CUDA         7   /* a CUDA runtime call failed                                */
 #define PAT_ERR_WORKSPACE    8   /* workspace or blob buffer too small                        */
+#define PAT_ERR_TIMEOUT      9   /* a bounded device-side wait expired (reported by pat_query_status) */
 
 #define PAT_F32 0                /* fp32 storage, fp32 accumulation                           */
 #define PAT_F16 1                /* fp16 storage (weights, activations), fp32 accumulation    */
@@ -140,7 +141,8 @@ int pat_conv3x3_dense(const float *w, int F, int C, int dtype, const void *x, vo
                       int N, int H, int W, int stride, void *stream);
 
 /* Synchronises `stream` and returns the device-side status word: PAT_OK, or PAT_ERR_BLOB when a
- * kernel found a blob header that did not match its arguments (the kernel then wrote nothing).
+ * kernel found a blob header that did not match its arguments (the kernel then wrote nothing),
+ * or PAT_ERR_TIMEOUT when a bounded wait inside a kernel expired (its output is then incomplete).
  * The word is cleared by the call. */
 int pat_query_status(void *stream);
 

@@ -73,6 +73,7 @@ const char* pat_strerror(int code) {
     case PAT_ERR_BLOB: return "blob does not match arguments";
     case PAT_ERR_CUDA: return "CUDA error";
     case PAT_ERR_WORKSPACE: return "buffer too small";
+    case PAT_ERR_TIMEOUT: return "device-side wait timed out";
     default: return "unknown error";
   }
 }

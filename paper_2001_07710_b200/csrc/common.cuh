@@ -11,6 +11,7 @@ namespace pat {
 constexpr uint32_t kBlobMagic = 0x50415443u;  // "PATC"
 constexpr uint32_t kBlobVersion = 1u;
 constexpr int kChanTile = 16;                 // granularity (input channels) of the execution section
+constexpr int kExecGroup = 32;                // filters per execution group (aligned groups of original filters)
 constexpr int kMaxK = 255;
 
 // First 256 bytes of every blob.
@@ -27,8 +28,8 @@ constexpr size_t kHeaderBytes = 768;
 // Byte offsets of every array in a blob; a pure function of (F, C, K, n_keep, dtype).
 struct BlobLayout {
   size_t perm, fptr, pptr, chan, w4;   // canonical section
-  size_t tptr, tmeta, tw4;             // execution section
-  size_t scratch;                      // pack-time temporaries: hist[F][K], count[F], inverse permutation[F]
+  size_t xfilt, tptr, tmeta, tw4;      // execution section (its own filter order, see pack.cu)
+  size_t scratch;                      // pack-time temporaries: hist[F][K], count[F], inv[F], xinv[F], xbase[F]
   size_t total;
   int nct;                             // number of 16-channel tiles = ceil(C / 16)
 };
@@ -47,10 +48,11 @@ __host__ __device__ inline BlobLayout blob_layout(int F, int C, int K, int64_t n
   L.pptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 1));
   L.chan = o;  o = align256(o + sizeof(uint16_t) * nk);
   L.w4 = o;    o = align256(o + 4 * e * nk);
+  L.xfilt = o; o = align256(o + sizeof(int32_t) * (size_t)F);
   L.tptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)L.nct + 1));
   L.tmeta = o; o = align256(o + sizeof(uint32_t) * nk);
   L.tw4 = o;   o = align256(o + 4 * e * nk);
-  L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 2));
+  L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 4));
   L.total = o;
   return L;
 }

@@ -4,6 +4,9 @@
 namespace pat {
 int conv_generic(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep, int dtype,
                  const void* x, void* y, int N, int H, int W, int stride, cudaStream_t st);
+bool conv_f16_fast_supported(int F, int C, const uint16_t* masks, int K, int dtype, int N, int H, int W, int stride);
+int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                  const void* x, void* y, int N, int H, int W, cudaStream_t st);
 }
 
 using namespace pat;
@@ -22,5 +25,7 @@ extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks
   const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
   if ((size_t)N * ((Ho + 7) / 8) * ((Wo + 31) / 32) > 0x7FFFFFFFull) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: too many tiles");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (conv_f16_fast_supported(F, C, masks, K, dtype, N, H, W, stride))
+    return conv_f16_fast(blob, F, C, masks, K, n_keep, x, y, N, H, W, st);
   return conv_generic(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, st);
 }

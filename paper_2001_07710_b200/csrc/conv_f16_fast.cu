@@ -1,0 +1,608 @@
+// Tuned sparse 3x3 convolution for fp16 storage / fp32 accumulation, stride 1 (sm_100a).
+//
+// What Section 6.2 asks of the execution code - one branch-free code path per pattern with the tap positions
+// known ahead of time, kernels of a filter grouped, filters balanced across thread groups - mapped to B200:
+//
+//  * persistent, warp-specialised thread blocks (one per SM): 16 consumer warps + 4 producer warps; the
+//    producers hand most of their registers to the consumers (setmaxnreg);
+//  * activations come from NHWC global memory by TMA (one tiled copy per tile row, 16 channels deep, zero
+//    fill outside the image = the padding), land as [row][pixel][16 ch], and are transposed by the producer
+//    warps (ldmatrix.trans -> stmatrix) into a channel-planar layout [ch][row][segment][16 px] in which every
+//    thread finds the 14 pixels of its tile row plus both halo pixels in two 16-byte loads;
+//  * a consumer thread owns a 2 x 14 pixel tile of R = 2 filters (56 fp32 accumulators); lanes of a warp are 32
+//    different tiles of the same filter, so weights are warp-uniform; the 16 warps cover 32 filters;
+//  * per kept kernel: the 4 x 16 pixel window of its channel is loaded once (8 x 16-byte loads); then, for each
+//    of the nine kernel positions, a warp-uniform test of the pattern mask guards fully unrolled code whose
+//    register offsets are immediates - nine tap bodies serve every pattern, so any library runs and the hot
+//    code stays inside the instruction cache; the multiply-adds are fma.rn.f32.f16 (fp16 x fp16 products are
+//    exact in fp32, the sum is fp32), so no conversion instruction sits in the loop;
+//  * channel blocks flow through a 3-deep planar ring and a 2-deep raw ring guarded by mbarriers, so warps
+//    with more kernels in one channel block catch up in the next; every wait is bounded;
+//  * the output of a work item goes through the same ring: two extra ring stages per item receive the fp16
+//    results (one row of every thread tile each) in a [pixel][32 channels] layout, and a store warp writes
+//    them to NHWC global memory as full 64-byte runs (the 32 adjacent output channels of the filter group).
+#include <cuda.h>
+#include <algorithm>
+#include "common.cuh"
+
+namespace pat {
+namespace fast16 {
+
+constexpr int TR = 2, TC = 14;          // pixel tile of a thread
+constexpr int LX = 4, LY = 8;           // tiles of a warp: 4 column slots x 8 tile rows
+constexpr int CB = kChanTile;           // channels per pipeline stage (16)
+constexpr int RF = 2;                   // filters per consumer warp
+constexpr int NCW = 16, NFW = 3, NSW = 1;  // consumer warps, fill (producer) warps, store warp
+constexpr int NPW = NFW + NSW;
+constexpr int FG = NCW * RF;            // filters per work item (32)
+static_assert(FG == kExecGroup, "a work item is one execution group of the blob");
+constexpr int PS = 3, RS = 2;           // planar / raw ring depth
+constexpr int NTHREADS = (NCW + NPW) * 32;
+constexpr int MAXROWS = LY * TR + 4;    // two bands, each with a top and a bottom halo row
+constexpr int SEGB = 32;                // bytes of a segment: 16 px (cols -1..14) of one channel
+constexpr int ROWB = LX * SEGB;         // 128
+constexpr int CHP = MAXROWS * ROWB + 16;  // channel plane pitch (odd multiple of 16 B: conflict-free stmatrix)
+constexpr int PLANAR_STAGE = CB * CHP;    // 41216
+constexpr int RAW_POS = 64;               // positions per raw row (58, 60 or 64 used)
+constexpr int RAW_ROWB = RAW_POS * CB * 2;  // 2048
+constexpr int RAW_STAGE = MAXROWS * RAW_ROWB;  // 40960
+// kernel descriptors of a stage: per filter slot a count, the original filter id, and up to 16 entries of
+// 16 bytes {channel-in-block | 4 tap codes << 4, taps 0-1 (fp16 x2), taps 2-3 (fp16 x2), unused}
+constexpr int DESC_HDR = FG * 8;
+constexpr int DESC_STAGE = DESC_HDR + FG * CB * 16;   // 8448
+constexpr int OFF_RAW = PS * PLANAR_STAGE;
+constexpr int OFF_DESC = OFF_RAW + RS * RAW_STAGE;
+constexpr int OFF_BAR = OFF_DESC + PS * DESC_STAGE;
+constexpr int SMEM_BYTES = OFF_BAR + 128;
+// output staging inside a planar slot: [448 pixels of a tile row set][32 channels] fp16, pixel pitch 68 bytes
+constexpr int OUT_PITCH = FG * 2 + 4;
+constexpr int OUT_PIX = 32 * TC;
+static_assert(OUT_PIX * OUT_PITCH <= PLANAR_STAGE, "a half tile of results fits one planar slot");
+static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
+// Register split between the warp groups.  The pool is what the block got at launch (threads x registers per
+// thread as compiled), so the split must fit inside it or the increase would wait forever; the host checks the
+// compiled count before launching.
+constexpr int LAUNCH_REGS = 96, CONSUMER_REGS = 104, PRODUCER_REGS = 64;
+static_assert(NCW * 32 * CONSUMER_REGS + NPW * 32 * PRODUCER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
+
+struct Params {
+  const __half* x;
+  __half* y;
+  const int32_t* xfilt;    // execution position -> original filter
+  const int32_t* tptr;     // [F][nct+1], execution order
+  const uint32_t* tmeta;   // channel | pattern << 16
+  const uint2* tw4;        // four fp16 taps per kernel
+  const BlobHeader* hdr;
+  int* status;
+  int N, H, W, C, F, K, nct;
+  long long n_keep;
+  int TY;                  // tile rows per image (H / 2)
+  int TXe, NI, BW;         // tile columns per region, images side by side, box width (pixels)
+  int CG, NIG;             // column groups per image, image groups
+  int NG;                  // filter groups (F / 32)
+  int n_items;             // regions * NG
+  int n_row_blocks;        // ceil(NIG * TY / LY)
+  uint16_t masks[256];     // the library (checked against the blob header)
+};
+
+// ------------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kWaitNs of wall time (or kSpinLimit polls), raises the block-wide abort flag
+// and returns false; also returns false as soon as another thread of the block has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(32);                      // leave the issue slots to the warps that have work
+    if ((spin & 15u) == 15u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitNs) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};"
+               ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void lds128(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t addr, unsigned short a) {
+  asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(a) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t a) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(a) : "memory");
+}
+__device__ __forceinline__ void fma_f32_f16(float& acc, unsigned short a, unsigned short b) {
+  asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(a), "h"(b));
+}
+__device__ __forceinline__ void split_h2(uint32_t v, unsigned short& lo, unsigned short& hi) {
+  asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(v));
+}
+
+// ------------------------------------------------------------------------------------------ work items
+// A work item = one region (8 tile rows x 4 column slots = 32 thread tiles) x one group of 32 filters.
+// Tile rows are numbered through all image groups (group g, tile row t -> g * TY + t), so a region may
+// straddle two image groups: it then has two bands, each with its own halo rows in shared memory.
+struct Item {
+  int g;            // filter group
+  int cg;           // column group
+  int ig0, ta0, n0; // band 0: image group, first tile row, number of tile rows
+  bool band1;       // band 1 exists (image group ig0 + 1, tile rows 0 .. LY - n0)
+  int nrows;        // shared-memory rows in use
+};
+
+__device__ __forceinline__ Item decode_item(const Params& p, int item) {
+  Item it;
+  it.g = item % p.NG;
+  const int reg = item / p.NG;
+  it.cg = reg % p.CG;
+  const int rb = reg / p.CG;
+  const int gt0 = rb * LY;
+  it.ig0 = gt0 / p.TY;
+  it.ta0 = gt0 % p.TY;
+  it.n0 = min(LY, p.TY - it.ta0);
+  it.band1 = (it.n0 < LY) && (it.ig0 + 1 < p.NIG);
+  it.nrows = it.band1 ? MAXROWS : 2 * it.n0 + 2;
+  return it;
+}
+
+// ------------------------------------------------------------------------------------------ consumer math
+// One tap of one kept kernel at kernel position B = 3*r + s:  acc[y][x] += w * in[y + r][x + s], where `in` is
+// the thread's (TR+2) x 16 window (row 0 / column 0 = the halo above / left of the tile).  B is a template
+// argument, so every register index below is fixed at compile time (Section 6.2: access code per pattern
+// position known ahead of time); the code of a tap is shared by all patterns that contain it.
+template <int B>
+__device__ __forceinline__ void tap_body(float (&acc)[TR][TC], const unsigned short (&h)[TR + 2][16], unsigned short w) {
+  constexpr int r = B / 3, s = B % 3;
+#pragma unroll
+  for (int y = 0; y < TR; ++y)
+#pragma unroll
+    for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[y + r][x + s], w);
+}
+
+// One kept kernel.  meta = channel-in-block | 9-bit pattern mask << 4; w01 / w23 = its four taps (fp16) in
+// ascending position order.  The mask test is warp-uniform (the whole warp works on the same kernel).
+__device__ __forceinline__ void one_kernel(float (&acc)[TR][TC], uint32_t baseA, uint32_t baseB, uint32_t meta,
+                                           uint32_t w01, uint32_t w23) {
+  unsigned short h[TR + 2][16];
+#pragma unroll
+  for (int i = 0; i < TR + 2; ++i) {       // window row i = image row (tile row + i - 1)
+    const int u = (i >> 1) & 1;            // physical chunk = logical chunk ^ u ^ lane swizzle
+    uint32_t q[8];
+    lds128((u ? baseB : baseA) + i * ROWB, q[0], q[1], q[2], q[3]);   // logical chunk 0: cols -1..6
+    lds128((u ? baseA : baseB) + i * ROWB, q[4], q[5], q[6], q[7]);   // logical chunk 1: cols 7..14
+#pragma unroll
+    for (int e = 0; e < 8; ++e) split_h2(q[e], h[i][2 * e], h[i][2 * e + 1]);
+  }
+#define PAT_TAP(B)                                                   \
+  if (meta & (16u << (B))) {                                         \
+    tap_body<B>(acc, h, (unsigned short)(w01 & 0xFFFFu));            \
+    w01 = __funnelshift_r(w01, w23, 16);                             \
+    w23 >>= 16;                                                      \
+  }
+  PAT_TAP(0) PAT_TAP(1) PAT_TAP(2) PAT_TAP(3) PAT_TAP(4) PAT_TAP(5) PAT_TAP(6) PAT_TAP(7) PAT_TAP(8)
+#undef PAT_TAP
+}
+
+// ------------------------------------------------------------------------------------------ the kernel
+// Ring protocol.  Every work item takes nct "real" ring stages (one channel block each) followed by two
+// "output" stages.  Stage number s uses planar slot s % PS in phase s / PS.
+//   real stage:    fill warps wait pl_empty, transpose + write descriptors, arrive pl_full (3 arrivals);
+//                  consumers wait pl_full, compute, arrive pl_empty (16 arrivals).
+//   output stage:  fill warps wait pl_empty and arrive pl_full at once (the slot is free to be written);
+//                  consumers wait pl_full, write one tile row of results, arrive out_ready (16 arrivals);
+//                  the store warp waits out_ready, copies the slot to global memory and arrives pl_empty
+//                  with a count of 16 in the consumers' place.
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ int s_abort;
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + OFF_BAR;
+  auto raw_full = [&](int s) { return bar0 + 8u * s; };
+  auto raw_empty = [&](int s) { return bar0 + 8u * (RS + s); };
+  auto pl_full = [&](int s) { return bar0 + 8u * (2 * RS + s); };
+  auto pl_empty = [&](int s) { return bar0 + 8u * (2 * RS + PS + s); };
+  auto out_ready = [&](int s) { return bar0 + 8u * (2 * RS + 2 * PS + s); };
+  static_assert(8 * (2 * RS + 3 * PS) <= 128, "barrier block");
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // refuse a blob packed with other parameters (uniform decision: every thread reads the same header)
+  {
+    const BlobHeader* h = p.hdr;
+    bool ok = h->magic == kBlobMagic && h->version == kBlobVersion && h->F == p.F && h->C == p.C &&
+              h->K == p.K && h->dtype == PAT_F16 && h->n_keep == p.n_keep;
+    for (int j = 0; ok && j < p.K; ++j) ok = h->masks[j] == p.masks[j];
+    if (!ok) {
+      if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
+      return;
+    }
+  }
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), NFW); }
+    for (int s = 0; s < PS; ++s) { mbar_init(pl_full(s), NFW); mbar_init(pl_empty(s), NCW); mbar_init(out_ready(s), NCW); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &s_abort;
+
+  const int n_my_items = (p.n_items > (int)blockIdx.x) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int nct = p.nct;
+  const int spi = nct + TR;                                  // ring stages per item
+  auto item_of = [&](int it_idx) { return decode_item(p, (int)blockIdx.x + it_idx * (int)gridDim.x); };
+
+  if (warp >= NCW) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PRODUCER_REGS));
+    if (warp < NCW + NFW) {
+      // ========================================================================= fill warps
+      const int pw = warp - NCW;
+      // lane constants of the transposition: lane -> (matrix m = lane / 8, row i = lane % 8) for both ld and st
+      const int m = lane >> 3, i8 = lane & 7;
+      const int hch = m >> 1, oct = m & 1;                     // pixel chunk (0/1), channel octet (0/1)
+      const uint32_t ld_lane = (uint32_t)((8 * hch + i8) * (CB * 2) + oct * 16);
+      const uint32_t st_lane = (uint32_t)((oct * 8 + i8) * CHP);
+      const int row_bytes = p.NI * p.BW * CB * 2;              // bytes one row copy brings in
+      const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+      // lane roles for the kernel descriptors: 3 lanes per filter slot over the 96 fill lanes
+      const int dslot = (pw * 32 + lane) / 3, dj = (pw * 32 + lane) % 3;
+      static_assert(NFW * 32 / 3 == FG, "three lanes per filter slot");
+
+      // all row copies of a stage: lane l of fill warp 0 issues the copy of shared-memory row l
+      auto issue_tma = [&](const Item& it, int cb, int slot) {
+        const uint32_t dst0 = sbase + OFF_RAW + slot * RAW_STAGE;
+        if (lane == 0) mbar_arrive_expect_tx(raw_full(slot), (uint32_t)(it.nrows * row_bytes));
+        __syncwarp();
+        if (lane < it.nrows) {
+          const int pr = lane;
+          const int b = (pr >= 2 * it.n0 + 2) ? 1 : 0;
+          const int yrow = b ? (pr - (2 * it.n0 + 2) - 1) : (2 * it.ta0 - 1 + pr);
+          tma_load_4d(dst0 + pr * RAW_ROWB, &tmap, cb * CB, it.cg * p.TXe * TC - 1, yrow, (it.ig0 + b) * p.NI, raw_full(slot));
+        }
+      };
+      static_assert(MAXROWS <= 32, "one lane per row copy");
+      // kernel range of this lane's filter slot in a channel block (global loads; prefetched one block ahead)
+      auto load_range = [&](int g, int cb, int& kb, int& ke) {
+        const int32_t* row = p.tptr + (size_t)(g * FG + dslot) * (nct + 1) + cb;
+        kb = __ldg(row); ke = __ldg(row + 1);
+      };
+
+      const int n_real = n_my_items * nct;         // real stages (raw ring positions)
+      int issued = 0, landed = 0;                  // real stages whose copies have been issued / have landed
+      int issue_it = 0, issue_cb = 0;              // (item, channel block) of the next copy to issue
+      Item issue_item = item_of(0);
+      auto issue_next = [&]() {
+        issue_tma(issue_item, issue_cb, issued % RS);
+        ++issued;
+        if (++issue_cb == nct) { issue_cb = 0; ++issue_it; if (issue_it < n_my_items) issue_item = item_of(issue_it); }
+      };
+      if (pw == 0)
+        for (int s = 0; s < RS && s < n_real; ++s) issue_next();
+
+      bool alive = true;
+      int stage = 0, rstage = 0;
+      int kb = 0, ke = 0;
+      for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
+        const Item it = item_of(it_idx);
+        if (dslot < FG) load_range(it.g, 0, kb, ke);
+        const int forig = (dslot < FG) ? __ldg(p.xfilt + it.g * FG + dslot) : 0;
+        for (int cb = 0; cb < nct && alive; ++cb, ++stage, ++rstage) {
+          const int rslot = rstage % RS, pslot = stage % PS;
+          // descriptors of this block: issue the global loads of the first entries now, use them after the transposition
+          const int nk = ke - kb, kb_cur = kb;
+          uint32_t dmeta = 0u;
+          uint2 dw = make_uint2(0u, 0u);
+          if (dj < nk) { dmeta = __ldg(p.tmeta + kb + dj); dw = __ldg(p.tw4 + kb + dj); }
+          if (cb + 1 < nct) load_range(it.g, cb + 1, kb, ke);
+
+          if (!mbar_wait(raw_full(rslot), (uint32_t)((rstage / RS) & 1), abort_flag)) { alive = false; break; }
+          landed = rstage + 1;
+          if (!mbar_wait(pl_empty(pslot), (uint32_t)(((stage / PS) & 1) ^ 1), abort_flag)) { alive = false; break; }
+          const uint32_t raw0 = sbase + OFF_RAW + rslot * RAW_STAGE;
+          const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
+          // transposition: op = (row, segment); four independent loads in flight before their stores
+          const int nops = it.nrows * LX;
+          for (int op0 = pw * 4; op0 < nops; op0 += NFW * 4) {
+            uint32_t v[4][4];
+            uint32_t dst[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int op = op0 + u;                 // nops is a multiple of 4: all four are valid
+              const int pr = op >> 2, seg = op & 3;
+              const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
+              const int j0 = ni * p.BW + TC * tx;     // raw position of image column 14*tx - 1
+              const int sw = (pr >> 1) & 1;
+              ldmatrix_x4_trans(raw0 + pr * RAW_ROWB + j0 * (CB * 2) + ld_lane, v[u][0], v[u][1], v[u][2], v[u][3]);
+              dst[u] = pl0 + pr * ROWB + seg * SEGB + ((hch ^ sw) << 4) + st_lane;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) stmatrix_x4(dst[u], v[u][0], v[u][1], v[u][2], v[u][3]);
+          }
+          // kernel descriptors
+          {
+            const uint32_t d0 = sbase + OFF_DESC + pslot * DESC_STAGE;
+            if (dj == 0) { sts32(d0 + dslot * 4, (uint32_t)nk); sts32(d0 + FG * 4 + dslot * 4, (uint32_t)forig); }
+            auto put = [&](int e, uint32_t mt, uint2 wv) {
+              const uint32_t cl = (mt & 0xFFFFu) - (uint32_t)(cb * CB);
+              const uint32_t mm = cl | ((uint32_t)p.masks[mt >> 16] << 4);
+              sts128(d0 + DESC_HDR + (dslot * CB + e) * 16, mm, wv.x, wv.y, 0u);
+            };
+            if (dj < nk) put(dj, dmeta, dw);
+            for (int e = dj + 3; e < nk; e += 3) put(e, __ldg(p.tmeta + kb_cur + e), __ldg(p.tw4 + kb_cur + e));   // rare
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(pl_full(pslot));
+            mbar_arrive(raw_empty(rslot));
+          }
+          if (pw == 0 && issued < n_real) {
+            // refill the raw slot once all fill warps have read it
+            if (!mbar_wait(raw_empty(rslot), (uint32_t)((rstage / RS) & 1), abort_flag)) alive = false;
+            else issue_next();
+          }
+        }
+        // output stages: hand the next TR slots to the consumers as they become free
+        for (int y = 0; y < TR && alive; ++y, ++stage) {
+          const int pslot = stage % PS;
+          if (!mbar_wait(pl_empty(pslot), (uint32_t)(((stage / PS) & 1) ^ 1), abort_flag)) { alive = false; break; }
+          if (lane == 0) mbar_arrive(pl_full(pslot));
+        }
+      }
+      if (!alive && pw == 0 && lane == 0) {
+        // copies already issued still write into this block's shared memory: give them (bounded) time to land
+        const unsigned long long t0 = global_ns();
+        for (int s = landed; s < issued; ++s)
+          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+            if (mbar_try_wait(raw_full(s % RS), (uint32_t)((s / RS) & 1))) break;
+            if (global_ns() - t0 > kWaitNs) break;
+          }
+        atomicExch(p.status, PAT_ERR_TIMEOUT);
+      }
+    } else {
+      // ========================================================================= store warp
+      uint32_t opar = 0;                           // phase parity of out_ready, one bit per planar slot
+      bool alive = true;
+      for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
+        const Item it = item_of(it_idx);
+        for (int y = 0; y < TR && alive; ++y) {
+          const int stage = it_idx * spi + nct + y;
+          const int pslot = stage % PS;
+          if (!mbar_wait(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
+          opar ^= 1u << pslot;
+          const uint32_t o0 = sbase + pslot * PLANAR_STAGE;
+          // 448 pixels x 4 chunks of 8 channels; consecutive lanes take consecutive chunks: 64-byte runs in global memory
+          for (int q = lane; q < OUT_PIX * 4; q += 32) {
+            const int pi = q >> 2, j = q & 3;
+            const int t = pi / TC, x = pi - t * TC;          // thread tile (= consumer lane) and column inside it
+            const int ly = t >> 2, lx = t & 3;
+            const int b = (ly < it.n0) ? 0 : 1;
+            const int ni = lx / p.TXe, tx = lx % p.TXe;
+            const int ig = it.ig0 + b;
+            const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+            const int n_img = ig * p.NI + ni;
+            if ((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) {
+              const uint32_t src = o0 + pi * OUT_PITCH + j * 16;
+              uint4 v;
+              v.x = lds32(src); v.y = lds32(src + 4); v.z = lds32(src + 8); v.w = lds32(src + 12);
+              const int col = (it.cg * p.TXe + tx) * TC + x;
+              __half* dst = p.y + (((size_t)n_img * p.H + (TR * ty + y)) * p.W + col) * p.F + it.g * FG + j * 8;
+              *reinterpret_cast<uint4*>(dst) = v;
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive_n(pl_empty(pslot), NCW);   // the slot goes back to the ring
+        }
+      }
+    }
+  } else {
+    // =========================================================================== consumer warps
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(CONSUMER_REGS));
+    const int ly = lane >> 2, lx = lane & 3;
+    int stage = 0;
+    bool alive = true;
+    for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
+      uint32_t offA, offB;               // the lane's two chunk addresses of window row 0, relative to a channel plane
+      {
+        const Item it = item_of(it_idx);
+        const int b = (ly < it.n0) ? 0 : 1;                  // band of this lane's tile row
+        const uint32_t lane_off = (uint32_t)((2 * ly + 2 * b) * ROWB + lx * SEGB);
+        const int swl = (ly + b) & 1;
+        offA = lane_off + (uint32_t)(swl << 4);
+        offB = lane_off + (uint32_t)((swl ^ 1) << 4);
+      }
+      float acc[RF][TR][TC];
+#pragma unroll
+      for (int r = 0; r < RF; ++r)
+#pragma unroll
+        for (int y = 0; y < TR; ++y)
+#pragma unroll
+          for (int x = 0; x < TC; ++x) acc[r][y][x] = 0.0f;
+      uint32_t cpos[RF] = {0u, 0u};      // byte offset of each filter inside its group of 32 output channels
+
+      for (int cb = 0; cb < nct; ++cb, ++stage) {
+        const int pslot = stage % PS;
+        if (!mbar_wait(pl_full(pslot), (uint32_t)((stage / PS) & 1), abort_flag)) { alive = false; break; }
+        const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
+        const uint32_t d0 = sbase + OFF_DESC + pslot * DESC_STAGE;
+#pragma unroll
+        for (int r = 0; r < RF; ++r) {
+          // warp w takes slots w and 31 - w: the most loaded filter of the group with the least loaded one, ...
+          const int slot = (r == 0) ? warp : FG - 1 - warp;
+          const int nk = (int)lds32(d0 + slot * 4);
+          if (cb == nct - 1) cpos[r] = (lds32(d0 + FG * 4 + slot * 4) & (uint32_t)(FG - 1)) * 2u;
+          uint32_t e = d0 + DESC_HDR + slot * CB * 16;
+          for (int k = 0; k < nk; ++k, e += 16) {
+            uint32_t m0, w01, w23, pad;
+            lds128(e, m0, w01, w23, pad);
+            const uint32_t base = pl0 + (m0 & 15u) * CHP;
+            one_kernel(acc[r], base + offA, base + offB, m0, w01, w23);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pl_empty(pslot));
+      }
+      if (!alive) break;
+
+      // results: fp32 -> fp16 (round to nearest even) into the two output stages, one tile row each
+#pragma unroll
+      for (int y = 0; y < TR; ++y, ++stage) {
+        const int pslot = stage % PS;
+        if (!mbar_wait(pl_full(pslot), (uint32_t)((stage / PS) & 1), abort_flag)) { alive = false; break; }
+        const uint32_t o0 = sbase + pslot * PLANAR_STAGE + (uint32_t)(lane * TC) * OUT_PITCH;
+#pragma unroll
+        for (int r = 0; r < RF; ++r)
+#pragma unroll
+          for (int x = 0; x < TC; ++x)
+            sts16(o0 + x * OUT_PITCH + cpos[r], __half_as_ushort(__float2half_rn(acc[r][y][x])));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(out_ready(pslot));
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+}  // namespace fast16
+
+// True when the tuned kernel covers this layer.
+bool conv_f16_fast_supported(int F, int C, const uint16_t* masks, int K, int dtype, int N, int H, int W, int stride) {
+  using namespace fast16;
+  if (dtype != PAT_F16 || stride != 1) return false;
+  if (W % TC != 0 || H % TR != 0 || H < 2 * (LY - 1)) return false;
+  const int TX = W / TC;
+  if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
+  if (C % CB != 0 || F % FG != 0) return false;
+  (void)N; (void)masks; (void)K;
+  return encode_fn() != nullptr;
+}
+
+int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                  const void* x, void* y, int N, int H, int W, cudaStream_t st) {
+  using namespace fast16;
+  const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F16);
+  const char* b = static_cast<const char*>(blob);
+  Params p;
+  p.x = static_cast<const __half*>(x);
+  p.y = static_cast<__half*>(y);
+  p.hdr = reinterpret_cast<const BlobHeader*>(b);
+  p.tptr = reinterpret_cast<const int32_t*>(b + L.tptr);
+  p.tmeta = reinterpret_cast<const uint32_t*>(b + L.tmeta);
+  p.tw4 = reinterpret_cast<const uint2*>(b + L.tw4);
+  p.xfilt = reinterpret_cast<const int32_t*>(b + L.xfilt);
+  p.status = status_word();
+  if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
+  p.N = N; p.H = H; p.W = W; p.C = C; p.F = F; p.K = K; p.nct = L.nct; p.n_keep = n_keep;
+  p.TY = H / TR;
+  const int TX = W / TC;
+  p.TXe = TX >= LX ? LX : TX;
+  p.NI = LX / p.TXe;
+  p.BW = p.TXe * TC + 2;
+  p.CG = TX / p.TXe;
+  p.NIG = (N + p.NI - 1) / p.NI;
+  p.NG = F / FG;
+  p.n_row_blocks = (int)(((long long)p.NIG * p.TY + LY - 1) / LY);
+  const long long items = (long long)p.n_row_blocks * p.CG * p.NG;
+  if (items > 0x7FFFFFFFll) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: too many work items");
+  p.n_items = (int)items;
+  for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
+
+  CUtensorMap tm;
+  const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)CB, (cuuint32_t)p.BW, 1u, (cuuint32_t)p.NI};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult cr = encode_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cuTensorMapEncodeTiled failed (%d)", (int)cr);
+
+  static thread_local int sm_count = 0;
+  static thread_local bool attr_set = false;
+  if (!attr_set) {
+    int dev = 0;
+    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
+    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
+    if (int rc = check_cuda(cudaFuncSetAttribute(k_conv_f16_s1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
+    cudaFuncAttributes fa;
+    if (int rc = check_cuda(cudaFuncGetAttributes(&fa, k_conv_f16_s1), "query kernel attributes")) return rc;
+    if (fa.numRegs < LAUNCH_REGS)
+      return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
+    attr_set = true;
+  }
+  const int grid = (int)std::min<long long>(items, sm_count);
+  k_conv_f16_s1<<<grid, NTHREADS, SMEM_BYTES, st>>>(tm, p);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
+}
+
+}  // namespace pat

@@ -246,7 +246,7 @@ int conv_generic(const void* blob, int F, int C, const uint16_t* masks, int K, i
   ConvArgs a;
   a.x = x; a.y = y;
   a.hdr = reinterpret_cast<const BlobHeader*>(b);
-  a.perm = reinterpret_cast<const int32_t*>(b + L.perm);
+  a.perm = reinterpret_cast<const int32_t*>(b + L.xfilt);   // execution order of the filters
   a.tptr = reinterpret_cast<const int32_t*>(b + L.tptr);
   a.tmeta = reinterpret_cast<const uint32_t*>(b + L.tmeta);
   a.tw4 = b + L.tw4;

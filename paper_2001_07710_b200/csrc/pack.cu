@@ -4,7 +4,10 @@
 // group) and groups, inside each filter, the kernels that share a pattern (one code path per group, no
 // branches inside it).  The blob holds a canonical section in exactly that order and an execution section in
 // which each filter's kernels are re-sorted by blocks of 16 input channels (the unit in which the convolution
-// kernels stage activations), then pattern, then channel.
+// kernels stage activations), then pattern, then channel.  The execution section has its own filter order:
+// filters stay inside their aligned group of 32 original filters (so that a thread block that owns a group
+// writes 32 adjacent output channels) and are sorted inside the group by kept-kernel count, descending, so
+// that pairing position i with position 31 - i gives every warp the same amount of work.
 #include "common.cuh"
 
 namespace pat {
@@ -15,10 +18,11 @@ struct BlobPtrs {
   int32_t *perm, *fptr, *pptr;
   uint16_t* chan;
   void* w4;
+  int32_t* xfilt;      // execution position -> original filter
   int32_t* tptr;
   uint32_t* tmeta;
   void* tw4;
-  int32_t *hist, *cnt, *inv;
+  int32_t *hist, *cnt, *inv, *xinv, *xbase;
 };
 
 __host__ __device__ inline BlobPtrs blob_ptrs(void* blob, const BlobLayout& L, int F, int K) {
@@ -30,12 +34,15 @@ __host__ __device__ inline BlobPtrs blob_ptrs(void* blob, const BlobLayout& L, i
   p.pptr = reinterpret_cast<int32_t*>(b + L.pptr);
   p.chan = reinterpret_cast<uint16_t*>(b + L.chan);
   p.w4 = b + L.w4;
+  p.xfilt = reinterpret_cast<int32_t*>(b + L.xfilt);
   p.tptr = reinterpret_cast<int32_t*>(b + L.tptr);
   p.tmeta = reinterpret_cast<uint32_t*>(b + L.tmeta);
   p.tw4 = b + L.tw4;
   p.hist = reinterpret_cast<int32_t*>(b + L.scratch);
   p.cnt = p.hist + (size_t)F * K;
   p.inv = p.cnt + F;
+  p.xinv = p.inv + F;
+  p.xbase = p.xinv + F;
   return p;
 }
 
@@ -83,6 +90,15 @@ __global__ void k_pack_rank(int F, int K, BlobPtrs bp) {
   }
   bp.perm[rank] = f;
   bp.inv[f] = rank;
+  // execution order: inside the aligned group of 32 original filters, by kept count (descending), then index
+  const int g0 = (f / kExecGroup) * kExecGroup, g1 = min(F, g0 + kExecGroup);
+  int xr = g0;
+  for (int g = g0; g < g1; ++g) {
+    const int ng = bp.cnt[g];
+    xr += (ng > nf || (ng == nf && g < f)) ? 1 : 0;
+  }
+  bp.xfilt[xr] = f;
+  bp.xinv[f] = xr;
 }
 
 // One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
@@ -115,9 +131,30 @@ __global__ void __launch_bounds__(1024) k_pack_ptrs(int F, int C, int K, long lo
     if (threadIdx.x == 1023) carry += part[1023];
     __syncthreads();
   }
+  // same scan in execution order
+  const int total = carry;
+  __syncthreads();
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < F; base += 1024) {
+    const int e = base + threadIdx.x;
+    const int v = (e < F) ? bp.cnt[bp.xfilt[e]] : 0;
+    part[threadIdx.x] = v;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+      const int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0;
+      __syncthreads();
+      part[threadIdx.x] += a;
+      __syncthreads();
+    }
+    if (e < F) bp.xbase[e] = carry + part[threadIdx.x] - v;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry += part[1023];
+    __syncthreads();
+  }
   if (threadIdx.x == 0) {
-    bp.fptr[F] = carry;
-    const bool ok = (long long)carry == n_keep;
+    bp.fptr[F] = total;
+    const bool ok = (long long)total == n_keep;
     if (!ok) atomicExch(status, PAT_ERR_BLOB);
     BlobHeader* h = bp.hdr;
     h->magic = ok ? kBlobMagic : 0u;
@@ -142,13 +179,14 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
   const int q = bp.inv[f];
   for (int c = threadIdx.x; c < C; c += blockDim.x) spid[c] = pid[(size_t)f * C + c];
   __syncthreads();
-  const int f0 = bp.fptr[q];
+  const int xe = bp.xinv[f];
+  const int f0 = bp.xbase[xe];
   // execution-section pointers: kernels of this filter before channel tile t
   for (int t = threadIdx.x; t <= nct; t += blockDim.x) {
     int n = 0;
     const int cend = min(t * kChanTile, C);
     for (int c = 0; c < cend; ++c) n += (spid[c] != PAT_PRUNED) ? 1 : 0;
-    bp.tptr[(size_t)q * (nct + 1) + t] = f0 + n;
+    bp.tptr[(size_t)xe * (nct + 1) + t] = f0 + n;
   }
   T* w4 = static_cast<T*>(bp.w4);
   T* tw4 = static_cast<T*>(bp.tw4);

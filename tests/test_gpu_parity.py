@@ -133,6 +133,40 @@ def test_conv_matches_oracle(case, dtype):
         assert not y.any()
 
 
+# Shapes that take the tuned fp16 kernel (W multiple of 14, even H >= 14, C % 16 == 0, F % 32 == 0): regions that
+# straddle two images, images packed side by side (W = 14, 28), batch sizes that leave image slots empty,
+# several column groups (W = 112), all three library sizes.
+TUNED_CASES = [
+    (5, 14, 14, 64, 32, 8, 1, 8),
+    (3, 28, 28, 32, 64, 12, 1, 4),
+    (3, 56, 56, 32, 32, 8, 1, 8),
+    (1, 18, 56, 16, 32, 4, 1, 2),
+    (2, 30, 112, 48, 64, 8, 3, 10),
+    (1, 224, 224, 16, 32, 8, 1, 8),
+    (7, 16, 14, 16, 32, 8, 1, 1),
+    (2, 14, 28, 256, 32, 8, 1, 8),
+]
+
+
+@pytest.mark.parametrize("case", TUNED_CASES)
+def test_conv_tuned_f16_matches_oracle(case):
+    N, H, W, C, F, K, num, den = case
+    rng = np.random.default_rng(hash(case) % (2 ** 32))
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, "f16"), x, 1)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    y = torch.full((N, H, W, F), float("nan"), dtype=torch.float16, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y)
+    assert pc.pat_query_status() == 0
+    out = y.float().cpu().numpy()
+    assert np.isfinite(out).all()                                   # every output element was written
+    check_close(out, ref, "f16")
+
+
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
 @pytest.mark.parametrize("N,H,W,C,F,stride", [(2, 40, 70, 3, 64, 1), (1, 9, 9, 1, 8, 1), (2, 17, 33, 3, 40, 2), (1, 16, 16, 16, 32, 1)])
 def test_dense_conv_matches_oracle(N, H, W, C, F, stride, dtype):
