@@ -11,10 +11,10 @@
 //    thread finds the 14 pixels of its tile row plus both halo pixels in two 16-byte loads;
 //  * a consumer thread owns a 2 x 14 pixel tile of R = 2 filters (56 fp32 accumulators); lanes of a warp are 32
 //    different tiles of the same filter, so weights are warp-uniform; the 16 warps cover 32 filters;
-//  * per kept kernel: the 4 x 16 pixel window of its channel is loaded once (8 x 16-byte loads); then, for each
-//    of the nine kernel positions, a warp-uniform test of the pattern mask guards fully unrolled code whose
-//    register offsets are immediates - nine tap bodies serve every pattern, so any library runs and the hot
-//    code stays inside the instruction cache; the multiply-adds are fma.rn.f32.f16 (fp16 x fp16 products are
+//  * per kept kernel: the 16-pixel-wide window of its channel is loaded with 16-byte loads, then one
+//    warp-uniform jump on the pattern selects fully unrolled code whose register offsets are immediates
+//    (patterns that are a built-in pattern shifted down one row share its code; other libraries run through
+//    nine guarded per-position bodies); the multiply-adds are fma.rn.f32.f16 (fp16 x fp16 products are
 //    exact in fp32, the sum is fp32), so no conversion instruction sits in the loop;
 //  * channel blocks flow through a 3-deep planar ring and a 2-deep raw ring guarded by mbarriers, so warps
 //    with more kernels in one channel block catch up in the next; every wait is bounded;
@@ -85,6 +85,7 @@ struct Params {
   int n_items;             // regions * NG
   int n_row_blocks;        // ceil(NIG * TY / LY)
   uint16_t masks[256];     // the library (checked against the blob header)
+  uint32_t pword[256];     // pattern id -> descriptor word (mask, compiled code, window shift)
 };
 
 // ------------------------------------------------------------------------------------------ PTX helpers
@@ -123,7 +124,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   const unsigned long long t0 = global_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(32);                      // leave the issue slots to the warps that have work
     if ((spin & 15u) == 15u) {
       if (*abort_flag) return false;
       if (global_ns() - t0 > kWaitNs) break;
@@ -210,28 +210,89 @@ __device__ __forceinline__ void tap_body(float (&acc)[TR][TC], const unsigned sh
     for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[y + r][x + s], w);
 }
 
-// One kept kernel.  meta = channel-in-block | 9-bit pattern mask << 4; w01 / w23 = its four taps (fp16) in
-// ascending position order.  The mask test is warp-uniform (the whole warp works on the same kernel).
+// Compiled pattern codes.  A pattern whose top row is empty is the same shape one row lower, so it runs the
+// code of the shifted-up pattern on a window that starts one row lower: the twelve built-in patterns need ten
+// codes (the eight patterns of Section 4.2 need six).  Any other pattern takes the generic code (kGenericCode).
+constexpr int kNumCodes = 10;
+constexpr int kGenericCode = 15;
+__host__ __device__ constexpr uint32_t code_mask(int i) {
+  constexpr uint32_t m[kNumCodes] = {0x03A, 0x017, 0x0B2, 0x09A, 0x01B, 0x036, 0x093, 0x03C, 0x192, 0x00F};
+  return m[i];
+}
+__host__ __device__ constexpr int nth_bit(uint32_t mask, int t) {
+  int seen = 0;
+  for (int b = 0; b < 9; ++b)
+    if (mask & (1u << b)) { if (seen == t) return b; ++seen; }
+  return 4;
+}
+
+// descriptor word: bits 0-3 channel inside the block, 4-12 pattern mask, 13-16 code, 17 window row shift
+__host__ __device__ inline uint32_t pattern_word(uint32_t mask) {
+  const uint32_t shift = (mask & 7u) == 0u ? 1u : 0u;
+  const uint32_t norm = mask >> (3u * shift);
+  uint32_t code = kGenericCode;
+  for (int i = 0; i < kNumCodes; ++i)
+    if (code_mask(i) == norm) code = (uint32_t)i;
+  if (code == (uint32_t)kGenericCode) return (mask << 4) | (code << 13);
+  return (mask << 4) | (code << 13) | (shift << 17);
+}
+
+__device__ __forceinline__ void load_row(unsigned short (&hrow)[16], uint32_t a0, uint32_t a1) {
+  uint32_t q[8];
+  lds128(a0, q[0], q[1], q[2], q[3]);   // logical chunk 0: cols -1..6
+  lds128(a1, q[4], q[5], q[6], q[7]);   // logical chunk 1: cols 7..14
+#pragma unroll
+  for (int e = 0; e < 8; ++e) split_h2(q[e], hrow[2 * e], hrow[2 * e + 1]);
+}
+
+template <uint32_t MASK>
+__device__ __forceinline__ void pattern_body(float (&acc)[TR][TC], const unsigned short (&h)[TR + 2][16], uint32_t w01, uint32_t w23) {
+  unsigned short w0, w1, w2, w3;
+  split_h2(w01, w0, w1);
+  split_h2(w23, w2, w3);
+  tap_body<nth_bit(MASK, 0)>(acc, h, w0);
+  tap_body<nth_bit(MASK, 1)>(acc, h, w1);
+  tap_body<nth_bit(MASK, 2)>(acc, h, w2);
+  tap_body<nth_bit(MASK, 3)>(acc, h, w3);
+}
+
+// One kept kernel.  meta = descriptor word (see pattern_word); w01 / w23 = its four taps (fp16) in ascending
+// position order; baseA / baseB = the lane's two chunk addresses of window row 0 in the kernel's channel plane.
+// The switch is warp-uniform (the whole warp works on the same kernel).
 __device__ __forceinline__ void one_kernel(float (&acc)[TR][TC], uint32_t baseA, uint32_t baseB, uint32_t meta,
                                            uint32_t w01, uint32_t w23) {
+  static_assert(TR == 2, "window addressing below is written for two-row tiles");
   unsigned short h[TR + 2][16];
-#pragma unroll
-  for (int i = 0; i < TR + 2; ++i) {       // window row i = image row (tile row + i - 1)
-    const int u = (i >> 1) & 1;            // physical chunk = logical chunk ^ u ^ lane swizzle
-    uint32_t q[8];
-    lds128((u ? baseB : baseA) + i * ROWB, q[0], q[1], q[2], q[3]);   // logical chunk 0: cols -1..6
-    lds128((u ? baseA : baseB) + i * ROWB, q[4], q[5], q[6], q[7]);   // logical chunk 1: cols 7..14
-#pragma unroll
-    for (int e = 0; e < 8; ++e) split_h2(q[e], h[i][2 * e], h[i][2 * e + 1]);
-  }
+  // window rows shift .. shift+2 (physical chunk = logical chunk ^ ((row >> 1) & 1) ^ lane swizzle)
+  const uint32_t sh = (meta >> 17) & 1u;
+  const uint32_t rb = sh * ROWB;
+  load_row(h[0], baseA + rb, baseB + rb);                                   // row 0 or 1: u = 0
+  load_row(h[1], (sh ? baseB : baseA) + rb + ROWB, (sh ? baseA : baseB) + rb + ROWB);   // row 1 (u = 0) or 2 (u = 1)
+  load_row(h[2], baseB + rb + 2 * ROWB, baseA + rb + 2 * ROWB);             // row 2 or 3: u = 1
+  switch ((meta >> 13) & 15u) {
+    case 0: pattern_body<code_mask(0)>(acc, h, w01, w23); break;
+    case 1: pattern_body<code_mask(1)>(acc, h, w01, w23); break;
+    case 4: pattern_body<code_mask(4)>(acc, h, w01, w23); break;
+    case 5: pattern_body<code_mask(5)>(acc, h, w01, w23); break;
+    case 7: pattern_body<code_mask(7)>(acc, h, w01, w23); break;
+    case 9: pattern_body<code_mask(9)>(acc, h, w01, w23); break;
+    case 2: load_row(h[3], baseB + 3 * ROWB, baseA + 3 * ROWB); pattern_body<code_mask(2)>(acc, h, w01, w23); break;
+    case 3: load_row(h[3], baseB + 3 * ROWB, baseA + 3 * ROWB); pattern_body<code_mask(3)>(acc, h, w01, w23); break;
+    case 6: load_row(h[3], baseB + 3 * ROWB, baseA + 3 * ROWB); pattern_body<code_mask(6)>(acc, h, w01, w23); break;
+    case 8: load_row(h[3], baseB + 3 * ROWB, baseA + 3 * ROWB); pattern_body<code_mask(8)>(acc, h, w01, w23); break;
+    default: {
+      // any other pattern: a warp-uniform test of each of the nine positions guards the code of that position
+      load_row(h[3], baseB + 3 * ROWB, baseA + 3 * ROWB);
 #define PAT_TAP(B)                                                   \
   if (meta & (16u << (B))) {                                         \
     tap_body<B>(acc, h, (unsigned short)(w01 & 0xFFFFu));            \
     w01 = __funnelshift_r(w01, w23, 16);                             \
     w23 >>= 16;                                                      \
   }
-  PAT_TAP(0) PAT_TAP(1) PAT_TAP(2) PAT_TAP(3) PAT_TAP(4) PAT_TAP(5) PAT_TAP(6) PAT_TAP(7) PAT_TAP(8)
+      PAT_TAP(0) PAT_TAP(1) PAT_TAP(2) PAT_TAP(3) PAT_TAP(4) PAT_TAP(5) PAT_TAP(6) PAT_TAP(7) PAT_TAP(8)
 #undef PAT_TAP
+    } break;
+  }
 }
 
 // ------------------------------------------------------------------------------------------ the kernel
@@ -247,10 +308,10 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ int s_abort;
+  __shared__ int s_rawdone[RS];          // fill warps that have finished reading a raw slot
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = sbase + OFF_BAR;
   auto raw_full = [&](int s) { return bar0 + 8u * s; };
-  auto raw_empty = [&](int s) { return bar0 + 8u * (RS + s); };
   auto pl_full = [&](int s) { return bar0 + 8u * (2 * RS + s); };
   auto pl_empty = [&](int s) { return bar0 + 8u * (2 * RS + PS + s); };
   auto out_ready = [&](int s) { return bar0 + 8u * (2 * RS + 2 * PS + s); };
@@ -272,7 +333,7 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); mbar_init(raw_empty(s), NFW); }
+    for (int s = 0; s < RS; ++s) { mbar_init(raw_full(s), 1); s_rawdone[s] = 0; }
     for (int s = 0; s < PS; ++s) { mbar_init(pl_full(s), NFW); mbar_init(pl_empty(s), NCW); mbar_init(out_ready(s), NCW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -281,94 +342,100 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
 
   const int n_my_items = (p.n_items > (int)blockIdx.x) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const int nct = p.nct;
-  const int spi = nct + TR;                                  // ring stages per item
   auto item_of = [&](int it_idx) { return decode_item(p, (int)blockIdx.x + it_idx * (int)gridDim.x); };
 
   if (warp >= NCW) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PRODUCER_REGS));
+    const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
     if (warp < NCW + NFW) {
       // ========================================================================= fill warps
+      // These warps share the issue slots of their SM partition with four consumer warps, so every instruction
+      // here is paid for with multiply-add slots: ring positions are kept incrementally, addresses are lane
+      // constants plus small per-row terms, and item geometry is decoded once per item.
       const int pw = warp - NCW;
       // lane constants of the transposition: lane -> (matrix m = lane / 8, row i = lane % 8) for both ld and st
       const int m = lane >> 3, i8 = lane & 7;
       const int hch = m >> 1, oct = m & 1;                     // pixel chunk (0/1), channel octet (0/1)
-      const uint32_t ld_lane = (uint32_t)((8 * hch + i8) * (CB * 2) + oct * 16);
+      uint32_t ldoff[LX];                                      // per segment: raw offset of the lane's matrix row
+#pragma unroll
+      for (int seg = 0; seg < LX; ++seg) {
+        const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
+        ldoff[seg] = (uint32_t)((ni * p.BW + TC * tx + 8 * hch + i8) * (CB * 2) + oct * 16);
+      }
       const uint32_t st_lane = (uint32_t)((oct * 8 + i8) * CHP);
+      const uint32_t stoff0 = st_lane + (uint32_t)(hch << 4), stoff1 = st_lane + (uint32_t)((hch ^ 1) << 4);
       const int row_bytes = p.NI * p.BW * CB * 2;              // bytes one row copy brings in
-      const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
       // lane roles for the kernel descriptors: 3 lanes per filter slot over the 96 fill lanes
       const int dslot = (pw * 32 + lane) / 3, dj = (pw * 32 + lane) % 3;
       static_assert(NFW * 32 / 3 == FG, "three lanes per filter slot");
+      static_assert(MAXROWS <= 32, "one lane per row copy");
 
-      // all row copies of a stage: lane l of fill warp 0 issues the copy of shared-memory row l
-      auto issue_tma = [&](const Item& it, int cb, int slot) {
-        const uint32_t dst0 = sbase + OFF_RAW + slot * RAW_STAGE;
-        if (lane == 0) mbar_arrive_expect_tx(raw_full(slot), (uint32_t)(it.nrows * row_bytes));
-        __syncwarp();
-        if (lane < it.nrows) {
-          const int pr = lane;
-          const int b = (pr >= 2 * it.n0 + 2) ? 1 : 0;
-          const int yrow = b ? (pr - (2 * it.n0 + 2) - 1) : (2 * it.ta0 - 1 + pr);
-          tma_load_4d(dst0 + pr * RAW_ROWB, &tmap, cb * CB, it.cg * p.TXe * TC - 1, yrow, (it.ig0 + b) * p.NI, raw_full(slot));
+      // Issue cursor: the (item, channel block) whose copies go out next; it runs RS real stages ahead of the
+      // stage being transposed.  Lane l holds the coordinates of shared-memory row l of the cursor's item.
+      int cur_it = 0, cur_cb = 0, cur_y = 0, cur_n = 0, cur_x = 0, cur_rows = 0;
+      auto cursor_load = [&]() {
+        if (cur_it < n_my_items) {
+          const Item ci = item_of(cur_it);
+          const int b = (lane >= 2 * ci.n0 + 2) ? 1 : 0;
+          cur_y = b ? (lane - (2 * ci.n0 + 2) - 1) : (2 * ci.ta0 - 1 + lane);
+          cur_n = (ci.ig0 + b) * p.NI;
+          cur_x = ci.cg * p.TXe * TC - 1;
+          cur_rows = ci.nrows;
         }
       };
-      static_assert(MAXROWS <= 32, "one lane per row copy");
+      auto cursor_advance = [&]() {
+        if (++cur_cb == nct) { cur_cb = 0; ++cur_it; cursor_load(); }
+      };
+      auto cursor_issue = [&](int slot) {                     // whole warp: lane l copies row l
+        if (lane == 0) mbar_arrive_expect_tx(raw_full(slot), (uint32_t)(cur_rows * row_bytes));
+        __syncwarp();
+        if (lane < cur_rows)
+          tma_load_4d(sbase + OFF_RAW + slot * RAW_STAGE + lane * RAW_ROWB, &tmap, cur_cb * CB, cur_x, cur_y, cur_n, raw_full(slot));
+      };
+      const int n_real = n_my_items * nct;         // real stages (raw ring positions)
+      cursor_load();
+      for (int s = 0; s < RS && s < n_real; ++s) {   // prologue: fill warp 0 issues, every warp advances its cursor
+        if (pw == 0) cursor_issue(s);
+        cursor_advance();
+      }
       // kernel range of this lane's filter slot in a channel block (global loads; prefetched one block ahead)
       auto load_range = [&](int g, int cb, int& kb, int& ke) {
         const int32_t* row = p.tptr + (size_t)(g * FG + dslot) * (nct + 1) + cb;
         kb = __ldg(row); ke = __ldg(row + 1);
       };
 
-      const int n_real = n_my_items * nct;         // real stages (raw ring positions)
-      int issued = 0, landed = 0;                  // real stages whose copies have been issued / have landed
-      int issue_it = 0, issue_cb = 0;              // (item, channel block) of the next copy to issue
-      Item issue_item = item_of(0);
-      auto issue_next = [&]() {
-        issue_tma(issue_item, issue_cb, issued % RS);
-        ++issued;
-        if (++issue_cb == nct) { issue_cb = 0; ++issue_it; if (issue_it < n_my_items) issue_item = item_of(issue_it); }
-      };
-      if (pw == 0)
-        for (int s = 0; s < RS && s < n_real; ++s) issue_next();
-
       bool alive = true;
-      int stage = 0, rstage = 0;
+      int rstage = 0, landed = 0;                  // real stages done / whose copies this warp has seen land
+      int pslot = 0, rslot = 0;
+      uint32_t ppar = 1u, rpar = 0u;               // parity to wait for: pl_empty of the slot, raw_full of the raw slot
       int kb = 0, ke = 0;
       for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
-        const Item it = item_of(it_idx);
-        if (dslot < FG) load_range(it.g, 0, kb, ke);
-        const int forig = (dslot < FG) ? __ldg(p.xfilt + it.g * FG + dslot) : 0;
-        for (int cb = 0; cb < nct && alive; ++cb, ++stage, ++rstage) {
-          const int rslot = rstage % RS, pslot = stage % PS;
+        int g, nrows;
+        { const Item it = item_of(it_idx); g = it.g; nrows = it.nrows; }
+        load_range(g, 0, kb, ke);
+        const int forig = __ldg(p.xfilt + g * FG + dslot);
+        for (int cb = 0; cb < nct && alive; ++cb, ++rstage) {
           // descriptors of this block: issue the global loads of the first entries now, use them after the transposition
           const int nk = ke - kb, kb_cur = kb;
           uint32_t dmeta = 0u;
           uint2 dw = make_uint2(0u, 0u);
           if (dj < nk) { dmeta = __ldg(p.tmeta + kb + dj); dw = __ldg(p.tw4 + kb + dj); }
-          if (cb + 1 < nct) load_range(it.g, cb + 1, kb, ke);
+          if (cb + 1 < nct) load_range(g, cb + 1, kb, ke);
 
-          if (!mbar_wait(raw_full(rslot), (uint32_t)((rstage / RS) & 1), abort_flag)) { alive = false; break; }
+          if (!mbar_wait(raw_full(rslot), rpar, abort_flag)) { alive = false; break; }
           landed = rstage + 1;
-          if (!mbar_wait(pl_empty(pslot), (uint32_t)(((stage / PS) & 1) ^ 1), abort_flag)) { alive = false; break; }
+          if (!mbar_wait(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
           const uint32_t raw0 = sbase + OFF_RAW + rslot * RAW_STAGE;
           const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
-          // transposition: op = (row, segment); four independent loads in flight before their stores
-          const int nops = it.nrows * LX;
-          for (int op0 = pw * 4; op0 < nops; op0 += NFW * 4) {
-            uint32_t v[4][4];
-            uint32_t dst[4];
+          // transposition, one shared-memory row (4 segments) at a time: four independent loads, then their stores
+          for (int pr = pw; pr < nrows; pr += NFW) {
+            const uint32_t lr = raw0 + pr * RAW_ROWB;
+            const uint32_t sr = pl0 + pr * ROWB + ((pr & 2) ? stoff1 : stoff0);   // chunk swizzle by (row >> 1) & 1
+            uint32_t v[LX][4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int op = op0 + u;                 // nops is a multiple of 4: all four are valid
-              const int pr = op >> 2, seg = op & 3;
-              const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
-              const int j0 = ni * p.BW + TC * tx;     // raw position of image column 14*tx - 1
-              const int sw = (pr >> 1) & 1;
-              ldmatrix_x4_trans(raw0 + pr * RAW_ROWB + j0 * (CB * 2) + ld_lane, v[u][0], v[u][1], v[u][2], v[u][3]);
-              dst[u] = pl0 + pr * ROWB + seg * SEGB + ((hch ^ sw) << 4) + st_lane;
-            }
+            for (int seg = 0; seg < LX; ++seg) ldmatrix_x4_trans(lr + ldoff[seg], v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) stmatrix_x4(dst[u], v[u][0], v[u][1], v[u][2], v[u][3]);
+            for (int seg = 0; seg < LX; ++seg) stmatrix_x4(sr + seg * SEGB, v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
           }
           // kernel descriptors
           {
@@ -376,34 +443,39 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
             if (dj == 0) { sts32(d0 + dslot * 4, (uint32_t)nk); sts32(d0 + FG * 4 + dslot * 4, (uint32_t)forig); }
             auto put = [&](int e, uint32_t mt, uint2 wv) {
               const uint32_t cl = (mt & 0xFFFFu) - (uint32_t)(cb * CB);
-              const uint32_t mm = cl | ((uint32_t)p.masks[mt >> 16] << 4);
+              const uint32_t mm = cl | p.pword[mt >> 16];
               sts128(d0 + DESC_HDR + (dslot * CB + e) * 16, mm, wv.x, wv.y, 0u);
             };
             if (dj < nk) put(dj, dmeta, dw);
             for (int e = dj + 3; e < nk; e += 3) put(e, __ldg(p.tmeta + kb_cur + e), __ldg(p.tw4 + kb_cur + e));   // rare
           }
           __syncwarp();
+          // the fill warp that is last to finish with the raw slot refills it
+          int last = 0;
           if (lane == 0) {
             mbar_arrive(pl_full(pslot));
-            mbar_arrive(raw_empty(rslot));
+            last = (atomicAdd(&s_rawdone[rslot], 1) == NFW - 1) ? 1 : 0;
+            if (last) s_rawdone[rslot] = 0;
           }
-          if (pw == 0 && issued < n_real) {
-            // refill the raw slot once all fill warps have read it
-            if (!mbar_wait(raw_empty(rslot), (uint32_t)((rstage / RS) & 1), abort_flag)) alive = false;
-            else issue_next();
+          last = __shfl_sync(0xFFFFFFFFu, last, 0);
+          if (rstage + RS < n_real) {
+            if (last) cursor_issue(rslot);
+            cursor_advance();
           }
+          if (++pslot == PS) { pslot = 0; ppar ^= 1u; }
+          if (++rslot == RS) { rslot = 0; rpar ^= 1u; }
         }
         // output stages: hand the next TR slots to the consumers as they become free
-        for (int y = 0; y < TR && alive; ++y, ++stage) {
-          const int pslot = stage % PS;
-          if (!mbar_wait(pl_empty(pslot), (uint32_t)(((stage / PS) & 1) ^ 1), abort_flag)) { alive = false; break; }
+        for (int y = 0; y < TR && alive; ++y) {
+          if (!mbar_wait(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
           if (lane == 0) mbar_arrive(pl_full(pslot));
+          if (++pslot == PS) { pslot = 0; ppar ^= 1u; }
         }
       }
       if (!alive && pw == 0 && lane == 0) {
         // copies already issued still write into this block's shared memory: give them (bounded) time to land
         const unsigned long long t0 = global_ns();
-        for (int s = landed; s < issued; ++s)
+        for (int s = landed; s < landed + RS && s < n_real; ++s)   // issued or not: a copy that was issued lands long before the limit
           for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
             if (mbar_try_wait(raw_full(s % RS), (uint32_t)((s / RS) & 1))) break;
             if (global_ns() - t0 > kWaitNs) break;
@@ -414,35 +486,42 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
       // ========================================================================= store warp
       uint32_t opar = 0;                           // phase parity of out_ready, one bit per planar slot
       bool alive = true;
+      int pslot = 0;
       for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
         const Item it = item_of(it_idx);
+        pslot = (pslot + nct) % PS;                // skip the real stages of the item
         for (int y = 0; y < TR && alive; ++y) {
-          const int stage = it_idx * spi + nct + y;
-          const int pslot = stage % PS;
           if (!mbar_wait(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
           opar ^= 1u << pslot;
           const uint32_t o0 = sbase + pslot * PLANAR_STAGE;
-          // 448 pixels x 4 chunks of 8 channels; consecutive lanes take consecutive chunks: 64-byte runs in global memory
-          for (int q = lane; q < OUT_PIX * 4; q += 32) {
-            const int pi = q >> 2, j = q & 3;
-            const int t = pi / TC, x = pi - t * TC;          // thread tile (= consumer lane) and column inside it
+          // one thread tile (= one consumer lane) at a time: 14 pixels x 4 chunks of 8 channels; consecutive lanes
+          // take consecutive chunks, so every pixel is written as one 64-byte run
+          for (int t = 0; t < 32; ++t) {
             const int ly = t >> 2, lx = t & 3;
             const int b = (ly < it.n0) ? 0 : 1;
-            const int ni = lx / p.TXe, tx = lx % p.TXe;
+            const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
             const int ig = it.ig0 + b;
             const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
             const int n_img = ig * p.NI + ni;
-            if ((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) {
-              const uint32_t src = o0 + pi * OUT_PITCH + j * 16;
-              uint4 v;
-              v.x = lds32(src); v.y = lds32(src + 4); v.z = lds32(src + 8); v.w = lds32(src + 12);
-              const int col = (it.cg * p.TXe + tx) * TC + x;
-              __half* dst = p.y + (((size_t)n_img * p.H + (TR * ty + y)) * p.W + col) * p.F + it.g * FG + j * 8;
-              *reinterpret_cast<uint4*>(dst) = v;
+            if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
+            const int col0 = (it.cg * p.TXe + tx) * TC;
+            __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR * ty + y)) * p.W + col0) * p.F + it.g * FG;
+            const uint32_t src_tile = o0 + (uint32_t)(t * TC) * OUT_PITCH;
+#pragma unroll
+            for (int q0 = 0; q0 < TC * 4; q0 += 32) {
+              const int q = q0 + lane;
+              if (q < TC * 4) {
+                const int x = q >> 2, j = q & 3;
+                const uint32_t src = src_tile + x * OUT_PITCH + j * 16;
+                uint4 v;
+                v.x = lds32(src); v.y = lds32(src + 4); v.z = lds32(src + 8); v.w = lds32(src + 12);
+                *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = v;
+              }
             }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive_n(pl_empty(pslot), NCW);   // the slot goes back to the ring
+          if (++pslot == PS) pslot = 0;
         }
       }
     }
@@ -450,7 +529,10 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
     // =========================================================================== consumer warps
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(CONSUMER_REGS));
     const int ly = lane >> 2, lx = lane & 3;
-    int stage = 0;
+    // warp w takes filter slots w and 31 - w of the group: the most loaded filter with the least loaded one, ...
+    const uint32_t slot_off[RF] = {(uint32_t)warp, (uint32_t)(FG - 1 - warp)};
+    int pslot = 0;
+    uint32_t fpar = 0u;                    // parity to wait for on pl_full of the current slot
     bool alive = true;
     for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
       uint32_t offA, offB;               // the lane's two chunk addresses of window row 0, relative to a channel plane
@@ -471,18 +553,15 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
           for (int x = 0; x < TC; ++x) acc[r][y][x] = 0.0f;
       uint32_t cpos[RF] = {0u, 0u};      // byte offset of each filter inside its group of 32 output channels
 
-      for (int cb = 0; cb < nct; ++cb, ++stage) {
-        const int pslot = stage % PS;
-        if (!mbar_wait(pl_full(pslot), (uint32_t)((stage / PS) & 1), abort_flag)) { alive = false; break; }
+      for (int cb = 0; cb < nct; ++cb) {
+        if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
         const uint32_t d0 = sbase + OFF_DESC + pslot * DESC_STAGE;
 #pragma unroll
         for (int r = 0; r < RF; ++r) {
-          // warp w takes slots w and 31 - w: the most loaded filter of the group with the least loaded one, ...
-          const int slot = (r == 0) ? warp : FG - 1 - warp;
-          const int nk = (int)lds32(d0 + slot * 4);
-          if (cb == nct - 1) cpos[r] = (lds32(d0 + FG * 4 + slot * 4) & (uint32_t)(FG - 1)) * 2u;
-          uint32_t e = d0 + DESC_HDR + slot * CB * 16;
+          const int nk = (int)lds32(d0 + slot_off[r] * 4);
+          if (cb == nct - 1) cpos[r] = (lds32(d0 + FG * 4 + slot_off[r] * 4) & (uint32_t)(FG - 1)) * 2u;
+          uint32_t e = d0 + DESC_HDR + slot_off[r] * (CB * 16);
           for (int k = 0; k < nk; ++k, e += 16) {
             uint32_t m0, w01, w23, pad;
             lds128(e, m0, w01, w23, pad);
@@ -492,14 +571,14 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(pl_empty(pslot));
+        if (++pslot == PS) { pslot = 0; fpar ^= 1u; }
       }
       if (!alive) break;
 
       // results: fp32 -> fp16 (round to nearest even) into the two output stages, one tile row each
 #pragma unroll
-      for (int y = 0; y < TR; ++y, ++stage) {
-        const int pslot = stage % PS;
-        if (!mbar_wait(pl_full(pslot), (uint32_t)((stage / PS) & 1), abort_flag)) { alive = false; break; }
+      for (int y = 0; y < TR; ++y) {
+        if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t o0 = sbase + pslot * PLANAR_STAGE + (uint32_t)(lane * TC) * OUT_PITCH;
 #pragma unroll
         for (int r = 0; r < RF; ++r)
@@ -508,6 +587,7 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
             sts16(o0 + x * OUT_PITCH + cpos[r], __half_as_ushort(__float2half_rn(acc[r][y][x])));
         __syncwarp();
         if (lane == 0) mbar_arrive(out_ready(pslot));
+        if (++pslot == PS) { pslot = 0; fpar ^= 1u; }
       }
     }
   }
@@ -574,7 +654,10 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
   const long long items = (long long)p.n_row_blocks * p.CG * p.NG;
   if (items > 0x7FFFFFFFll) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: too many work items");
   p.n_items = (int)items;
-  for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
+  for (int j = 0; j < 256; ++j) {
+    p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
+    p.pword[j] = (j < K) ? pattern_word(masks[j]) : 0u;
+  }
 
   CUtensorMap tm;
   const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};

@@ -167,6 +167,25 @@ def test_conv_tuned_f16_matches_oracle(case):
     check_close(out, ref, "f16")
 
 
+def test_conv_tuned_f16_arbitrary_library():
+    """Masks outside the built-in set (some without the centre) run through the per-position code of the tuned kernel."""
+    N, H, W, C, F = 3, 28, 28, 48, 64
+    masks = np.array([0b000001111, 0b111100000, 0b101000101, 0b010101010 & 0x1FF | 0, 0x03A, 0x0D8, 0b100110001], dtype=np.uint16)
+    masks = np.array([m for m in masks if bin(int(m)).count("1") == 4], dtype=np.uint16)
+    assert len(masks) >= 6
+    rng = np.random.default_rng(77)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
+    n_keep = F * C // 4
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, "f16"), x, 1)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1)
+    assert pc.pat_query_status() == 0
+    check_close(y.float().cpu().numpy(), ref, "f16")
+
+
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
 @pytest.mark.parametrize("N,H,W,C,F,stride", [(2, 40, 70, 3, 64, 1), (1, 9, 9, 1, 8, 1), (2, 17, 33, 3, 40, 2), (1, 16, 16, 16, 32, 1)])
 def test_dense_conv_matches_oracle(N, H, W, C, F, stride, dtype):
