@@ -44,8 +44,8 @@ constexpr int ROWB = LX * SEGB;         // 128
 constexpr int CHP = MAXROWS * ROWB + 16;  // channel plane pitch (odd multiple of 16 B: conflict-free stmatrix)
 constexpr int PLANAR_STAGE = CB * CHP;    // 41216
 constexpr int RAW_POS = 64;               // positions per raw row (58, 60 or 64 used)
-constexpr int RAW_ROWB = RAW_POS * CB * 2;  // 2048
-constexpr int RAW_STAGE = MAXROWS * RAW_ROWB;  // 40960
+constexpr int RAW_STAGE = MAXROWS * RAW_POS * CB * 2;  // 40960
+constexpr int NMAPS = LY;                 // one tensor map per band height (2n + 2 rows, n = 1..8 tile rows)
 // kernel descriptors of a stage: per filter slot a count, the original filter id, and up to 16 entries of
 // 16 bytes {channel-in-block | 4 tap codes << 4, taps 0-1 (fp16 x2), taps 2-3 (fp16 x2), unused}
 constexpr int DESC_HDR = FG * 8;
@@ -66,6 +66,11 @@ constexpr int LAUNCH_REGS = 96, CONSUMER_REGS = 104, PRODUCER_REGS = 64;
 static_assert(NCW * 32 * CONSUMER_REGS + NPW * 32 * PRODUCER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
+constexpr uint32_t kSuspendNs = 100000u;                // longest stay inside one try_wait (0.1 ms)
+
+// One tiled copy brings a whole band (all its rows, all images side by side), because issuing a copy costs far
+// more than the copy engine needs per row; the box height is part of a tensor map, hence one map per height.
+struct alignas(64) TmapSet { CUtensorMap m[NMAPS]; };
 
 struct Params {
   const __half* x;
@@ -112,6 +117,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Same test, but the thread may stay suspended inside the instruction for up to `ns` nanoseconds while the
+// phase is incomplete: a waiting warp then issues next to nothing, which matters here because waiting warps
+// share their issue slots with the warps that are doing the multiply-adds.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -123,11 +140,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 15u) == 15u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitNs) break;
-    }
+    if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitNs) break;
   }
   *abort_flag = 1;
   return false;
@@ -305,7 +320,7 @@ __device__ __forceinline__ void one_kernel(float (&acc)[TR][TC], uint32_t baseA,
 //                  the store warp waits out_ready, copies the slot to global memory and arrives pl_empty
 //                  with a count of 16 in the consumers' place.
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
+k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ int s_abort;
   __shared__ int s_rawdone[RS];          // fill warps that have finished reading a raw slot
@@ -356,11 +371,13 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
       // lane constants of the transposition: lane -> (matrix m = lane / 8, row i = lane % 8) for both ld and st
       const int m = lane >> 3, i8 = lane & 7;
       const int hch = m >> 1, oct = m & 1;                     // pixel chunk (0/1), channel octet (0/1)
-      uint32_t ldoff[LX];                                      // per segment: raw offset of the lane's matrix row
+      // raw layout of a band: [image slot][row][pixel -1 .. BW-2][16 channels]
+      const uint32_t rowpitch = (uint32_t)(p.BW * CB * 2);
+      uint32_t ldoff[LX];                                      // per segment: offset of the lane's matrix row inside a raw row
 #pragma unroll
       for (int seg = 0; seg < LX; ++seg) {
-        const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
-        ldoff[seg] = (uint32_t)((ni * p.BW + TC * tx + 8 * hch + i8) * (CB * 2) + oct * 16);
+        const int tx = seg & (p.TXe - 1);
+        ldoff[seg] = (uint32_t)((TC * tx + 8 * hch + i8) * (CB * 2) + oct * 16);
       }
       const uint32_t st_lane = (uint32_t)((oct * 8 + i8) * CHP);
       const uint32_t stoff0 = st_lane + (uint32_t)(hch << 4), stoff1 = st_lane + (uint32_t)((hch ^ 1) << 4);
@@ -371,26 +388,28 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
       static_assert(MAXROWS <= 32, "one lane per row copy");
 
       // Issue cursor: the (item, channel block) whose copies go out next; it runs RS real stages ahead of the
-      // stage being transposed.  Lane l holds the coordinates of shared-memory row l of the cursor's item.
-      int cur_it = 0, cur_cb = 0, cur_y = 0, cur_n = 0, cur_x = 0, cur_rows = 0;
+      // stage being transposed.  Lane 0 holds the coordinates of band 0 of the cursor's item, lane 1 those of band 1.
+      int cur_it = 0, cur_cb = 0, cur_y = 0, cur_n = 0, cur_x = 0, cur_rows = 0, cur_map = -1;
+      uint32_t cur_dst = 0;
       auto cursor_load = [&]() {
         if (cur_it < n_my_items) {
           const Item ci = item_of(cur_it);
-          const int b = (lane >= 2 * ci.n0 + 2) ? 1 : 0;
-          cur_y = b ? (lane - (2 * ci.n0 + 2) - 1) : (2 * ci.ta0 - 1 + lane);
-          cur_n = (ci.ig0 + b) * p.NI;
-          cur_x = ci.cg * p.TXe * TC - 1;
+          const int rows0 = 2 * ci.n0 + 2;
           cur_rows = ci.nrows;
+          cur_x = ci.cg * p.TXe * TC - 1;
+          cur_map = -1;
+          if (lane == 0) { cur_y = 2 * ci.ta0 - 1; cur_n = ci.ig0 * p.NI; cur_dst = 0u; cur_map = ci.n0 - 1; }
+          if (lane == 1 && ci.band1) { cur_y = -1; cur_n = (ci.ig0 + 1) * p.NI; cur_dst = (uint32_t)(p.NI * rows0) * rowpitch; cur_map = LY - ci.n0 - 1; }
         }
       };
       auto cursor_advance = [&]() {
         if (++cur_cb == nct) { cur_cb = 0; ++cur_it; cursor_load(); }
       };
-      auto cursor_issue = [&](int slot) {                     // whole warp: lane l copies row l
+      auto cursor_issue = [&](int slot) {                     // whole warp: lanes 0 and 1 each copy one band
         if (lane == 0) mbar_arrive_expect_tx(raw_full(slot), (uint32_t)(cur_rows * row_bytes));
         __syncwarp();
-        if (lane < cur_rows)
-          tma_load_4d(sbase + OFF_RAW + slot * RAW_STAGE + lane * RAW_ROWB, &tmap, cur_cb * CB, cur_x, cur_y, cur_n, raw_full(slot));
+        if (cur_map >= 0)
+          tma_load_4d(sbase + OFF_RAW + slot * RAW_STAGE + cur_dst, &tms.m[cur_map], cur_cb * CB, cur_x, cur_y, cur_n, raw_full(slot));
       };
       const int n_real = n_my_items * nct;         // real stages (raw ring positions)
       cursor_load();
@@ -410,8 +429,16 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
       uint32_t ppar = 1u, rpar = 0u;               // parity to wait for: pl_empty of the slot, raw_full of the raw slot
       int kb = 0, ke = 0;
       for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
-        int g, nrows;
-        { const Item it = item_of(it_idx); g = it.g; nrows = it.nrows; }
+        int g, nrows, rows0;
+        { const Item it = item_of(it_idx); g = it.g; nrows = it.nrows; rows0 = 2 * it.n0 + 2; }
+        // per band: where image slot ni of the band starts in the raw buffer (segments of a row may belong to different slots)
+        uint32_t nioff[2][LX];
+#pragma unroll
+        for (int seg = 0; seg < LX; ++seg) {
+          const uint32_t ni = (uint32_t)(seg >> txe_shift);
+          nioff[0][seg] = ni * (uint32_t)rows0 * rowpitch + ldoff[seg];
+          nioff[1][seg] = (uint32_t)(p.NI * rows0) * rowpitch + ni * (uint32_t)(nrows - rows0) * rowpitch + ldoff[seg];
+        }
         load_range(g, 0, kb, ke);
         const int forig = __ldg(p.xfilt + g * FG + dslot);
         for (int cb = 0; cb < nct && alive; ++cb, ++rstage) {
@@ -429,11 +456,13 @@ k_conv_f16_s1(const __grid_constant__ CUtensorMap tmap, const Params p) {
           const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
           // transposition, one shared-memory row (4 segments) at a time: four independent loads, then their stores
           for (int pr = pw; pr < nrows; pr += NFW) {
-            const uint32_t lr = raw0 + pr * RAW_ROWB;
+            const bool b1 = pr >= rows0;
+            const uint32_t lr = raw0 + (uint32_t)(b1 ? pr - rows0 : pr) * rowpitch;
             const uint32_t sr = pl0 + pr * ROWB + ((pr & 2) ? stoff1 : stoff0);   // chunk swizzle by (row >> 1) & 1
             uint32_t v[LX][4];
 #pragma unroll
-            for (int seg = 0; seg < LX; ++seg) ldmatrix_x4_trans(lr + ldoff[seg], v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
+            for (int seg = 0; seg < LX; ++seg)
+              ldmatrix_x4_trans(lr + (b1 ? nioff[1][seg] : nioff[0][seg]), v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
 #pragma unroll
             for (int seg = 0; seg < LX; ++seg) stmatrix_x4(sr + seg * SEGB, v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
           }
@@ -659,15 +688,17 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
     p.pword[j] = (j < K) ? pattern_word(masks[j]) : 0u;
   }
 
-  CUtensorMap tm;
+  TmapSet tm;
   const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
   const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-  const cuuint32_t box[4] = {(cuuint32_t)CB, (cuuint32_t)p.BW, 1u, (cuuint32_t)p.NI};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  const CUresult cr = encode_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (cr != CUDA_SUCCESS) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cuTensorMapEncodeTiled failed (%d)", (int)cr);
+  for (int n = 1; n <= NMAPS; ++n) {          // band of n tile rows: 2n rows + a halo row above and below
+    const cuuint32_t box[4] = {(cuuint32_t)CB, (cuuint32_t)p.BW, (cuuint32_t)(TR * n + 2), (cuuint32_t)p.NI};
+    const CUresult cr = encode_fn()(&tm.m[n - 1], CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cuTensorMapEncodeTiled failed (%d)", (int)cr);
+  }
 
   static thread_local int sm_count = 0;
   static thread_local bool attr_set = false;
