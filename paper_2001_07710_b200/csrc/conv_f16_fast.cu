@@ -64,6 +64,7 @@ static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 // compiled count before launching.
 constexpr int LAUNCH_REGS = 96, CONSUMER_REGS = 104, PRODUCER_REGS = 64;
 static_assert(NCW * 32 * CONSUMER_REGS + NPW * 32 * PRODUCER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
+constexpr uint32_t TMEM_COLS = 256;        // 4 consumer warps per lane quarter x 2 filters x 32 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
 constexpr uint32_t kSuspendNs = 100000u;                // longest stay inside one try_wait (0.1 ms)
@@ -182,6 +183,48 @@ __device__ __forceinline__ void fma_f32_f16(float& acc, unsigned short a, unsign
 }
 __device__ __forceinline__ void split_h2(uint32_t v, unsigned short& lo, unsigned short& hi) {
   asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(v));
+}
+
+// ---- tensor memory (256 KB per SM, 128 lanes x 512 columns of 32 bits).  No tensor-core instruction is used
+// here: the memory only parks the accumulators of the filter a warp is not working on, so that the per-pattern
+// code exists once (for one set of accumulator registers) and stays inside the instruction cache.  A warp may
+// touch the 32 lanes of its own quarter (warp index % 4); thread i of the warp reads / writes lane i.
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {      // whole warp; ncols: power of two >= 32
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {         // whole warp
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// 32 consecutive columns of the thread's lane <-> 32 registers (28 accumulators + 4 unused)
+__device__ __forceinline__ void tmem_store32(uint32_t taddr, const float (&a)[TR][TC]) {
+  static_assert(TR * TC == 28, "accumulator tile is 28 values");
+  const float z = 0.0f;
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%29,%29,%29};\n\t"
+      "tcgen05.wait::st.sync.aligned;"
+      ::"r"(taddr),
+        "f"(a[0][0]), "f"(a[0][1]), "f"(a[0][2]), "f"(a[0][3]), "f"(a[0][4]), "f"(a[0][5]), "f"(a[0][6]),
+        "f"(a[0][7]), "f"(a[0][8]), "f"(a[0][9]), "f"(a[0][10]), "f"(a[0][11]), "f"(a[0][12]), "f"(a[0][13]),
+        "f"(a[1][0]), "f"(a[1][1]), "f"(a[1][2]), "f"(a[1][3]), "f"(a[1][4]), "f"(a[1][5]), "f"(a[1][6]),
+        "f"(a[1][7]), "f"(a[1][8]), "f"(a[1][9]), "f"(a[1][10]), "f"(a[1][11]), "f"(a[1][12]), "f"(a[1][13]),
+        "f"(z)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&a)[TR][TC]) {
+  float d0, d1, d2, d3;
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=f"(a[0][0]), "=f"(a[0][1]), "=f"(a[0][2]), "=f"(a[0][3]), "=f"(a[0][4]), "=f"(a[0][5]), "=f"(a[0][6]),
+        "=f"(a[0][7]), "=f"(a[0][8]), "=f"(a[0][9]), "=f"(a[0][10]), "=f"(a[0][11]), "=f"(a[0][12]), "=f"(a[0][13]),
+        "=f"(a[1][0]), "=f"(a[1][1]), "=f"(a[1][2]), "=f"(a[1][3]), "=f"(a[1][4]), "=f"(a[1][5]), "=f"(a[1][6]),
+        "=f"(a[1][7]), "=f"(a[1][8]), "=f"(a[1][9]), "=f"(a[1][10]), "=f"(a[1][11]), "=f"(a[1][12]), "=f"(a[1][13]),
+        "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+      : "r"(taddr)
+      : "memory");
 }
 
 // ------------------------------------------------------------------------------------------ work items
@@ -323,6 +366,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ int s_abort;
+  __shared__ uint32_t s_tmem;            // base address of the block's tensor-memory columns
   __shared__ int s_rawdone[RS];          // fill warps that have finished reading a raw slot
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = sbase + OFF_BAR;
@@ -352,8 +396,12 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
     for (int s = 0; s < PS; ++s) { mbar_init(pl_full(s), NFW); mbar_init(pl_empty(s), NCW); mbar_init(out_ready(s), NCW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 0) tmem_alloc(smem_u32(&s_tmem), TMEM_COLS);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   volatile int* abort_flag = &s_abort;
+  const uint32_t tmem_base = s_tmem;
 
   const int n_my_items = (p.n_items > (int)blockIdx.x) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const int nct = p.nct;
@@ -558,8 +606,10 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
     // =========================================================================== consumer warps
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(CONSUMER_REGS));
     const int ly = lane >> 2, lx = lane & 3;
-    // warp w takes filter slots w and 31 - w of the group: the most loaded filter with the least loaded one, ...
-    const uint32_t slot_off[RF] = {(uint32_t)warp, (uint32_t)(FG - 1 - warp)};
+    // Warp w owns filter slots w and 31 - w of the group (the most loaded filter with the least loaded one, ...).
+    // Only one of the two accumulator tiles is in registers at a time; the other is parked in tensor memory:
+    // columns [64 * (w / 4) + 32 * f, +32) of the lanes of quarter w % 4.
+    const uint32_t tm0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 64);
     int pslot = 0;
     uint32_t fpar = 0u;                    // parity to wait for on pl_full of the current slot
     bool alive = true;
@@ -573,29 +623,43 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         offA = lane_off + (uint32_t)(swl << 4);
         offB = lane_off + (uint32_t)((swl ^ 1) << 4);
       }
-      float acc[RF][TR][TC];
+      float acc[TR][TC];
 #pragma unroll
-      for (int r = 0; r < RF; ++r)
+      for (int y = 0; y < TR; ++y)
 #pragma unroll
-        for (int y = 0; y < TR; ++y)
-#pragma unroll
-          for (int x = 0; x < TC; ++x) acc[r][y][x] = 0.0f;
-      uint32_t cpos[RF] = {0u, 0u};      // byte offset of each filter inside its group of 32 output channels
+        for (int x = 0; x < TC; ++x) acc[y][x] = 0.0f;
+      tmem_store32(tm0 + 32u, acc);      // filter 1 starts from zero in tensor memory, filter 0 in registers
+      uint32_t cur = 0u;                 // which of the two filters the registers hold
 
+      // the kernels of filter f in the current stage
+      auto run_filter = [&](uint32_t f, uint32_t pl0, uint32_t d0) {
+        const uint32_t slot = f ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp;
+        const int nk = (int)lds32(d0 + slot * 4);
+        uint32_t e = d0 + DESC_HDR + slot * (CB * 16);
+        for (int k = 0; k < nk; ++k, e += 16) {
+          uint32_t m0, w01, w23, pad;
+          lds128(e, m0, w01, w23, pad);
+          const uint32_t base = pl0 + (m0 & 15u) * CHP;
+          one_kernel(acc, base + offA, base + offB, m0, w01, w23);
+        }
+      };
+
+      uint32_t cposA = 0u, cposB = 0u;   // byte offsets of filters 0 / 1 inside the group of 32 output channels
       for (int cb = 0; cb < nct; ++cb) {
         if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
         const uint32_t d0 = sbase + OFF_DESC + pslot * DESC_STAGE;
-#pragma unroll
-        for (int r = 0; r < RF; ++r) {
-          const int nk = (int)lds32(d0 + slot_off[r] * 4);
-          if (cb == nct - 1) cpos[r] = (lds32(d0 + FG * 4 + slot_off[r] * 4) & (uint32_t)(FG - 1)) * 2u;
-          uint32_t e = d0 + DESC_HDR + slot_off[r] * (CB * 16);
-          for (int k = 0; k < nk; ++k, e += 16) {
-            uint32_t m0, w01, w23, pad;
-            lds128(e, m0, w01, w23, pad);
-            const uint32_t base = pl0 + (m0 & 15u) * CHP;
-            one_kernel(acc[r], base + offA, base + offB, m0, w01, w23);
+        if (cb == nct - 1) {
+          cposA = (lds32(d0 + FG * 4 + (uint32_t)warp * 4) & (uint32_t)(FG - 1)) * 2u;
+          cposB = (lds32(d0 + FG * 4 + (uint32_t)(FG - 1 - warp) * 4) & (uint32_t)(FG - 1)) * 2u;
+        }
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          run_filter(cur, pl0, d0);
+          if (half == 0) {               // swap: park this filter, fetch the other
+            tmem_store32(tm0 + cur * 32u, acc);
+            cur ^= 1u;
+            tmem_load32(tm0 + cur * 32u, acc);
           }
         }
         __syncwarp();
@@ -605,21 +669,36 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
       if (!alive) break;
 
       // results: fp32 -> fp16 (round to nearest even) into the two output stages, one tile row each
-#pragma unroll
+#pragma unroll 1
       for (int y = 0; y < TR; ++y) {
         if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t o0 = sbase + pslot * PLANAR_STAGE + (uint32_t)(lane * TC) * OUT_PITCH;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t cp = cur ? cposB : cposA;
+          if (y == 0) {
 #pragma unroll
-        for (int r = 0; r < RF; ++r)
+            for (int x = 0; x < TC; ++x) sts16(o0 + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[0][x])));
+          } else {
 #pragma unroll
-          for (int x = 0; x < TC; ++x)
-            sts16(o0 + x * OUT_PITCH + cpos[r], __half_as_ushort(__float2half_rn(acc[r][y][x])));
+            for (int x = 0; x < TC; ++x) sts16(o0 + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[1][x])));
+          }
+          if (half == 0) {
+            if (y == 0) tmem_store32(tm0 + cur * 32u, acc);   // still needed for the second tile row
+            cur ^= 1u;
+            tmem_load32(tm0 + cur * 32u, acc);
+          }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(out_ready(pslot));
         if (++pslot == PS) { pslot = 0; fpar ^= 1u; }
       }
     }
   }
+  // every warp comes here, also after a failed wait: the tensor memory must be given back before the block ends
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 // ------------------------------------------------------------------------------------------ host side
