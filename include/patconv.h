@@ -86,6 +86,25 @@ int pat_project(const float *w, int F, int C, const uint16_t *masks, int K, int6
                 uint8_t *pattern_id, float *w_masked, void *workspace, size_t workspace_bytes,
                 void *stream);
 
+/* pat_project without a caller-supplied workspace, and without any allocation.  (The paper has no counterpart
+ * for this entry point: it exists for the way the library is embedded, not for the method.)
+ * Who needs it: code that is not allowed to allocate device memory where it runs - a server that gave its
+ * whole device budget to a memory pool at start-up, a plug-in living inside another framework's allocator,
+ * a real-time loop that cannot accept the device-wide synchronisation an allocation may cause.
+ * The scratch space is a fixed array inside the library image (about 2.7 MB on every GPU that loads the
+ * library, held until the process exits), sized for layers of up to pat_project_static_max_kernels() =
+ * 262144 kernels (F * C; a 512 x 512 layer).  Larger layers are refused with PAT_ERR_WORKSPACE and nothing
+ * is launched; use pat_project for them.  Arguments and results are those of pat_project.
+ * - The first call on each device looks up the array's device address (no allocation, but a runtime call
+ *   that is not stream work): make that first call before any stream capture.
+ * - All calls share the one array and it keeps whatever the previous call left there; the kernels
+ *   re-initialise every counter they rely on, so stale contents never matter.  Two calls whose kernels
+ *   may overlap on the GPU (different streams, no dependency between them) race on the array: order them.
+ * - Calls cudaMalloc / cudaFree or any allocating routine: never. */
+int pat_project_static(const float *w, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+                       uint8_t *pattern_id, float *w_masked, void *stream);
+int64_t pat_project_static_max_kernels(void);
+
 /* Size in bytes of the packed blob of a layer (0 on invalid arguments).  A pure function of its
  * arguments, so no device-to-host transfer is ever needed to size a buffer. */
 size_t pat_pack_size(int F, int C, int K, int64_t n_keep, int dtype);

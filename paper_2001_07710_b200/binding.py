@@ -23,7 +23,7 @@ TORCH_DTYPE = {PAT_F32: torch.float32, PAT_F16: torch.float16}
 
 EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project_workspace", "pat_project",
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
-           "pat_query_status", "pat_launch_count"]
+           "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels"]
 
 
 class PatError(RuntimeError):
@@ -57,6 +57,8 @@ def load() -> C.CDLL:
     L.pat_conv3x3_dense.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp]
     L.pat_query_status.argtypes = [vp]
     L.pat_launch_count.argtypes = []; L.pat_launch_count.restype = C.c_uint64
+    L.pat_project_static.argtypes = [vp, i32, i32, vp, i32, i64, vp, vp, vp]
+    L.pat_project_static_max_kernels.argtypes = []; L.pat_project_static_max_kernels.restype = i64
     _lib = L
     return L
 
@@ -168,3 +170,17 @@ def pat_query_status(stream=None) -> int:
 
 def pat_launch_count() -> int:
     return int(load().pat_launch_count())
+
+
+def pat_project_static_max_kernels() -> int:
+    return int(load().pat_project_static_max_kernels())
+
+
+def pat_project_static(w: torch.Tensor, masks, n_keep: int, pattern_id: torch.Tensor, w_masked: torch.Tensor, stream=None):
+    """pat_project with the library's built-in scratch array: the library allocates nothing and the caller passes
+    no workspace (for callers that may not allocate device memory).  Outputs must be preallocated by the caller."""
+    F, Cc = int(w.shape[0]), int(w.shape[1])
+    m = _masks(masks)
+    _check(load().pat_project_static(_ptr(w), F, Cc, m.ctypes.data, len(m), int(n_keep), _ptr(pattern_id), _ptr(w_masked),
+                                     _stream(stream)))
+    return pattern_id, w_masked

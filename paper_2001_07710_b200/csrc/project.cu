@@ -239,3 +239,59 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   count_launches(mode < 0 ? 13 : 2);
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
+
+// ------------------------------------------------------------------------------------------------------------
+// pat_project_static: the same projection for callers that cannot hand over a workspace.
+//
+// Some hosts of this library may not allocate device memory at the point where they project a layer: a serving
+// process whose whole device budget was reserved up front by another component, a plug-in that runs inside
+// somebody else's memory pool, or a latency-critical loop that must not risk the implicit device-wide
+// synchronisation of an allocation.  For them the scratch space lives in the library image itself.
+namespace pat {
+namespace {
+
+constexpr int64_t kStaticMaxKernels = 262144;   // F * C limit of pat_project_static (a 512 x 512 layer)
+constexpr size_t kStaticScratchBytes =
+    ((8 * (size_t)kStaticMaxKernels + 255) / 256 * 256) + (((size_t)kStaticMaxKernels + 255) / 256 * 256) +
+    4 * (size_t)kBins + (((size_t)(kStaticMaxKernels / kSelBlock + 1) * 4 + 255) / 256 * 256) + 256;
+
+// Every GPU that loads the library holds this array until the process ends.
+static __device__ __align__(256) unsigned char g_project_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {};          // device address of the array, per device (host-side cache)
+
+// The array's name is only a host-side handle in host code; the device address has to be asked for, once per
+// device and with that device current.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
+  if (dev < 0 || dev >= kMaxDevices) return set_error(PAT_ERR_CUDA, "pat_project_static: device index %d not supported", dev);
+  void* p = __atomic_load_n(&g_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (int rc = check_cuda(cudaGetSymbolAddress(&p, g_project_scratch), "cudaGetSymbolAddress(scratch)")) return rc;
+    __atomic_store_n(&g_scratch_addr[dev], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return PAT_OK;
+}
+
+}  // namespace
+}  // namespace pat
+
+extern "C" int64_t pat_project_static_max_kernels(void) { return kStaticMaxKernels; }
+
+extern "C" int pat_project_static(const float* w, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                                  uint8_t* pattern_id, float* w_masked, void* stream) {
+  if (F < 1 || C < 1 || F > 65535 || C > 65535)
+    return set_error(PAT_ERR_SHAPE, "pat_project_static: F=%d C=%d outside 1..65535", F, C);
+  if ((int64_t)F * C > kStaticMaxKernels)
+    return set_error(PAT_ERR_WORKSPACE, "pat_project_static: F*C = %lld exceeds the built-in scratch (%lld kernels); use pat_project with a workspace",
+                     (long long)F * C, (long long)kStaticMaxKernels);
+  static_assert(kStaticScratchBytes >= 8 * (size_t)kStaticMaxKernels, "scratch holds at least the keys");
+  if (carve(nullptr, (int64_t)F * C).bytes > kStaticScratchBytes)
+    return set_error(PAT_ERR_WORKSPACE, "pat_project_static: internal scratch too small for F=%d C=%d", F, C);
+  void* scratch = nullptr;
+  if (int rc = static_scratch(&scratch)) return rc;
+  return pat_project(w, F, C, masks, K, n_keep, pattern_id, w_masked, scratch, kStaticScratchBytes, stream);
+}
