@@ -208,6 +208,88 @@ __global__ void __launch_bounds__(NWARP * 32) k_conv_dense_small_c(DenseArgs a) 
   }
 }
 
+// Dense first layer of an RGB network (C = 3, stride 1): one output pixel per thread.  The 27 inputs of the
+// pixel sit in registers; filters are taken 8 at a time: for each of the 27 kernel entries one warp-uniform
+// 16-byte (fp16) or 2 x 16-byte (fp32) shared-memory load brings the entry of 8 filters, followed by 8
+// multiply-adds on the same input register; the 8 results leave as one 16-byte (32-byte) store.
+template <typename T> struct DenseC3;
+template <> struct DenseC3<__half> {
+  static __device__ __forceinline__ void mac8(float (&acc)[8], unsigned short in, const void* wrow) {
+    const uint4 w = *static_cast<const uint4*>(wrow);
+    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      unsigned short lo, hi;
+      asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ws[j]));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[2 * j]) : "h"(in), "h"(lo));
+      asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc[2 * j + 1]) : "h"(in), "h"(hi));
+    }
+  }
+  static __device__ __forceinline__ unsigned short load(const __half* p) { return __half_as_ushort(*p); }
+  static __device__ __forceinline__ unsigned short zero() { return 0; }
+  using In = unsigned short;
+  static __device__ __forceinline__ void store8(__half* dst, const float (&acc)[8]) {
+    uint4 v;
+    v.x = (uint32_t)__half_as_ushort(__float2half_rn(acc[0])) | ((uint32_t)__half_as_ushort(__float2half_rn(acc[1])) << 16);
+    v.y = (uint32_t)__half_as_ushort(__float2half_rn(acc[2])) | ((uint32_t)__half_as_ushort(__float2half_rn(acc[3])) << 16);
+    v.z = (uint32_t)__half_as_ushort(__float2half_rn(acc[4])) | ((uint32_t)__half_as_ushort(__float2half_rn(acc[5])) << 16);
+    v.w = (uint32_t)__half_as_ushort(__float2half_rn(acc[6])) | ((uint32_t)__half_as_ushort(__float2half_rn(acc[7])) << 16);
+    *reinterpret_cast<uint4*>(dst) = v;
+  }
+};
+template <> struct DenseC3<float> {
+  static __device__ __forceinline__ void mac8(float (&acc)[8], float in, const void* wrow) {
+    const float4 a = static_cast<const float4*>(wrow)[0], b = static_cast<const float4*>(wrow)[1];
+    acc[0] = fmaf(in, a.x, acc[0]); acc[1] = fmaf(in, a.y, acc[1]); acc[2] = fmaf(in, a.z, acc[2]); acc[3] = fmaf(in, a.w, acc[3]);
+    acc[4] = fmaf(in, b.x, acc[4]); acc[5] = fmaf(in, b.y, acc[5]); acc[6] = fmaf(in, b.z, acc[6]); acc[7] = fmaf(in, b.w, acc[7]);
+  }
+  static __device__ __forceinline__ float load(const float* p) { return *p; }
+  static __device__ __forceinline__ float zero() { return 0.0f; }
+  using In = float;
+  static __device__ __forceinline__ void store8(float* dst, const float (&acc)[8]) {
+    reinterpret_cast<float4*>(dst)[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_conv_dense_c3(DenseArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  T* wsm = reinterpret_cast<T*>(smem_raw);            // [F / 8][27][8]: entry k of 8 consecutive filters
+  using D = DenseC3<T>;
+  for (int i = threadIdx.x; i < a.F * 27; i += blockDim.x) {
+    const int f = i / 27, k = i % 27;                 // k = 9 * c + 3 * r + s  (weights are [F][3][3][3])
+    wsm[((f >> 3) * 27 + k) * 8 + (f & 7)] = from_f32<T>(a.w[i]);
+  }
+  __syncthreads();
+  const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long npix = (long long)a.N * a.H * a.W;
+  if (pix >= npix) return;
+  const int x = (int)(pix % a.W);
+  const int y = (int)((pix / a.W) % a.H);
+  const int n = (int)(pix / ((long long)a.W * a.H));
+  const T* xin = static_cast<const T*>(a.x);
+  typename D::In in[27];
+#pragma unroll
+  for (int r = 0; r < 3; ++r)
+#pragma unroll
+    for (int s2 = 0; s2 < 3; ++s2) {
+      const int yi = y + r - 1, xi = x + s2 - 1;
+      const bool ok = yi >= 0 && yi < a.H && xi >= 0 && xi < a.W;
+      const T* src = xin + (((size_t)n * a.H + (ok ? yi : 0)) * a.W + (ok ? xi : 0)) * 3;
+#pragma unroll
+      for (int c = 0; c < 3; ++c) in[9 * c + 3 * r + s2] = ok ? D::load(src + c) : D::zero();
+    }
+  T* yout = static_cast<T*>(a.y) + (size_t)pix * a.F;
+  for (int fb = 0; fb < a.F / 8; ++fb) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    const T* wrow = wsm + (size_t)fb * 27 * 8;
+#pragma unroll
+    for (int k = 0; k < 27; ++k) D::mac8(acc, in[k], wrow + k * 8);
+    D::store8(yout + fb * 8, acc);
+  }
+}
+
 template <typename KernelT>
 int prepare(KernelT kernel, size_t smem) {
   if (smem > 48 * 1024)
@@ -280,6 +362,14 @@ extern "C" int pat_conv3x3_dense(const float* w, int F, int C, int dtype, const 
   a.tiles_x = (a.Wo + TW - 1) / TW; a.tiles_y = (a.Ho + TH - 1) / TH;
   if ((size_t)N * a.tiles_x * a.tiles_y > 0x7FFFFFFFull) return set_error(PAT_ERR_SHAPE, "pat_conv3x3_dense: too many tiles");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (C == 3 && stride == 1 && F % 8 == 0 && (size_t)F * 27 * 4 <= 48 * 1024) {
+    const long long npix = (long long)N * H * W;
+    const unsigned blocks = (unsigned)((npix + 255) / 256);
+    if (dtype == PAT_F16) k_conv_dense_c3<__half><<<blocks, 256, (size_t)F * 27 * 2, st>>>(a);
+    else k_conv_dense_c3<float><<<blocks, 256, (size_t)F * 27 * 4, st>>>(a);
+    count_launches(1);
+    return check_cuda(cudaGetLastError(), "pat_conv3x3_dense launch");
+  }
   if (dtype == PAT_F16) return stride == 1 ? launch_dense<__half, 1>(a, st) : launch_dense<__half, 2>(a, st);
   return stride == 1 ? launch_dense<float, 1>(a, st) : launch_dense<float, 2>(a, st);
 }

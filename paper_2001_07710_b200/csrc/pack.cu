@@ -67,15 +67,19 @@ __global__ void __launch_bounds__(256) k_pack_count(const uint8_t* __restrict__ 
   }
 }
 
-// One thread per filter: position = number of filters that come before it in the ordering
-// (kept count descending, per-pattern counts lexicographically descending, original index ascending).
-__global__ void k_pack_rank(int F, int K, BlobPtrs bp) {
-  const int f = blockIdx.x * blockDim.x + threadIdx.x;
-  if (f >= F) return;
+// One block per filter: position = number of filters that come before it in the ordering
+// (kept count descending, per-pattern counts lexicographically descending, original index ascending);
+// the threads of the block share the comparisons.
+__global__ void __launch_bounds__(128) k_pack_rank(int F, int K, BlobPtrs bp) {
+  __shared__ int s_rank, s_xrank;
+  const int f = blockIdx.x;
+  if (threadIdx.x == 0) { s_rank = 0; s_xrank = 0; }
+  __syncthreads();
   const int nf = bp.cnt[f];
   const int32_t* hf = bp.hist + (size_t)f * K;
-  int rank = 0;
-  for (int g = 0; g < F; ++g) {
+  const int g0 = (f / kExecGroup) * kExecGroup, g1 = min(F, g0 + kExecGroup);
+  int rank = 0, xr = 0;
+  for (int g = threadIdx.x; g < F; g += blockDim.x) {
     if (g == f) continue;
     const int ng = bp.cnt[g];
     bool before;
@@ -87,18 +91,18 @@ __global__ void k_pack_rank(int F, int K, BlobPtrs bp) {
       before = (j < K) ? (hg[j] > hf[j]) : (g < f);
     }
     rank += before ? 1 : 0;
+    // execution order: inside the aligned group of 32 original filters, by kept count (descending), then index
+    if (g >= g0 && g < g1) xr += (ng > nf || (ng == nf && g < f)) ? 1 : 0;
   }
-  bp.perm[rank] = f;
-  bp.inv[f] = rank;
-  // execution order: inside the aligned group of 32 original filters, by kept count (descending), then index
-  const int g0 = (f / kExecGroup) * kExecGroup, g1 = min(F, g0 + kExecGroup);
-  int xr = g0;
-  for (int g = g0; g < g1; ++g) {
-    const int ng = bp.cnt[g];
-    xr += (ng > nf || (ng == nf && g < f)) ? 1 : 0;
+  atomicAdd(&s_rank, rank);
+  atomicAdd(&s_xrank, xr);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    bp.perm[s_rank] = f;
+    bp.inv[f] = s_rank;
+    bp.xfilt[g0 + s_xrank] = f;
+    bp.xinv[f] = g0 + s_xrank;
   }
-  bp.xfilt[xr] = f;
-  bp.xinv[f] = xr;
 }
 
 // One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
@@ -283,7 +287,7 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   const MaskTable lib = make_table(masks, K);
   const BlobPtrs bp = blob_ptrs(blob, L, F, K);
   k_pack_count<<<F, 256, K * sizeof(int), st>>>(pattern_id, C, K, bp, status);
-  k_pack_rank<<<(F + 127) / 128, 128, 0, st>>>(F, K, bp);
+  k_pack_rank<<<F, 128, 0, st>>>(F, K, bp);
   k_pack_ptrs<<<1, 1024, 0, st>>>(F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
   if (dtype == PAT_F16) k_pack_scatter<__half><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
   else k_pack_scatter<float><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);

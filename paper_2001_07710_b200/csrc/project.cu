@@ -22,33 +22,44 @@ struct SelectState {
 };
 
 // workspace layout
+constexpr int kCoarse = 256;                 // coarse histogram: the upper 8 bits of a 16-bit digit
+constexpr int kPasses = 4;                   // 64-bit keys, 16 bits per pass
+constexpr size_t kHistWords = (size_t)kPasses * (kBins + kCoarse);   // one fine + one coarse histogram per pass
+
 struct ProjWs {
   unsigned long long* key;     // [FC] energy bit patterns
   unsigned char* pid;          // [FC] best pattern per kernel
-  unsigned int* hist;          // [65536]
+  unsigned int* hist;          // [kPasses][65536 fine | 256 coarse]; zeroed by every call
   unsigned int* blk;           // [nblk + 1] tie counts per block, then exclusive offsets
   SelectState* st;
   size_t bytes;
 };
 
+constexpr size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
+constexpr size_t ws_bytes(int64_t FC) {
+  return ws_align(8 * (size_t)FC) + ws_align((size_t)FC) + ws_align(4 * kHistWords) +
+         ws_align(4 * ((size_t)((FC + kSelBlock - 1) / kSelBlock) + 1)) + ws_align(sizeof(SelectState));
+}
+
 inline ProjWs carve(void* base, int64_t FC) {
   ProjWs w;
   char* p = static_cast<char*>(base);
   size_t o = 0;
-  w.key = reinterpret_cast<unsigned long long*>(p + o); o = align256(o + 8 * (size_t)FC);
-  w.pid = reinterpret_cast<unsigned char*>(p + o);      o = align256(o + (size_t)FC);
-  w.hist = reinterpret_cast<unsigned int*>(p + o);      o = align256(o + 4 * (size_t)kBins);
-  const size_t nblk = (size_t)((FC + kSelBlock - 1) / kSelBlock);
-  w.blk = reinterpret_cast<unsigned int*>(p + o);       o = align256(o + 4 * (nblk + 1));
-  w.st = reinterpret_cast<SelectState*>(p + o);         o = align256(o + sizeof(SelectState));
+  w.key = reinterpret_cast<unsigned long long*>(p + o); o += ws_align(8 * (size_t)FC);
+  w.pid = reinterpret_cast<unsigned char*>(p + o);      o += ws_align((size_t)FC);
+  w.hist = reinterpret_cast<unsigned int*>(p + o);      o += ws_align(4 * kHistWords);
+  w.blk = reinterpret_cast<unsigned int*>(p + o);       o += ws_align(4 * ((size_t)((FC + kSelBlock - 1) / kSelBlock) + 1));
+  w.st = reinterpret_cast<SelectState*>(p + o);         o += ws_align(sizeof(SelectState));
   w.bytes = o;
   return w;
 }
 
 // One thread per kernel: energies of all masks, argmax (lowest id on ties).
 __global__ void k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
-                                 unsigned long long* __restrict__ key, unsigned char* __restrict__ pid) {
+                                 unsigned long long* __restrict__ key, unsigned char* __restrict__ pid,
+                                 SelectState* st, long long n_keep) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
   if (i >= FC) return;
   double sq[9];
 #pragma unroll
@@ -70,57 +81,74 @@ __global__ void k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTa
   pid[i] = (unsigned char)best;
 }
 
-__global__ void k_sel_init(SelectState* st, long long n_keep, unsigned int* hist) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
-  if (i < kBins) hist[i] = 0u;
-}
-
-// Histogram of the current 16-bit digit over the keys that match the decided prefix.
+// Histogram of the current 16-bit digit over the keys that match the decided prefix (fine: all 16 bits,
+// coarse: its upper 8 bits).  Identical digits inside a warp are merged into one atomic.
 __global__ void k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
                            const SelectState* __restrict__ st, unsigned int* __restrict__ hist) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= FC) return;
   const int shift = 48 - 16 * pass;
-  const unsigned long long k = key[i];
-  if (pass > 0 && (k >> (shift + 16)) != st->prefix) return;
-  atomicAdd(&hist[(unsigned)((k >> shift) & 0xFFFFull)], 1u);
+  bool in = i < FC;
+  unsigned d = 0;
+  if (in) {
+    const unsigned long long k = key[i];
+    in = (pass == 0) || ((k >> (shift + 16)) == st->prefix);
+    d = (unsigned)((k >> shift) & 0xFFFFull);
+  }
+  unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
+  unsigned int* coarse = fine + kBins;
+  const unsigned active = __ballot_sync(0xFFFFFFFFu, in);
+  if (!in) return;
+  const unsigned same = __match_any_sync(active, d);
+  const int lane = threadIdx.x & 31;
+  if ((int)(__ffs(same) - 1) == lane) atomicAdd(&fine[d], (unsigned)__popc(same));
+  const unsigned same_c = __match_any_sync(active, d >> 8);
+  if ((int)(__ffs(same_c) - 1) == lane) atomicAdd(&coarse[d >> 8], (unsigned)__popc(same_c));
 }
 
-// One block: find the digit d with  count(digit > d) < remaining <= count(digit >= d);  clears the histogram.
-__global__ void __launch_bounds__(1024) k_sel_pick(SelectState* st, unsigned int* hist) {
-  __shared__ unsigned long long part[1024];
-  const int t = threadIdx.x;
-  constexpr int per = kBins / 1024;   // 64 bins per thread; thread 0 owns the highest digits
-  const int top = kBins - 1 - t * per;
-  unsigned long long s = 0;
-  for (int q = 0; q < per; ++q) s += hist[top - q];
-  part[t] = s;
-  __syncthreads();
-  // inclusive scan (Hillis-Steele) over threads, highest digits first
-  for (int off = 1; off < 1024; off <<= 1) {
-    unsigned long long v = (t >= off) ? part[t - off] : 0ull;
-    __syncthreads();
-    part[t] += v;
-    __syncthreads();
+// Inclusive scan over the 256 threads of a block, thread 0 first.
+__device__ inline unsigned long long block_scan_256(unsigned long long v, unsigned long long* warp_tot) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned long long u = __shfl_up_sync(0xFFFFFFFFu, v, off);
+    if (lane >= off) v += u;
   }
-  const unsigned long long before = part[t] - s;   // keys with digits above this thread's range
-  const unsigned long long rem = (unsigned long long)st->remaining;
+  if (lane == 31) warp_tot[wid] = v;
   __syncthreads();
-  if (rem > before && rem <= before + s) {
-    unsigned long long above = before;
-    for (int q = 0; q < per; ++q) {
-      const unsigned int h = hist[top - q];
-      if (rem <= above + h) {
-        st->prefix = (st->prefix << 16) | (unsigned long long)(top - q);
-        st->remaining = (long long)(rem - above);
-        break;
-      }
-      above += h;
+  unsigned long long add = 0;
+  for (int q = 0; q < wid; ++q) add += warp_tot[q];
+  __syncthreads();
+  return v + add;
+}
+
+// One block of 256 threads: find the digit d with  count(digit > d) < remaining <= count(digit >= d), first in
+// the coarse histogram, then among the 256 fine bins of the coarse bin found.  Thread 0 owns the highest bin.
+__global__ void __launch_bounds__(256) k_sel_pick(SelectState* st, const unsigned int* __restrict__ hist, int pass) {
+  __shared__ unsigned long long warp_tot[8];
+  __shared__ int s_coarse;
+  __shared__ unsigned long long s_above;
+  const unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
+  const unsigned int* coarse = fine + kBins;
+  const int t = threadIdx.x;
+  const unsigned long long rem = (unsigned long long)st->remaining;
+  {
+    const int bin = kCoarse - 1 - t;
+    const unsigned long long c = coarse[bin];
+    const unsigned long long incl = block_scan_256(c, warp_tot);
+    if (rem > incl - c && rem <= incl) { s_coarse = bin; s_above = incl - c; }
+  }
+  __syncthreads();
+  const int cb = s_coarse;
+  const unsigned long long above = s_above;
+  {
+    const int bin = cb * 256 + (255 - t);
+    const unsigned long long c = fine[bin];
+    const unsigned long long incl = above + block_scan_256(c, warp_tot);
+    if (rem > incl - c && rem <= incl) {
+      st->prefix = (st->prefix << 16) | (unsigned long long)bin;
+      st->remaining = (long long)(rem - (incl - c));
     }
   }
-  __syncthreads();
-  for (int q = 0; q < per; ++q) hist[top - q] = 0u;
 }
 
 // Ties at the threshold: count per block of 1024 consecutive kernels.
@@ -200,7 +228,7 @@ using namespace pat;
 
 extern "C" size_t pat_project_workspace(int F, int C) {
   if (F < 1 || C < 1 || F > 65535 || C > 65535) return 0;
-  return carve(nullptr, (int64_t)F * C).bytes;
+  return ws_bytes((int64_t)F * C);
 }
 
 extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
@@ -222,21 +250,21 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   lib.K = K;
   const int nb256 = (int)((FC + 255) / 256);
   const int nblk = (int)((FC + kSelBlock - 1) / kSelBlock);
-  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid);
+  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep);
   int mode = -1;
   if (n_keep == FC) mode = 1;
   else if (n_keep == 0) mode = 0;
   if (mode < 0) {
-    k_sel_init<<<kBins / 256, 256, 0, st>>>(ws.st, (long long)n_keep, ws.hist);
-    for (int pass = 0; pass < 4; ++pass) {
+    if (int rc = check_cuda(cudaMemsetAsync(ws.hist, 0, 4 * kHistWords, st), "pat_project memset")) return rc;
+    for (int pass = 0; pass < kPasses; ++pass) {
       k_sel_hist<<<nb256, 256, 0, st>>>(ws.key, FC, pass, ws.st, ws.hist);
-      k_sel_pick<<<1, 1024, 0, st>>>(ws.st, ws.hist);
+      k_sel_pick<<<1, 256, 0, st>>>(ws.st, ws.hist, pass);
     }
     k_tie_count<<<nblk, kSelBlock, 0, st>>>(ws.key, FC, ws.st, ws.blk);
     k_tie_scan<<<1, 1024, 0, st>>>(ws.blk, nblk);
   }
   k_finalize<<<nblk, kSelBlock, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
-  count_launches(mode < 0 ? 13 : 2);
+  count_launches(mode < 0 ? 12 : 2);
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
 
@@ -251,9 +279,7 @@ namespace pat {
 namespace {
 
 constexpr int64_t kStaticMaxKernels = 262144;   // F * C limit of pat_project_static (a 512 x 512 layer)
-constexpr size_t kStaticScratchBytes =
-    ((8 * (size_t)kStaticMaxKernels + 255) / 256 * 256) + (((size_t)kStaticMaxKernels + 255) / 256 * 256) +
-    4 * (size_t)kBins + (((size_t)(kStaticMaxKernels / kSelBlock + 1) * 4 + 255) / 256 * 256) + 256;
+constexpr size_t kStaticScratchBytes = ws_bytes(kStaticMaxKernels);   // about 3.4 MB
 
 // Every GPU that loads the library holds this array until the process ends.
 static __device__ __align__(256) unsigned char g_project_scratch[kStaticScratchBytes];
