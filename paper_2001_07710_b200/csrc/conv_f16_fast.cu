@@ -62,7 +62,7 @@ static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 // Register split between the warp groups.  The pool is what the block got at launch (threads x registers per
 // thread as compiled), so the split must fit inside it or the increase would wait forever; the host checks the
 // compiled count before launching.
-constexpr int LAUNCH_REGS = 96, CONSUMER_REGS = 104, PRODUCER_REGS = 64;
+constexpr int LAUNCH_REGS = 96, CONSUMER_REGS = 88, PRODUCER_REGS = 128;
 static_assert(NCW * 32 * CONSUMER_REGS + NPW * 32 * PRODUCER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 256;        // 4 consumer warps per lane quarter x 2 filters x 32 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -225,6 +225,12 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&a)[TR][TC]) 
         "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
       : "r"(taddr)
       : "memory");
+}
+
+template <int REGS>
+__device__ __forceinline__ void set_warp_registers() {
+  if constexpr (REGS > LAUNCH_REGS) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS));
+  else if constexpr (REGS < LAUNCH_REGS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS));
 }
 
 // ------------------------------------------------------------------------------------------ work items
@@ -408,7 +414,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
   auto item_of = [&](int it_idx) { return decode_item(p, (int)blockIdx.x + it_idx * (int)gridDim.x); };
 
   if (warp >= NCW) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PRODUCER_REGS));
+    set_warp_registers<PRODUCER_REGS>();
     const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
     if (warp < NCW + NFW) {
       // ========================================================================= fill warps
@@ -492,9 +498,11 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         for (int cb = 0; cb < nct && alive; ++cb, ++rstage) {
           // descriptors of this block: issue the global loads of the first entries now, use them after the transposition
           const int nk = ke - kb, kb_cur = kb;
-          uint32_t dmeta = 0u;
-          uint2 dw = make_uint2(0u, 0u);
-          if (dj < nk) { dmeta = __ldg(p.tmeta + kb + dj); dw = __ldg(p.tw4 + kb + dj); }
+          uint32_t dmeta[2] = {0u, 0u};
+          uint2 dw[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+#pragma unroll
+          for (int u = 0; u < 2; ++u)
+            if (dj + 3 * u < nk) { dmeta[u] = __ldg(p.tmeta + kb + dj + 3 * u); dw[u] = __ldg(p.tw4 + kb + dj + 3 * u); }
           if (cb + 1 < nct) load_range(g, cb + 1, kb, ke);
 
           if (!mbar_wait(raw_full(rslot), rpar, abort_flag)) { alive = false; break; }
@@ -503,16 +511,34 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
           const uint32_t raw0 = sbase + OFF_RAW + rslot * RAW_STAGE;
           const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
           // transposition, one shared-memory row (4 segments) at a time: four independent loads, then their stores
-          for (int pr = pw; pr < nrows; pr += NFW) {
+          // (the loads of the next row are issued before the stores of the current one)
+          auto load_prow = [&](int pr, uint32_t (&v)[LX][4]) {
             const bool b1 = pr >= rows0;
             const uint32_t lr = raw0 + (uint32_t)(b1 ? pr - rows0 : pr) * rowpitch;
-            const uint32_t sr = pl0 + pr * ROWB + ((pr & 2) ? stoff1 : stoff0);   // chunk swizzle by (row >> 1) & 1
-            uint32_t v[LX][4];
 #pragma unroll
             for (int seg = 0; seg < LX; ++seg)
               ldmatrix_x4_trans(lr + (b1 ? nioff[1][seg] : nioff[0][seg]), v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
+          };
+          auto store_prow = [&](int pr, const uint32_t (&v)[LX][4]) {
+            const uint32_t sr = pl0 + pr * ROWB + ((pr & 2) ? stoff1 : stoff0);   // chunk swizzle by (row >> 1) & 1
 #pragma unroll
             for (int seg = 0; seg < LX; ++seg) stmatrix_x4(sr + seg * SEGB, v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
+          };
+          {
+            uint32_t va[LX][4], vb[LX][4];
+            int pr = pw;
+            if (pr < nrows) load_prow(pr, va);
+            while (pr < nrows) {
+              const int p1 = pr + NFW;
+              if (p1 < nrows) load_prow(p1, vb);
+              store_prow(pr, va);
+              const int p2 = p1 + NFW;
+              if (p1 < nrows) {
+                if (p2 < nrows) load_prow(p2, va);
+                store_prow(p1, vb);
+              }
+              pr = p2;
+            }
           }
           // kernel descriptors
           {
@@ -523,8 +549,10 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
               const uint32_t mm = cl | p.pword[mt >> 16];
               sts128(d0 + DESC_HDR + (dslot * CB + e) * 16, mm, wv.x, wv.y, 0u);
             };
-            if (dj < nk) put(dj, dmeta, dw);
-            for (int e = dj + 3; e < nk; e += 3) put(e, __ldg(p.tmeta + kb_cur + e), __ldg(p.tw4 + kb_cur + e));   // rare
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+              if (dj + 3 * u < nk) put(dj + 3 * u, dmeta[u], dw[u]);
+            for (int e = dj + 6; e < nk; e += 3) put(e, __ldg(p.tmeta + kb_cur + e), __ldg(p.tw4 + kb_cur + e));   // more than 6 kernels: rare
           }
           __syncwarp();
           // the fill warp that is last to finish with the raw slot refills it
@@ -604,7 +632,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
     }
   } else {
     // =========================================================================== consumer warps
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(CONSUMER_REGS));
+    set_warp_registers<CONSUMER_REGS>();
     const int ly = lane >> 2, lx = lane & 3;
     // Warp w owns filter slots w and 31 - w of the group (the most loaded filter with the least loaded one, ...).
     // Only one of the two accumulator tiles is in registers at a time; the other is parked in tensor memory:
@@ -636,11 +664,16 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         const uint32_t slot = f ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp;
         const int nk = (int)lds32(d0 + slot * 4);
         uint32_t e = d0 + DESC_HDR + slot * (CB * 16);
-        for (int k = 0; k < nk; ++k, e += 16) {
-          uint32_t m0, w01, w23, pad;
-          lds128(e, m0, w01, w23, pad);
+        uint32_t m0, w01, w23, pad;
+        lds128(e, m0, w01, w23, pad);          // (reads a stale entry when nk == 0: never used)
+        for (int k = 0; k < nk; ++k) {
+          e += 16;
+          uint32_t m1, v01, v23;
+          lds128(e, m1, v01, v23, pad);        // next descriptor while this kernel runs (one past the end at most:
+                                               // still inside the descriptor block or the barrier block after it)
           const uint32_t base = pl0 + (m0 & 15u) * CHP;
           one_kernel(acc, base + offA, base + offB, m0, w01, w23);
+          m0 = m1; w01 = v01; w23 = v23;
         }
       };
 
