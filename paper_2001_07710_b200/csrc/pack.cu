@@ -175,41 +175,75 @@ template <> __device__ inline float cvt_weight<float>(float v) { return v; }
 template <> __device__ inline __half cvt_weight<__half>(float v) { return __float2half_rn(v); }
 
 // One block per original filter: place every kept kernel in the canonical and in the execution order.
-template <typename T>
+// Positions are counted, never searched: per (16-channel tile, pattern) counts in shared memory give, after
+// prefix sums over the tiles, the start of every (pattern) run in the canonical order and of every tile in the
+// execution order; the rank of a kernel inside its tile needs a look at the 16 channels of that tile only.
+// TABLE = false (tile x pattern table too large for shared memory): the counts are taken by direct loops.
+template <typename T, bool TABLE>
 __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ wm, const uint8_t* __restrict__ pid,
                                                       int C, int K, int nct, MaskTable lib, BlobPtrs bp) {
-  extern __shared__ uint8_t spid[];   // C pattern ids of this filter
+  extern __shared__ __align__(16) uint8_t sm_raw[];
+  int* tile_pat = reinterpret_cast<int*>(sm_raw);                          // [nct][K] (TABLE only)
+  int* tile_start = tile_pat + (TABLE ? nct * K : 0);                      // [nct + 1] kept kernels before tile t
+  uint8_t* spid = reinterpret_cast<uint8_t*>(tile_start + nct + 1);        // C pattern ids of this filter
   const int f = blockIdx.x;
   const int q = bp.inv[f];
   for (int c = threadIdx.x; c < C; c += blockDim.x) spid[c] = pid[(size_t)f * C + c];
+  if (TABLE)
+    for (int i = threadIdx.x; i < nct * K; i += blockDim.x) tile_pat[i] = 0;
+  __syncthreads();
+  // kept kernels per tile (and per tile and pattern)
+  for (int t = threadIdx.x; t < nct; t += blockDim.x) {
+    int n = 0;
+    const int c0 = t * kChanTile, c1 = min(c0 + kChanTile, C);
+    for (int c = c0; c < c1; ++c) {
+      const int j = spid[c];
+      if (j == PAT_PRUNED || j >= K) continue;
+      ++n;
+      if (TABLE) tile_pat[t * K + j] += 1;        // one thread per tile: no race
+    }
+    tile_start[t + 1] = n;
+  }
+  __syncthreads();
+  // exclusive prefix sums over the tiles: one thread per pattern column, one more for the tile totals
+  if (TABLE) {
+    for (int j = threadIdx.x; j < K; j += blockDim.x) {
+      int run = 0;
+      for (int t = 0; t < nct; ++t) { const int v = tile_pat[t * K + j]; tile_pat[t * K + j] = run; run += v; }
+    }
+  }
+  if (threadIdx.x == blockDim.x - 1) {
+    int run = 0;
+    tile_start[0] = 0;
+    for (int t = 0; t < nct; ++t) { const int v = tile_start[t + 1]; tile_start[t + 1] = run + v; run += v; }
+  }
   __syncthreads();
   const int xe = bp.xinv[f];
   const int f0 = bp.xbase[xe];
-  // execution-section pointers: kernels of this filter before channel tile t
-  for (int t = threadIdx.x; t <= nct; t += blockDim.x) {
-    int n = 0;
-    const int cend = min(t * kChanTile, C);
-    for (int c = 0; c < cend; ++c) n += (spid[c] != PAT_PRUNED) ? 1 : 0;
-    bp.tptr[(size_t)xe * (nct + 1) + t] = f0 + n;
-  }
+  for (int t = threadIdx.x; t <= nct; t += blockDim.x) bp.tptr[(size_t)xe * (nct + 1) + t] = f0 + tile_start[t];
   T* w4 = static_cast<T*>(bp.w4);
   T* tw4 = static_cast<T*>(bp.tw4);
   for (int c = threadIdx.x; c < C; c += blockDim.x) {
     const int j = spid[c];
     if (j == PAT_PRUNED || j >= K) continue;
     const int tile = c / kChanTile;
-    int same_before = 0;      // kernels of the same pattern on lower channels      (canonical order)
-    int exec_before = 0;      // kernels ordered before (tile, pattern, channel)    (execution order)
-    for (int d = 0; d < C; ++d) {
+    const int c0 = tile * kChanTile, c1 = min(c0 + kChanTile, C);
+    int same_in_tile = 0;     // kernels of the same pattern on lower channels of this tile
+    int exec_in_tile = 0;     // kernels of this tile ordered before (pattern, channel)
+    for (int d = c0; d < c1; ++d) {
       const int pd = spid[d];
-      if (pd == PAT_PRUNED) continue;
-      same_before += (pd == j && d < c) ? 1 : 0;
-      const int td = d / kChanTile;
-      const bool lt = (td < tile) || (td == tile && (pd < j || (pd == j && d < c)));
-      exec_before += lt ? 1 : 0;
+      if (pd == PAT_PRUNED || pd >= K) continue;
+      same_in_tile += (pd == j && d < c) ? 1 : 0;
+      exec_in_tile += (pd < j || (pd == j && d < c)) ? 1 : 0;
+    }
+    int same_before;          // kernels of the same pattern on lower channels (canonical order)
+    if (TABLE) same_before = tile_pat[tile * K + j] + same_in_tile;
+    else {
+      same_before = same_in_tile;
+      for (int d = 0; d < c0; ++d) same_before += (spid[d] == j) ? 1 : 0;
     }
     const int pos = bp.pptr[(size_t)q * (K + 1) + j] + same_before;
-    const int tpos = f0 + exec_before;
+    const int tpos = f0 + tile_start[tile] + exec_in_tile;
     bp.chan[pos] = (uint16_t)c;
     bp.tmeta[tpos] = (uint32_t)c | ((uint32_t)j << 16);
     int bits[4];
@@ -289,8 +323,19 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   k_pack_count<<<F, 256, K * sizeof(int), st>>>(pattern_id, C, K, bp, status);
   k_pack_rank<<<F, 128, 0, st>>>(F, K, bp);
   k_pack_ptrs<<<1, 1024, 0, st>>>(F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
-  if (dtype == PAT_F16) k_pack_scatter<__half><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
-  else k_pack_scatter<float><<<F, 256, (size_t)C, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+  {
+    const size_t table = sizeof(int) * (size_t)L.nct * K;
+    const bool use_table = table <= 24 * 1024;
+    const size_t smem = (use_table ? table : 0) + sizeof(int) * ((size_t)L.nct + 1) + (size_t)C;
+    if (smem > 48 * 1024) return set_error(PAT_ERR_SHAPE, "pat_pack: C=%d too large for the packing kernel", C);
+    if (dtype == PAT_F16) {
+      if (use_table) k_pack_scatter<__half, true><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+      else k_pack_scatter<__half, false><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+    } else {
+      if (use_table) k_pack_scatter<float, true><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+      else k_pack_scatter<float, false><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+    }
+  }
   count_launches(4);
   return check_cuda(cudaGetLastError(), "pat_pack launch");
 }
