@@ -511,7 +511,6 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
           const uint32_t raw0 = sbase + OFF_RAW + rslot * RAW_STAGE;
           const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
           // transposition, one shared-memory row (4 segments) at a time: four independent loads, then their stores
-          // (the loads of the next row are issued before the stores of the current one)
           auto load_prow = [&](int pr, uint32_t (&v)[LX][4]) {
             const bool b1 = pr >= rows0;
             const uint32_t lr = raw0 + (uint32_t)(b1 ? pr - rows0 : pr) * rowpitch;
@@ -524,21 +523,10 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
 #pragma unroll
             for (int seg = 0; seg < LX; ++seg) stmatrix_x4(sr + seg * SEGB, v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
           };
-          {
-            uint32_t va[LX][4], vb[LX][4];
-            int pr = pw;
-            if (pr < nrows) load_prow(pr, va);
-            while (pr < nrows) {
-              const int p1 = pr + NFW;
-              if (p1 < nrows) load_prow(p1, vb);
-              store_prow(pr, va);
-              const int p2 = p1 + NFW;
-              if (p1 < nrows) {
-                if (p2 < nrows) load_prow(p2, va);
-                store_prow(p1, vb);
-              }
-              pr = p2;
-            }
+          for (int pr = pw; pr < nrows; pr += NFW) {
+            uint32_t va[LX][4];
+            load_prow(pr, va);
+            store_prow(pr, va);
           }
           // kernel descriptors
           {
@@ -664,16 +652,11 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         const uint32_t slot = f ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp;
         const int nk = (int)lds32(d0 + slot * 4);
         uint32_t e = d0 + DESC_HDR + slot * (CB * 16);
-        uint32_t m0, w01, w23, pad;
-        lds128(e, m0, w01, w23, pad);          // (reads a stale entry when nk == 0: never used)
-        for (int k = 0; k < nk; ++k) {
-          e += 16;
-          uint32_t m1, v01, v23;
-          lds128(e, m1, v01, v23, pad);        // next descriptor while this kernel runs (one past the end at most:
-                                               // still inside the descriptor block or the barrier block after it)
+        for (int k = 0; k < nk; ++k, e += 16) {
+          uint32_t m0, w01, w23, pad;
+          lds128(e, m0, w01, w23, pad);
           const uint32_t base = pl0 + (m0 & 15u) * CHP;
           one_kernel(acc, base + offA, base + offB, m0, w01, w23);
-          m0 = m1; w01 = v01; w23 = v23;
         }
       };
 
