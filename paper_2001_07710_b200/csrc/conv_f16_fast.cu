@@ -515,8 +515,12 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
             const bool b1 = pr >= rows0;
             const uint32_t lr = raw0 + (uint32_t)(b1 ? pr - rows0 : pr) * rowpitch;
 #pragma unroll
-            for (int seg = 0; seg < LX; ++seg)
-              ldmatrix_x4_trans(lr + (b1 ? nioff[1][seg] : nioff[0][seg]), v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
+            for (int seg = 0; seg < LX; ++seg) {
+              // the copies are written with the 32-byte swizzle (16-byte chunk index ^= address bit 7), which
+              // spreads the eight 32-byte-strided rows of a matrix over all banks
+              const uint32_t la = lr + (b1 ? nioff[1][seg] : nioff[0][seg]);
+              ldmatrix_x4_trans(la ^ ((la >> 3) & 16u), v[seg][0], v[seg][1], v[seg][2], v[seg][3]);
+            }
           };
           auto store_prow = [&](int pr, const uint32_t (&v)[LX][4]) {
             const uint32_t sr = pl0 + pr * ROWB + ((pr & 2) ? stoff1 : stoff0);   // chunk swizzle by (row >> 1) & 1
@@ -790,7 +794,7 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
   for (int n = 1; n <= NMAPS; ++n) {          // band of n tile rows: 2n rows + a halo row above and below
     const cuuint32_t box[4] = {(cuuint32_t)CB, (cuuint32_t)p.BW, (cuuint32_t)(TR * n + 2), (cuuint32_t)p.NI};
     const CUresult cr = encode_fn()(&tm.m[n - 1], CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr,
-                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cuTensorMapEncodeTiled failed (%d)", (int)cr);
   }
