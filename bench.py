@@ -163,12 +163,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    from paper_2001_07710_b200.sharding import job_throughput
 
     # ---- warm-up
     for _ in range(max(args.warmup, 3)):
@@ -190,9 +185,8 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     launches = pc.pat_launch_count() - launches0
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    value, ms_total, _ = job_throughput(float(N * args.steps), e0.elapsed_time(e1), "cuda")   # weak scaling: N images per rank
     ms_step = ms_total / args.steps
-    value = world * N * args.steps / (ms_total * 1e-3)
 
     # per-layer convolution times (mean over the timed steps)
     conv_ms = [float(np.mean([ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)])) for i in range(len(layers))]
@@ -206,7 +200,7 @@ def run_ours(args):
         step_e2e()
     e1.record(stream)
     barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+    e2e_value, ms_e2e, _ = job_throughput(float(N * e2e_steps), e0.elapsed_time(e1), "cuda")
     h2d = sum(st["hw"].numel() * 4 + st["hx"].numel() * elem for st in layers)
     d2h = sum(st["hy"].numel() * elem for st in layers)
     assert pc.pat_query_status() == 0
@@ -244,7 +238,7 @@ def run_ours(args):
                      "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
                      "min_layer_frac": min(p["roof_frac"] for p in per_layer if p["layer"] != "conv1")},
         "layers": per_layer,
-        "e2e": {"value": round(world * N * e2e_steps / (ms_e2e * 1e-3), 2), "unit": UNIT,
+        "e2e": {"value": round(e2e_value, 2), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
         "gpu_launches": int(launches),
         "clocks": clocks,

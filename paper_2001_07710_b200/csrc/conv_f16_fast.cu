@@ -67,7 +67,7 @@ static_assert(NCW * 32 * CONSUMER_REGS + NPW * 32 * PRODUCER_REGS <= NTHREADS * 
 constexpr uint32_t TMEM_COLS = 256;        // 4 consumer warps per lane quarter x 2 filters x 32 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
-constexpr uint32_t kSuspendNs = 100000u;                // longest stay inside one try_wait (0.1 ms)
+constexpr int kFillSleepNs = 200;                       // pause between polls of a waiting fill / store warp
 
 // One tiled copy brings a whole band (all its rows, all images side by side), because issuing a copy costs far
 // more than the copy engine needs per row; the box height is part of a tensor map, hence one map per height.
@@ -118,18 +118,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Same test, but the thread may stay suspended inside the instruction for up to `ns` nanoseconds while the
-// phase is incomplete: a waiting warp then issues next to nothing, which matters here because waiting warps
-// share their issue slots with the warps that are doing the multiply-adds.
-__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -137,13 +125,20 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait: gives up after kWaitNs of wall time (or kSpinLimit polls), raises the block-wide abort flag
 // and returns false; also returns false as soon as another thread of the block has given up.
+// SLEEP_NS > 0: sleep between polls.  The fill and store warps wait that way: a polling warp takes issue
+// slots from the four consumer warps of its SM partition, and those warps have slack (they work ahead by up
+// to three ring slots).  Consumers poll without sleeping: they rarely wait, and must restart at once.
+template <int SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-    if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
-    if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitNs) break;
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 31u) == 31u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitNs) break;
+    }
   }
   *abort_flag = 1;
   return false;
@@ -505,9 +500,9 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
             if (dj + 3 * u < nk) { dmeta[u] = __ldg(p.tmeta + kb + dj + 3 * u); dw[u] = __ldg(p.tw4 + kb + dj + 3 * u); }
           if (cb + 1 < nct) load_range(g, cb + 1, kb, ke);
 
-          if (!mbar_wait(raw_full(rslot), rpar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(raw_full(rslot), rpar, abort_flag)) { alive = false; break; }
           landed = rstage + 1;
-          if (!mbar_wait(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
           const uint32_t raw0 = sbase + OFF_RAW + rslot * RAW_STAGE;
           const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
           // transposition, one shared-memory row (4 segments) at a time: four independent loads, then their stores
@@ -564,7 +559,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         }
         // output stages: hand the next TR slots to the consumers as they become free
         for (int y = 0; y < TR && alive; ++y) {
-          if (!mbar_wait(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(pl_empty(pslot), ppar, abort_flag)) { alive = false; break; }
           if (lane == 0) mbar_arrive(pl_full(pslot));
           if (++pslot == PS) { pslot = 0; ppar ^= 1u; }
         }
@@ -588,7 +583,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
         const Item it = item_of(it_idx);
         pslot = (pslot + nct) % PS;                // skip the real stages of the item
         for (int y = 0; y < TR && alive; ++y) {
-          if (!mbar_wait(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
           opar ^= 1u << pslot;
           const uint32_t o0 = sbase + pslot * PLANAR_STAGE;
           // one thread tile (= one consumer lane) at a time: 14 pixels x 4 chunks of 8 channels; consecutive lanes
@@ -666,7 +661,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
 
       uint32_t cposA = 0u, cposB = 0u;   // byte offsets of filters 0 / 1 inside the group of 32 output channels
       for (int cb = 0; cb < nct; ++cb) {
-        if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
+        if (!mbar_wait<0>(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t pl0 = sbase + pslot * PLANAR_STAGE;
         const uint32_t d0 = sbase + OFF_DESC + pslot * DESC_STAGE;
         if (cb == nct - 1) {
@@ -691,7 +686,7 @@ k_conv_f16_s1(const __grid_constant__ TmapSet tms, const Params p) {
       // results: fp32 -> fp16 (round to nearest even) into the two output stages, one tile row each
 #pragma unroll 1
       for (int y = 0; y < TR; ++y) {
-        if (!mbar_wait(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
+        if (!mbar_wait<0>(pl_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t o0 = sbase + pslot * PLANAR_STAGE + (uint32_t)(lane * TC) * OUT_PITCH;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
