@@ -32,6 +32,9 @@ UNIT = "images/s"
 SM_COUNT, FMA_LANES, SM_MAX_MHZ = 148, 128, 1965.0
 FMA_PEAK_TFLOPS = 2 * FMA_LANES * SM_COUNT * SM_MAX_MHZ * 1e6 / 1e12     # 74.45: fp32 FMA, no tensor cores
 DEFAULT_CONFIG = 3
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_conv_f16_s1 launch (conv6 shape, batch 16), from
+# profiles/k_conv_f16_s1_conv6_b16.md
+CONV6_DRAM_BYTES_B16 = 25.876e6 + 0.121e6
 
 
 def measured_peaks():
@@ -234,7 +237,12 @@ def run_ours(args):
         "conv_only_images_per_s": round(world * N / (sum(conv_ms) * 1e-3), 2),
         "roofline": {"bound": "alu", "kernel": "sparse conv (12 launches per step)", "achieved": round(achieved, 3),
                      "peak": round(FMA_PEAK_TFLOPS, 2), "unit": "TFLOP/s", "frac": round(achieved / FMA_PEAK_TFLOPS, 4),
-                     "peak_kind": "derived: 2 x 128 fp32 lanes x 148 SMs x 1.965 GHz", "traffic": None,
+                     "peak_kind": "derived: 2 x 128 fp32 lanes x 148 SMs x 1.965 GHz",
+                     "traffic": CONV6_DRAM_BYTES_B16 * (N / 16.0) if (cfg.number == 3) else None,
+                     "traffic_note": ("DRAM read+write bytes of the conv6 launch (ncu, batch 16, scaled by batch/16; "
+                                      "input read once, the output is still in L2 when the kernel ends); "
+                                      "algorithmic bytes of that launch: %d" % layers[5]["L"].compulsory_bytes(N, elem))
+                                     if cfg.number == 3 else None,
                      "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
                      "min_layer_frac": min(p["roof_frac"] for p in per_layer if p["layer"] != "conv1")},
         "layers": per_layer,
