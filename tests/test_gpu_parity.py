@@ -167,6 +167,28 @@ def test_conv_tuned_f16_matches_oracle(case):
     check_close(out, ref, "f16")
 
 
+def test_conv_tuned_f16_many_regions_dense_keep():
+    """Several work items per thread block (672 regions) and up to 16 kernels per filter and 16-channel block
+    (keep 1/2, 12 patterns); sampled against the oracle."""
+    N, H, W, C, F, K = 12, 224, 224, 16, 128, 12
+    rng = np.random.default_rng(99)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
+    masks = oracle.library(K)
+    n_keep = F * C // 2
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    y = torch.full((N, H, W, F), float("nan"), dtype=torch.float16, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y)
+    assert pc.pat_query_status() == 0
+    assert bool(torch.isfinite(y).all())
+    coords = np.stack([rng.integers(0, N, 6000), rng.integers(0, H, 6000), rng.integers(0, W, 6000), rng.integers(0, F, 6000)], axis=1).astype(np.int32)
+    coords[:64, 1] = 0; coords[64:128, 1] = H - 1; coords[128:192, 2] = 0; coords[192:256, 2] = W - 1
+    ref = oracle.conv3x3_at(stored_weights(wm_o, "f16"), x, coords, 1)
+    out = y[coords[:, 0], coords[:, 1], coords[:, 2], coords[:, 3]].float().cpu().numpy()
+    check_close(out, ref, "f16")
+
+
 def test_conv_tuned_f16_arbitrary_library():
     """Masks outside the built-in set (some without the centre) run through the per-position code of the tuned kernel."""
     N, H, W, C, F = 3, 28, 28, 48, 64
