@@ -152,6 +152,20 @@ int pat_unpack(const void *blob, int F, int C, const uint16_t *masks, int K, int
 int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                 int dtype, const void *x, void *y, int N, int H, int W, int stride, void *stream);
 
+/* The same convolution with a caller-supplied device workspace.  For the layer shapes it covers (fp16, stride 1,
+ * C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k}, H even and >= 14) the
+ * activations are first re-arranged, once per call, into the channel-planar tiles the multiply-add kernel
+ * stages in shared memory; the kernel then needs no transposition of its own and runs a deeper pipeline.
+ * pat_conv3x3_workspace returns the bytes needed (about 1.43 x the size of x), or 0 for a layer the workspace
+ * path does not cover: pat_conv3x3_ws then behaves exactly like pat_conv3x3 and ignores the workspace.
+ *   workspace  dev, at least pat_conv3x3_workspace(...) bytes, 256-byte aligned; contents are scratch;
+ *              concurrent calls must use different workspaces
+ * Results are those of pat_conv3x3 (same products, fp32 sums in the same order). */
+size_t pat_conv3x3_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
+int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+                   int dtype, const void *x, void *y, int N, int H, int W, int stride,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
 /* Dense 3x3 convolution for layers that are not pruned (the first layer of VGG-16, C = 3).
  *   w   dev, [F][C][3][3] fp32 (converted to the activation type on the fly)
  *   x   dev NHWC [N][H][W][C]; y dev NHWC [N][Ho][Wo][F]; dtype of x and y = `dtype`

@@ -23,7 +23,8 @@ TORCH_DTYPE = {PAT_F32: torch.float32, PAT_F16: torch.float16}
 
 EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project_workspace", "pat_project",
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
-           "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels"]
+           "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels",
+           "pat_conv3x3_workspace", "pat_conv3x3_ws"]
 
 
 class PatError(RuntimeError):
@@ -54,6 +55,8 @@ def load() -> C.CDLL:
     L.pat_blob_layout.argtypes = [i32, i32, i32, i64, i32, vp]
     L.pat_unpack.argtypes = [vp, i32, i32, vp, i32, i64, i32, vp, vp]
     L.pat_conv3x3.argtypes = [vp, i32, i32, vp, i32, i64, i32, vp, vp, i32, i32, i32, i32, vp]
+    L.pat_conv3x3_workspace.argtypes = [i32, i32, i32, i32, i32, i32, i32]; L.pat_conv3x3_workspace.restype = sz
+    L.pat_conv3x3_ws.argtypes = [vp, i32, i32, vp, i32, i64, i32, vp, vp, i32, i32, i32, i32, vp, sz, vp]
     L.pat_conv3x3_dense.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp]
     L.pat_query_status.argtypes = [vp]
     L.pat_launch_count.argtypes = []; L.pat_launch_count.restype = C.c_uint64
@@ -140,15 +143,31 @@ def pat_unpack(blob: torch.Tensor, F: int, Cc: int, masks, n_keep: int, dtype,
     return out
 
 
+def pat_conv3x3_workspace(F: int, Cc: int, dtype, N: int, H: int, W: int, stride: int = 1) -> int:
+    """Bytes of workspace pat_conv3x3_ws wants for this layer (0: the layer runs without one)."""
+    return int(load().pat_conv3x3_workspace(F, Cc, _DT[dtype], N, H, W, int(stride)))
+
+
 def pat_conv3x3(blob: torch.Tensor, F: int, Cc: int, masks, n_keep: int, dtype, x: torch.Tensor,
-                stride: int = 1, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """x: cuda NHWC [N,H,W,C] in the blob's dtype.  Returns y NHWC [N,Ho,Wo,F]."""
+                stride: int = 1, y: Optional[torch.Tensor] = None, stream=None,
+                workspace: Optional[torch.Tensor] = None, use_workspace: bool = True) -> torch.Tensor:
+    """x: cuda NHWC [N,H,W,C] in the blob's dtype.  Returns y NHWC [N,Ho,Wo,F].
+
+    Calls pat_conv3x3_ws with `workspace` (a cuda uint8 tensor, allocated here when None and the layer wants
+    one); use_workspace=False calls the entry point without workspace, pat_conv3x3."""
     m = _masks(masks)
     N, H, W = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
     if y is None:
         y = torch.empty((N, (H - 1) // stride + 1, (W - 1) // stride + 1, F), dtype=x.dtype, device=x.device)
-    _check(load().pat_conv3x3(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
-                              N, H, W, int(stride), _stream(stream)))
+    need = pat_conv3x3_workspace(F, Cc, dtype, N, H, W, stride) if use_workspace else 0
+    if need == 0:
+        _check(load().pat_conv3x3(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
+                                  N, H, W, int(stride), _stream(stream)))
+        return y
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    _check(load().pat_conv3x3_ws(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
+                                 N, H, W, int(stride), _ptr(workspace), int(workspace.numel()), _stream(stream)))
     return y
 
 

@@ -9,10 +9,11 @@
 namespace pat {
 
 constexpr uint32_t kBlobMagic = 0x50415443u;  // "PATC"
-constexpr uint32_t kBlobVersion = 1u;
+constexpr uint32_t kBlobVersion = 2u;
 constexpr int kChanTile = 16;                 // granularity (input channels) of the execution section
 constexpr int kExecGroup = 32;                // filters per execution group (aligned groups of original filters)
 constexpr int kMaxK = 255;
+constexpr int kBlockHeaderBytes = 4 * kExecGroup;   // header of a descriptor block: one 32-bit word per filter slot
 
 // First 256 bytes of every blob.
 struct BlobHeader {
@@ -21,6 +22,7 @@ struct BlobHeader {
   int64_t n_keep;
   uint64_t total_bytes;
   uint16_t masks[kMaxK + 1];  // library the blob was packed with (entries >= K are 0)
+  int32_t max_block_entries;  // largest number of kernels in one descriptor block (0 when the blob has none)
 };
 static_assert(sizeof(BlobHeader) <= 768, "header must fit its slot");
 constexpr size_t kHeaderBytes = 768;
@@ -29,6 +31,8 @@ constexpr size_t kHeaderBytes = 768;
 struct BlobLayout {
   size_t perm, fptr, pptr, chan, w4;   // canonical section
   size_t xfilt, tptr, tmeta, tw4;      // execution section (its own filter order, see pack.cu)
+  size_t dboff, dblk;                  // descriptor blocks (fp16 blobs with F % 32 == 0 and C % 16 == 0; else empty)
+  int nblk;                            // number of descriptor blocks = (F / 32) * nct, or 0
   size_t scratch;                      // pack-time temporaries: hist[F][K], count[F], inv[F], xinv[F], xbase[F]
   size_t total;
   int nct;                             // number of 16-channel tiles = ceil(C / 16)
@@ -52,6 +56,9 @@ __host__ __device__ inline BlobLayout blob_layout(int F, int C, int K, int64_t n
   L.tptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)L.nct + 1));
   L.tmeta = o; o = align256(o + sizeof(uint32_t) * nk);
   L.tw4 = o;   o = align256(o + 4 * e * nk);
+  L.nblk = (dtype == PAT_F16 && F % kExecGroup == 0 && C % kChanTile == 0) ? (F / kExecGroup) * L.nct : 0;
+  L.dboff = o; o = align256(o + (L.nblk ? sizeof(uint32_t) * ((size_t)L.nblk + 1) : 0));
+  L.dblk = o;  o = align256(o + (L.nblk ? (size_t)L.nblk * kBlockHeaderBytes + 16 * nk : 0));
   L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 4));
   L.total = o;
   return L;
@@ -80,6 +87,34 @@ __host__ __device__ inline void mask_bits(uint32_t m, int bits[4]) {
   for (int b = 0; b < 9 && t < 4; ++b)
     if (m & (1u << b)) bits[t++] = b;
   for (; t < 4; ++t) bits[t] = 4;
+}
+
+// ---- execution codes of the fp16 convolution kernels (written into the blob's descriptor blocks by pat_pack)
+// Compiled pattern codes.  A pattern whose top row is empty is the same shape one row lower, so it runs the
+// code of the shifted-up pattern on a window that starts one row lower: the twelve built-in patterns need ten
+// codes (the eight patterns of Section 4.2 need six).  Any other pattern takes the generic code (kGenericCode).
+constexpr int kNumCodes = 10;
+constexpr int kGenericCode = 15;
+__host__ __device__ constexpr uint32_t code_mask(int i) {
+  constexpr uint32_t m[kNumCodes] = {0x03A, 0x017, 0x0B2, 0x09A, 0x01B, 0x036, 0x093, 0x03C, 0x192, 0x00F};
+  return m[i];
+}
+__host__ __device__ constexpr int nth_bit(uint32_t mask, int t) {
+  int seen = 0;
+  for (int b = 0; b < 9; ++b)
+    if (mask & (1u << b)) { if (seen == t) return b; ++seen; }
+  return 4;
+}
+
+// descriptor word: bits 0-3 channel inside the block, 4-12 pattern mask, 13-16 code, 17 window row shift
+__host__ __device__ inline uint32_t pattern_word(uint32_t mask) {
+  const uint32_t shift = (mask & 7u) == 0u ? 1u : 0u;
+  const uint32_t norm = mask >> (3u * shift);
+  uint32_t code = kGenericCode;
+  for (int i = 0; i < kNumCodes; ++i)
+    if (code_mask(i) == norm) code = (uint32_t)i;
+  if (code == (uint32_t)kGenericCode) return (mask << 4) | (code << 13);
+  return (mask << 4) | (code << 13) | (shift << 17);
 }
 
 }  // namespace pat

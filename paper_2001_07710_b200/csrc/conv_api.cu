@@ -7,12 +7,16 @@ int conv_generic(const void* blob, int F, int C, const uint16_t* masks, int K, i
 bool conv_f16_fast_supported(int F, int C, const uint16_t* masks, int K, int dtype, int N, int H, int W, int stride);
 int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                   const void* x, void* y, int N, int H, int W, cudaStream_t st);
+bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride);
+size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
+int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st);
 }
 
 using namespace pat;
 
-extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                           int dtype, const void* x, void* y, int N, int H, int W, int stride, void* stream) {
+static int check_conv_args(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep, int dtype,
+                           const void* x, const void* y, int N, int H, int W, int stride) {
   if (!blob || !x || !y) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3: null pointer");
   if (F < 1 || C < 1 || F > 65535 || C > 65535) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: F=%d C=%d outside 1..65535", F, C);
   if (int rc = check_library(masks, K)) return rc;
@@ -24,8 +28,31 @@ extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks
   if (!aligned(x, 16) || !aligned(y, 16)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3: x and y must be 16-byte aligned");
   const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
   if ((size_t)N * ((Ho + 7) / 8) * ((Wo + 31) / 32) > 0x7FFFFFFFull) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: too many tiles");
+  return PAT_OK;
+}
+
+extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                           int dtype, const void* x, void* y, int N, int H, int W, int stride, void* stream) {
+  if (int rc = check_conv_args(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride)) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (conv_f16_fast_supported(F, C, masks, K, dtype, N, H, W, stride))
     return conv_f16_fast(blob, F, C, masks, K, n_keep, x, y, N, H, W, st);
   return conv_generic(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, st);
+}
+
+extern "C" size_t pat_conv3x3_workspace(int F, int C, int dtype, int N, int H, int W, int stride) {
+  if (F < 1 || C < 1 || N < 1 || H < 1 || W < 1) return 0;
+  return conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
+}
+
+extern "C" int pat_conv3x3_ws(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                              int dtype, const void* x, void* y, int N, int H, int W, int stride,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+  if (int rc = check_conv_args(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride)) return rc;
+  const size_t need = conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
+  if (need == 0) return pat_conv3x3(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, stream);
+  if (!workspace || workspace_bytes < need)
+    return set_error(PAT_ERR_WORKSPACE, "pat_conv3x3_ws: workspace has %zu bytes, needs %zu", workspace_bytes, need);
+  if (!aligned(workspace, 256)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3_ws: workspace must be 256-byte aligned");
+  return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, workspace, reinterpret_cast<cudaStream_t>(stream));
 }

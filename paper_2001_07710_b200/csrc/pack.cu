@@ -22,6 +22,8 @@ struct BlobPtrs {
   int32_t* tptr;
   uint32_t* tmeta;
   void* tw4;
+  uint32_t* dboff;     // descriptor block -> offset inside dblk, in 16-byte units (nblk + 1 entries)
+  char* dblk;
   int32_t *hist, *cnt, *inv, *xinv, *xbase;
 };
 
@@ -38,6 +40,8 @@ __host__ __device__ inline BlobPtrs blob_ptrs(void* blob, const BlobLayout& L, i
   p.tptr = reinterpret_cast<int32_t*>(b + L.tptr);
   p.tmeta = reinterpret_cast<uint32_t*>(b + L.tmeta);
   p.tw4 = b + L.tw4;
+  p.dboff = reinterpret_cast<uint32_t*>(b + L.dboff);
+  p.dblk = b + L.dblk;
   p.hist = reinterpret_cast<int32_t*>(b + L.scratch);
   p.cnt = p.hist + (size_t)F * K;
   p.inv = p.cnt + F;
@@ -167,6 +171,7 @@ __global__ void __launch_bounds__(1024) k_pack_ptrs(int F, int C, int K, long lo
     h->n_keep = n_keep;
     h->total_bytes = total_bytes;
     for (int j = 0; j <= kMaxK; ++j) h->masks[j] = lib.m[j];
+    h->max_block_entries = 0;   // raised by k_pack_blocks
   }
 }
 
@@ -257,6 +262,46 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
   }
 }
 
+// Descriptor blocks of the fp16 convolution kernel that copies its kernel lists with one bulk copy per pipeline
+// stage.  One block per (group of 32 filters in execution order, 16-channel tile), groups major:
+//   header   32 words, one per filter slot of the group: first entry (bits 0-15) | number of entries (bits 16-31)
+//   entries  16 bytes per kept kernel, slot after slot, inside a slot in (pattern, channel) order:
+//            {channel inside the tile | pattern_word(mask), taps 0-1 (fp16 x2), taps 2-3 (fp16 x2), 0}
+// dboff[b] is the block's offset in 16-byte units.  Launched with one warp per block (lane = filter slot).
+__global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
+  const int blk = blockIdx.x, lane = threadIdx.x;
+  const int g = blk / nct, cb = blk % nct;
+  const int32_t* row = bp.tptr + (size_t)(g * kExecGroup + lane) * (nct + 1);
+  const int a = row[cb], n = row[cb + 1] - a;
+  int before = a - row[0];                 // kernels of this slot in earlier tiles
+  int incl = n;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += v;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
+  const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+  const int start = incl - n;
+  const uint32_t group_first = (uint32_t)bp.tptr[(size_t)(g * kExecGroup) * (nct + 1)];   // kernels of earlier groups
+  const uint32_t off16 = (uint32_t)blk * (kBlockHeaderBytes / 16) + group_first + (uint32_t)before;
+  if (lane == 0) {
+    bp.dboff[blk] = off16;
+    if (blk == nblk - 1) bp.dboff[nblk] = off16 + kBlockHeaderBytes / 16 + (uint32_t)tot;
+    atomicMax(&bp.hdr->max_block_entries, tot);
+  }
+  char* base = bp.dblk + (size_t)off16 * 16;
+  reinterpret_cast<uint32_t*>(base)[lane] = (uint32_t)start | ((uint32_t)n << 16);
+  uint4* ent = reinterpret_cast<uint4*>(base + kBlockHeaderBytes) + start;
+  const uint2* tw4 = static_cast<const uint2*>(bp.tw4);
+  for (int k = 0; k < n; ++k) {
+    const uint32_t mt = bp.tmeta[a + k];
+    const uint2 w = tw4[a + k];
+    ent[k] = make_uint4(((mt & 0xFFFFu) - (uint32_t)(cb * kChanTile)) | pattern_word(lib.m[mt >> 16]), w.x, w.y, 0u);
+  }
+}
+
 __device__ inline bool header_matches(const BlobHeader* h, int F, int C, int K, long long n_keep, int dtype, const MaskTable& lib) {
   if (h->magic != kBlobMagic || h->version != kBlobVersion) return false;
   if (h->F != F || h->C != C || h->K != K || h->dtype != dtype || h->n_keep != n_keep) return false;
@@ -337,6 +382,10 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
     }
   }
   count_launches(4);
+  if (L.nblk > 0) {
+    k_pack_blocks<<<L.nblk, 32, 0, st>>>(L.nct, L.nblk, lib, bp);
+    count_launches(1);
+  }
   return check_cuda(cudaGetLastError(), "pat_pack launch");
 }
 

@@ -148,9 +148,12 @@ TUNED_CASES = [
 ]
 
 
+@pytest.mark.parametrize("use_workspace", [True, False], ids=["workspace", "no_workspace"])
 @pytest.mark.parametrize("case", TUNED_CASES)
-def test_conv_tuned_f16_matches_oracle(case):
+def test_conv_tuned_f16_matches_oracle(case, use_workspace):
+    """Both tuned fp16 kernels: pat_conv3x3_ws (stage images in a workspace) and pat_conv3x3 (no workspace)."""
     N, H, W, C, F, K, num, den = case
+    assert (pc.pat_conv3x3_workspace(F, C, "f16", N, H, W, 1) > 0)
     rng = np.random.default_rng(hash(case) % (2 ** 32))
     w = workloads.make_weights(rng, F, C)
     x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
@@ -160,16 +163,34 @@ def test_conv_tuned_f16_matches_oracle(case):
     ref = oracle.conv3x3(stored_weights(wm_o, "f16"), x, 1)
     pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
     y = torch.full((N, H, W, F), float("nan"), dtype=torch.float16, device="cuda")
-    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y)
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y, use_workspace=use_workspace)
     assert pc.pat_query_status() == 0
     out = y.float().cpu().numpy()
     assert np.isfinite(out).all()                                   # every output element was written
     check_close(out, ref, "f16")
 
 
-def test_conv_tuned_f16_many_regions_dense_keep():
+def test_conv_workspace_entry_point_is_bit_identical():
+    """pat_conv3x3_ws adds the products of a filter in the same order as pat_conv3x3: identical fp16 results; a
+    caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
+    N, H, W, C, F, K = 6, 28, 28, 128, 96, 8
+    rng = np.random.default_rng(5)
+    w = workloads.make_weights(rng, F, C)
+    xt = torch.from_numpy(store(workloads.make_inputs(rng, N, H, W, C), "f16")).cuda()
+    masks = oracle.library(K)
+    n_keep = F * C // 8
+    _, _, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    ws = torch.full((pc.pat_conv3x3_workspace(F, C, "f16", N, H, W, 1),), 0xFF, dtype=torch.uint8, device="cuda")
+    y0 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1, use_workspace=False)
+    y1 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1, workspace=ws)
+    assert pc.pat_query_status() == 0
+    assert torch.equal(y0.view(torch.int16), y1.view(torch.int16))
+
+
+@pytest.mark.parametrize("use_workspace", [True, False], ids=["workspace", "no_workspace"])
+def test_conv_tuned_f16_many_regions_dense_keep(use_workspace):
     """Several work items per thread block (672 regions) and up to 16 kernels per filter and 16-channel block
-    (keep 1/2, 12 patterns); sampled against the oracle."""
+    (keep 1/2, 12 patterns; descriptor blocks too large for the five-slot ring); sampled against the oracle."""
     N, H, W, C, F, K = 12, 224, 224, 16, 128, 12
     rng = np.random.default_rng(99)
     w = workloads.make_weights(rng, F, C)
@@ -179,7 +200,7 @@ def test_conv_tuned_f16_many_regions_dense_keep():
     pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
     pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
     y = torch.full((N, H, W, F), float("nan"), dtype=torch.float16, device="cuda")
-    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y)
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y, use_workspace=use_workspace)
     assert pc.pat_query_status() == 0
     assert bool(torch.isfinite(y).all())
     coords = np.stack([rng.integers(0, N, 6000), rng.integers(0, H, 6000), rng.integers(0, W, 6000), rng.integers(0, F, 6000)], axis=1).astype(np.int32)
