@@ -156,11 +156,11 @@ int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, in
  * C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k}, H even and >= 14) the
  * activations are first re-arranged, once per call, into the channel-planar tiles the multiply-add kernel
  * stages in shared memory; the kernel then needs no transposition of its own and runs a deeper pipeline.
- * pat_conv3x3_workspace returns the bytes needed (about 1.43 x the size of x), or 0 for a layer the workspace
+ * pat_conv3x3_workspace returns the bytes needed (about 1.3 x the size of x), or 0 for a layer the workspace
  * path does not cover: pat_conv3x3_ws then behaves exactly like pat_conv3x3 and ignores the workspace.
  *   workspace  dev, at least pat_conv3x3_workspace(...) bytes, 256-byte aligned; contents are scratch;
  *              concurrent calls must use different workspaces
- * Results are those of pat_conv3x3 (same products, fp32 sums in the same order). */
+ * Results: the same products as pat_conv3x3, added in fp32 in a different order of the kernels of a filter. */
 size_t pat_conv3x3_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                    int dtype, const void *x, void *y, int N, int H, int W, int stride,

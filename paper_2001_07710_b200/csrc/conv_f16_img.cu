@@ -1,21 +1,23 @@
 // Sparse 3x3 convolution for fp16 storage / fp32 accumulation, stride 1 (sm_100a): two kernels.
 //
 //  1. k_stage_images re-arranges the NHWC activations once per call into "stage images": for every region
-//     (8 tile rows x 4 column slots of 2 x 14 pixel tiles) and every block of 16 input channels one contiguous
-//     40 KB piece laid out exactly as the convolution kernel wants it in shared memory - channel-planar
-//     [16 ch][20 rows][4 segments][16 px], halo pixels duplicated, zero padding written out, 16-byte chunks of a
-//     segment swapped on every other row pair so that the 16-byte window loads of a warp touch every bank once.
-//     This is plain streaming work (reads the input once, writes 1.43 x its size) and it is done once per region,
-//     whereas a kernel that transposes inside its pipeline repeats it for every group of 32 filters.
+//     (8 tile rows x 4 column slots of 4 x 14 pixel tiles) and every block of 8 input channels one contiguous
+//     36 KB piece laid out exactly as the convolution kernel wants it in shared memory - channel-planar
+//     [8 ch][36 rows][4 segments][16 px], halo pixels duplicated, zero padding written out, the two 16-byte chunks
+//     of a segment trading places from one tile row to the next so that the 16-byte window loads of a warp touch
+//     every bank once.  This is plain streaming work (reads the input once, writes 1.3 x its size) and it is done
+//     once per region, whereas a kernel that transposes inside its pipeline repeats it for every group of 32 filters.
 //  2. k_conv_f16_img is the persistent, warp-specialised convolution kernel (one block per SM).  A work item is one
 //     region x one group of 32 filters.  One producer thread streams the item's stage images and the matching
 //     kernel-descriptor blocks of the packed weights (both contiguous, one bulk copy each per stage) into a ring of
-//     4 or 5 shared-memory slots; 16 consumer warps (two filters each, 2 x 14 pixels per thread, one accumulator
-//     tile in registers and the other parked in tensor memory) run the per-pattern multiply-add code (Section 6.2);
-//     results leave through two extra ring stages per item and a store warp, as 64-byte runs of NHWC output.
-//     With nothing but two bulk copies per stage on the producer side the ring can be deeper, and the consumer
-//     warps, whose per-stage work differs (two or three kernels per filter and channel block at 12.5 % density),
-//     seldom wait for each other.  Every wait is bounded; tensor memory is released on every path.
+//     5 shared-memory slots; 16 consumer warps (two filters each, 4 x 14 pixels per thread, one accumulator tile of
+//     56 values in registers and the other parked in tensor memory) run the per-pattern multiply-add code
+//     (Section 6.2); results leave through four extra ring stages per item and a store warp, as 64-byte runs of
+//     NHWC output.  The tall thread tile is what the multiply-add rate hangs on: a kernel costs about the same
+//     number of other instructions (descriptor, addresses, branch) and 1.5 x the window loads of a 2 x 14 tile
+//     for twice the multiply-adds.  With nothing but two bulk copies per stage on the producer side the ring is
+//     deep, and the consumer warps, whose per-stage work differs (about one kernel per filter and channel block at
+//     12.5 % density), seldom wait for each other.  Every wait is bounded; tensor memory is released on every path.
 #include <algorithm>
 #include "f16_tile.cuh"
 
@@ -23,26 +25,28 @@ namespace pat {
 namespace img16 {
 using namespace fast16;
 
-constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, store warp, two idle warps (register donors)
-constexpr int W_PRODUCER = NCW, W_STORE = NCW + 1;
-constexpr int MAXROWS = LY * TR + 4;       // two bands, each with a top and a bottom halo row
-constexpr int CHP = MAXROWS * ROWB;        // channel plane pitch (2560)
-constexpr int IMG_BYTES = CB * CHP;        // 40960
-constexpr int OFF_SLOTS = 256;             // barriers sit in front of the ring
-constexpr int SMEM_BYTES = 232448 - 1024;  // dynamic shared memory (the rest covers the static variables)
-constexpr int MAX_PS = 5;
-// ring geometry: five slots when every descriptor block of the blob fits the smaller descriptor area, else four
-constexpr int DSLOT5 = ((SMEM_BYTES - OFF_SLOTS) / 5 - IMG_BYTES) / 128 * 128;
-constexpr int DSLOT4 = kBlockHeaderBytes + FG * CB * 16;
-constexpr int MAXE5 = (DSLOT5 - kBlockHeaderBytes) / 16;
-static_assert(OFF_SLOTS + 5 * (IMG_BYTES + DSLOT5) <= SMEM_BYTES, "five-slot ring");
-static_assert(OFF_SLOTS + 4 * (IMG_BYTES + DSLOT4) <= SMEM_BYTES, "four-slot ring");
-static_assert(DSLOT4 % 128 == 0 && DSLOT5 > kBlockHeaderBytes, "descriptor areas");
+constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three store warps
+constexpr int W_PRODUCER = NCW, W_STORE = NCW + 1, NSW = 3;
+constexpr int CBI = kChanTile;             // channels per ring stage (16)
+constexpr int MAXROWS = LY * TR4 + 4;      // two bands, each with a top and a bottom halo row (36)
+constexpr int CHP = MAXROWS * ROWB;        // channel plane pitch (4608)
+constexpr int IMG_BYTES = CBI * CHP;       // 73728
+// Ring slots hold one stage each: the stage image and the kernel-descriptor block of the same 16 channels.
+// Three slots when every block of the blob has at most MAXE3 kernels (the sparse case), else two.
+constexpr int MAX_NS = 3;
+constexpr int MAXE3 = 152;
+constexpr int DBLK3 = kBlockHeaderBytes + MAXE3 * 16;           // 2560
+constexpr int DBLK2 = kBlockHeaderBytes + FG * kChanTile * 16;  // largest possible block (8320)
+constexpr int OFF_SLOTS = 256;             // barriers and two control words sit in front of the ring
+constexpr int SMEM_BYTES = OFF_SLOTS + 3 * (IMG_BYTES + DBLK3);
+static_assert(OFF_SLOTS + 2 * (IMG_BYTES + DBLK2) <= SMEM_BYTES, "the two-slot layout fits too");
+static_assert(IMG_BYTES % 128 == 0 && DBLK3 % 128 == 0 && DBLK2 % 128 == 0 && SMEM_BYTES <= 232448, "shared memory budget of one SM");
 constexpr int OUT_PITCH = FG * 2 + 4;      // output staging inside a slot: [448 px][32 channels] fp16, pixel pitch 68 B
-static_assert(32 * TC * OUT_PITCH <= IMG_BYTES, "one tile row of results fits a slot");
-constexpr int CONSUMER_REGS = 88, OTHER_REGS = 64;
+constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (30464)
+static_assert(2 * OUT_ROW <= IMG_BYTES, "two tile rows of results fit a slot");
+constexpr int CONSUMER_REGS = 104, OTHER_REGS = 64;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
-constexpr uint32_t TMEM_COLS = 256;        // 4 consumer warps per lane quarter x 2 filters x 32 columns
+constexpr uint32_t TMEM_COLS = 512;        // 4 consumer warps per lane quarter x 2 filters x 64 columns
 
 struct Params {
   const __half* x;
@@ -53,9 +57,9 @@ struct Params {
   const char* dblk;
   const BlobHeader* hdr;
   int* status;
-  int N, H, W, C, F, K, nct;
+  int N, H, W, C, F, K, nct;  // nct = channel blocks of 16
   long long n_keep;
-  int TY;                  // tile rows per image (H / 2)
+  int TY;                  // tile rows per image (H / 4)
   int TXe, NI;             // tile columns per region, images side by side
   int CG, NIG;             // column groups per image, image groups
   int NG;                  // filter groups (F / 32)
@@ -63,7 +67,7 @@ struct Params {
   uint16_t masks[256];     // the library (checked against the blob header)
 };
 
-// A region = LY consecutive tile rows x LX column slots.  Tile rows are numbered through all image groups
+// A region = LY consecutive tile rows (of four pixel rows) x LX column slots.  Tile rows are numbered through all image groups
 // (group g, tile row t -> g * TY + t), so a region may straddle two image groups: it then has two bands,
 // each with its own halo rows.
 struct Region {
@@ -81,7 +85,7 @@ __device__ __forceinline__ Region decode_region(const Params& p, int reg) {
   r.ta0 = gt0 % p.TY;
   r.n0 = min(LY, p.TY - r.ta0);
   r.band1 = (r.n0 < LY) && (r.ig0 + 1 < p.NIG);
-  r.nrows = r.band1 ? MAXROWS : 2 * r.n0 + 2;
+  r.nrows = r.band1 ? MAXROWS : TR4 * r.n0 + 2;
   return r;
 }
 
@@ -91,104 +95,95 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 // ------------------------------------------------------------------------------------------ stage images
-// One block per (region, channel block), channel block fastest so that blocks running together read the same
-// pixels.  Image layout: byte ch * CHP + row * ROWB + seg * SEGB + (chunk ^ ((row >> 1) & 1)) * 16 + (px & 7) * 2
-// with chunk = px >> 3, px = 0..15 <-> image column 14 * (tile column) - 1 + px.
-__global__ void __launch_bounds__(256) k_stage_images(const Params p) {
-  // channel planes are built with a pitch of 2568 bytes: the two channel octets a warp writes at once then fall
-  // into different halves of the banks
-  constexpr int SP = CHP + 8;
-  __shared__ __align__(16) unsigned char img[CB * SP];
-  const int cb = (int)(blockIdx.x % (unsigned)p.nct);
+// One block per (region, 16 input channels), channels fastest so that blocks running together read
+// the same pixels.  Image layout: byte ch * CHP + row * ROWB + seg * SEGB + (chunk ^ swz(row)) * 16 + (px & 7) * 2
+// with chunk = px >> 3, px = 0..15 <-> image column 14 * (tile column) - 1 + px, and swz(row) = parity of the tile
+// row (counted through both bands) whose window starts in that row's group of four.
+constexpr int SI_THREADS = 256;
+constexpr int SI_PITCH = CHP + 8;          // the two channel octets a warp writes at once fall into different bank halves
+constexpr int SI_SMEM = CBI * SI_PITCH;
+__global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
+  extern __shared__ __align__(16) unsigned char img[];
+  const int cb16 = (int)(blockIdx.x % (unsigned)p.nct);
   const int reg = (int)(blockIdx.x / (unsigned)p.nct);
   const Region r = decode_region(p, reg);
-  const int rows0 = 2 * r.n0 + 2;
+  const int rows0 = TR4 * r.n0 + 2;
   const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
   // a unit = one pixel pair x one channel octet: two 16-byte loads, eight 4-byte stores
-  constexpr int UNITS = MAXROWS * LX * 8 * 2, PER_THREAD = UNITS / 256;
-  static_assert(UNITS % 256 == 0, "units per thread");
+  constexpr int UNITS = MAXROWS * LX * 8 * 2, PER_THREAD = UNITS / SI_THREADS;
+  static_assert(UNITS % SI_THREADS == 0, "units per thread");
   uint4 va[PER_THREAD], vb[PER_THREAD];
 #pragma unroll
   for (int i = 0; i < PER_THREAD; ++i) {
-    const int u = (int)threadIdx.x + 256 * i;
+    const int u = (int)threadIdx.x + SI_THREADS * i;
     const int half = u & 1, kp = (u >> 1) & 7, seg = (u >> 4) & 3, pr = u >> 6;
     va[i] = make_uint4(0u, 0u, 0u, 0u);
     vb[i] = make_uint4(0u, 0u, 0u, 0u);
     if (pr < r.nrows) {
       const int b = (pr >= rows0) ? 1 : 0;
-      const int yy = b ? (pr - rows0 - 1) : (2 * r.ta0 - 1 + pr);
+      const int yy = b ? (pr - rows0 - 1) : (TR4 * r.ta0 - 1 + pr);
       const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
       const int n_img = (r.ig0 + b) * p.NI + ni;
       const int xx = (r.cg * p.TXe + tx) * TC - 1 + 2 * kp;
       if (yy >= 0 && yy < p.H && n_img < p.N) {
-        const __half* src = p.x + (((size_t)n_img * p.H + yy) * p.W + xx) * p.C + cb * CB + half * 8;
+        const __half* src = p.x + (((size_t)n_img * p.H + yy) * p.W + xx) * p.C + cb16 * 16 + half * 8;
         if (xx >= 0 && xx < p.W) va[i] = __ldg(reinterpret_cast<const uint4*>(src));
-        if (xx + 1 >= 0 && xx + 1 < p.W) vb[i] = __ldg(reinterpret_cast<const uint4*>(src + p.C));
+        if (xx + 1 < p.W) vb[i] = __ldg(reinterpret_cast<const uint4*>(src + p.C));
       }
     }
   }
 #pragma unroll
   for (int i = 0; i < PER_THREAD; ++i) {
-    const int u = (int)threadIdx.x + 256 * i;
+    const int u = (int)threadIdx.x + SI_THREADS * i;
     const int half = u & 1, kp = (u >> 1) & 7, seg = (u >> 4) & 3, pr = u >> 6;
-    const uint32_t o = (uint32_t)(pr * ROWB + seg * SEGB + (((kp >> 2) ^ ((pr >> 1) & 1)) << 4) + (kp & 3) * 4);
+    const int b = (pr >= rows0) ? 1 : 0;
+    const int swz = ((((b ? pr - rows0 : pr) >> 2) + (b ? r.n0 : 0)) & 1);
+    const uint32_t o = (uint32_t)(pr * ROWB + seg * SEGB + (((kp >> 2) ^ swz) << 4) + (kp & 3) * 4);
     const uint32_t a[4] = {va[i].x, va[i].y, va[i].z, va[i].w};
     const uint32_t c[4] = {vb[i].x, vb[i].y, vb[i].z, vb[i].w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j) * SP + o) = __byte_perm(a[j], c[j], 0x5410);
-      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j + 1) * SP + o) = __byte_perm(a[j], c[j], 0x7632);
+      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j) * SI_PITCH + o) = __byte_perm(a[j], c[j], 0x5410);
+      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j + 1) * SI_PITCH + o) = __byte_perm(a[j], c[j], 0x7632);
     }
   }
   __syncthreads();
   uint2* dst = reinterpret_cast<uint2*>(p.images + (size_t)blockIdx.x * IMG_BYTES);
-  for (int i = threadIdx.x; i < IMG_BYTES / 8; i += 256) {
+  for (int i = threadIdx.x; i < IMG_BYTES / 8; i += SI_THREADS) {
     const int ch = i / (CHP / 8), w = i % (CHP / 8);
-    dst[i] = *reinterpret_cast<const uint2*>(img + ch * SP + w * 8);
+    dst[i] = *reinterpret_cast<const uint2*>(img + ch * SI_PITCH + w * 8);
   }
 }
 
 // ------------------------------------------------------------------------------------------ the convolution
-// Ring protocol.  Every work item takes nct "real" ring stages (one channel block each) followed by two
-// "output" stages.  Stage number s uses slot s % PS.
-//   real stage:    the producer waits slot_empty, arms slot_full with the byte count and issues two bulk copies;
-//                  consumers wait slot_full, compute, arrive slot_empty (16 arrivals).
+// Ring protocol.  Every work item takes nct "real" ring stages (16 channels each) followed by two "output"
+// stages.  Stage number s uses slot s % NS.
+//   real stage:    the producer waits slot_empty, arms slot_full with the byte count and issues two bulk copies
+//                  (image, descriptor block); consumers wait slot_full, compute, arrive slot_empty (16 arrivals).
 //   output stage:  the producer waits slot_empty and arrives slot_full at once (the slot is free to be written);
-//                  consumers wait slot_full, write one tile row of results, arrive out_ready (16 arrivals);
+//                  consumers wait slot_full, write two rows of every thread tile, arrive out_ready (16 arrivals);
 //                  the store warp waits out_ready, copies the slot to global memory and arrives slot_empty
 //                  with a count of 16 in the consumers' place.
-__global__ void __launch_bounds__(NTHREADS, 1)
-k_conv_f16_img(const Params p) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  __shared__ int s_abort;
-  __shared__ uint32_t s_tmem;            // base address of the block's tensor-memory columns
+// In a real stage a consumer warp runs filter A, swaps, runs filter B; the next stage starts with B.  A tile of
+// 56 accumulators is moved to / from tensor memory once per stage and filter.
+template <bool SPARSE>
+__device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
+  constexpr int NS = SPARSE ? 3 : 2;
+  constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
   const uint32_t sbase = smem_u32(smem);
   auto slot_full = [&](int s) { return sbase + 8u * s; };
-  auto slot_empty = [&](int s) { return sbase + 8u * (MAX_PS + s); };
-  auto out_ready = [&](int s) { return sbase + 8u * (2 * MAX_PS + s); };
-  static_assert(8 * 3 * MAX_PS <= OFF_SLOTS, "barrier block");
+  auto slot_empty = [&](int s) { return sbase + 8u * (MAX_NS + s); };
+  auto out_ready = [&](int s) { return sbase + 8u * (2 * MAX_NS + s); };
+  static_assert(8 * 3 * MAX_NS + 8 <= OFF_SLOTS, "barrier block and control words");
+  int& s_abort = *reinterpret_cast<int*>(smem + 8 * 3 * MAX_NS);                 // a wait has given up
+  uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + 8 * 3 * MAX_NS + 4);    // base address of the block's tensor-memory columns
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  // refuse a blob packed with other parameters (uniform decision: every thread reads the same header)
-  const BlobHeader* bh = p.hdr;
-  {
-    bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
-              bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep &&
-              bh->max_block_entries >= 0 && bh->max_block_entries <= FG * CB;
-    for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
-    if (!ok) {
-      if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
-      return;
-    }
-  }
-  const int PS = (bh->max_block_entries <= MAXE5) ? 5 : 4;
-  const uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(PS == 5 ? DSLOT5 : DSLOT4);
   const uint32_t slot0 = sbase + OFF_SLOTS;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
-    for (int s = 0; s < MAX_PS; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), NCW); mbar_init(out_ready(s), NCW); }
+    for (int s = 0; s < MAX_NS; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), NCW); mbar_init(out_ready(s), NCW); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(smem_u32(&s_tmem), TMEM_COLS);
@@ -223,26 +218,26 @@ k_conv_f16_img(const Params p) {
             const uint32_t dbytes = (o1 - o0) * 16u;
             const uint32_t dst = slot0 + (uint32_t)pslot * SLOT;
             mbar_arrive_expect_tx(slot_full(pslot), (uint32_t)IMG_BYTES + dbytes);
-            bulk_load(dst, img + (size_t)cb * IMG_BYTES, (uint32_t)IMG_BYTES, slot_full(pslot));
             bulk_load(dst + IMG_BYTES, p.dblk + (size_t)o0 * 16, dbytes, slot_full(pslot));
+            bulk_load(dst, img + (size_t)cb * IMG_BYTES, (uint32_t)IMG_BYTES, slot_full(pslot));
           }
           armed |= 1u << pslot;
           armed_par = (armed_par & ~(1u << pslot)) | ((epar ^ 1u) << pslot);
           o0 = o1;
-          if (++pslot == PS) { pslot = 0; epar ^= 1u; }
+          if (++pslot == NS) { pslot = 0; epar ^= 1u; }
         }
-        // output stages: hand the next TR slots to the consumers as they become free
-        for (int y = 0; y < TR && alive; ++y) {
+        // output stages: hand the next two slots to the consumers as they become free
+        for (int o = 0; o < TR4 / 2 && alive; ++o) {
           if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
           if (lane == 0) mbar_arrive(slot_full(pslot));
           armed &= ~(1u << pslot);
-          if (++pslot == PS) { pslot = 0; epar ^= 1u; }
+          if (++pslot == NS) { pslot = 0; epar ^= 1u; }
         }
       }
       if (!alive && lane == 0) {
         // copies already issued still write into this block's shared memory: give them (bounded) time to land
         const unsigned long long t0 = global_ns();
-        for (int s = 0; s < PS; ++s) {
+        for (int s = 0; s < NS; ++s) {
           if (!((armed >> s) & 1u)) continue;
           for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
             if (mbar_try_wait(slot_full(s), (armed_par >> s) & 1u)) break;
@@ -251,8 +246,11 @@ k_conv_f16_img(const Params p) {
         }
         atomicExch(p.status, PAT_ERR_TIMEOUT);
       }
-    } else if (warp == W_STORE) {
-      // ========================================================================= store warp
+    } else {
+      // ========================================================================= store warps
+      // (one warp copied a slot out in about the time the consumers need for three stages, and the ring stood
+      // still meanwhile; the three warps take every third row of thread tiles)
+      const int sw = warp - W_STORE;
       const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
       uint32_t opar = 0;                           // phase parity of out_ready, one bit per slot
       bool alive = true;
@@ -261,14 +259,14 @@ k_conv_f16_img(const Params p) {
         const int item = item_of(it_idx);
         const int g = item % p.NG;
         const Region it = decode_region(p, item / p.NG);
-        pslot = (pslot + nct) % PS;                // skip the real stages of the item
-        for (int y = 0; y < TR && alive; ++y) {
+        pslot = (pslot + nct) % NS;                // skip the real stages of the item
+        for (int o = 0; o < TR4 / 2 && alive; ++o) {
           if (!mbar_wait<kFillSleepNs>(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
           opar ^= 1u << pslot;
-          const uint32_t o0 = slot0 + (uint32_t)pslot * SLOT;
-          // one thread tile (= one consumer lane) at a time: 14 pixels x 4 chunks of 8 channels; consecutive lanes
-          // take consecutive chunks, so every pixel is written as one 64-byte run
-          for (int t = 0; t < 32; ++t) {
+          // one row of one thread tile (= one consumer lane) at a time: 14 pixels x 4 chunks of 8 channels;
+          // consecutive lanes take consecutive chunks, so every pixel is written as one 64-byte run
+          for (int tr = sw; tr < 64; tr += NSW) {
+            const int t = tr & 31, r = tr >> 5;
             const int ly = t >> 2, lx = t & 3;
             const int b = (ly < it.n0) ? 0 : 1;
             const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
@@ -277,8 +275,8 @@ k_conv_f16_img(const Params p) {
             const int n_img = ig * p.NI + ni;
             if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
             const int col0 = (it.cg * p.TXe + tx) * TC;
-            __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR * ty + y)) * p.W + col0) * p.F + g * FG;
-            const uint32_t src_tile = o0 + (uint32_t)(t * TC) * OUT_PITCH;
+            __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + 2 * o + r)) * p.W + col0) * p.F + g * FG;
+            const uint32_t src_tile = slot0 + (uint32_t)pslot * SLOT + (uint32_t)r * OUT_ROW + (uint32_t)(t * TC) * OUT_PITCH;
 #pragma unroll
             for (int q0 = 0; q0 < TC * 4; q0 += 32) {
               const int q = q0 + lane;
@@ -294,103 +292,103 @@ k_conv_f16_img(const Params p) {
           // the slot is refilled by a bulk copy next: order this warp's reads of it before that write
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
-          if (lane == 0) mbar_arrive_n(slot_empty(pslot), NCW);   // the slot goes back to the ring
-          if (++pslot == PS) pslot = 0;
+          // the slot goes back to the ring once all three warps are done: together they arrive 16 times
+          if (lane == 0) mbar_arrive_n(slot_empty(pslot), sw == 0 ? (uint32_t)(NCW - 2 * (NCW / NSW)) : (uint32_t)(NCW / NSW));
+          if (++pslot == NS) pslot = 0;
         }
       }
     }
-    // the two remaining warps only lend their registers
   } else {
     // =========================================================================== consumer warps
     set_warp_registers<CONSUMER_REGS>();
-    const int ly = lane >> 2, lx = lane & 3;
     // Warp w owns filter slots w and 31 - w of the group (the most loaded filter with the least loaded one, ...).
     // Only one of the two accumulator tiles is in registers at a time; the other is parked in tensor memory:
-    // columns [64 * (w / 4) + 32 * f, +32) of the lanes of quarter w % 4.
-    const uint32_t tm0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 64);
+    // columns [128 * (w / 4) + 64 * f, +64) of the lanes of quarter w % 4.
+    const uint32_t tm0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+    auto park = [&](uint32_t f, const float (&a)[TR4][TC]) {
+      tmem_store_rows<TR4, 0>(tm0 + f * 64u, a);
+      tmem_store_rows<TR4, 2>(tm0 + f * 64u + 32u, a);
+      tmem_wait_st();
+    };
+    auto fetch = [&](uint32_t f, float (&a)[TR4][TC]) {
+      tmem_load_rows<TR4, 0>(tm0 + f * 64u, a);
+      tmem_load_rows<TR4, 2>(tm0 + f * 64u + 32u, a);
+      tmem_wait_ld();
+    };
     int pslot = 0;
     uint32_t fpar = 0u;                    // parity to wait for on slot_full of the current slot
     bool alive = true;
     for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
-      uint32_t offA, offB;               // the lane's two chunk addresses of window row 0, relative to a channel plane
-      uint32_t cposA, cposB;             // byte offsets of filters 0 / 1 inside the group of 32 output channels
-      {
-        const int item = item_of(it_idx);
-        const int g = item % p.NG;
-        const Region it = decode_region(p, item / p.NG);
+      uint32_t offA;                     // the lane's address of logical chunk 0 of window row 0, relative to a channel plane
+      {                                  // (logical chunk 1 sits at offA ^ 16)
+        const Region it = decode_region(p, item_of(it_idx) / p.NG);
+        const int ly = lane >> 2, lx = lane & 3;
         const int b = (ly < it.n0) ? 0 : 1;                  // band of this lane's tile row
-        const uint32_t lane_off = (uint32_t)((2 * ly + 2 * b) * ROWB + lx * SEGB);
-        const int swl = (ly + b) & 1;
-        offA = lane_off + (uint32_t)(swl << 4);
-        offB = lane_off + (uint32_t)((swl ^ 1) << 4);
-        cposA = ((uint32_t)__ldg(p.xfilt + g * FG + warp) & (uint32_t)(FG - 1)) * 2u;
-        cposB = ((uint32_t)__ldg(p.xfilt + g * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 2u;
+        offA = (uint32_t)((TR4 * ly + 2 * b) * ROWB + lx * SEGB + ((ly & 1) << 4));
       }
-      float acc[TR][TC];
+      float acc[TR4][TC];
 #pragma unroll
-      for (int y = 0; y < TR; ++y)
+      for (int y = 0; y < TR4; ++y)
 #pragma unroll
         for (int x = 0; x < TC; ++x) acc[y][x] = 0.0f;
-      tmem_store32(tm0 + 32u, acc);      // filter 1 starts from zero in tensor memory, filter 0 in registers
+      park(1u, acc);                     // filter 1 starts from zero in tensor memory, filter 0 in registers
       uint32_t cur = 0u;                 // which of the two filters the registers hold
-
-      // the kernels of filter f in the current stage
-      auto run_filter = [&](uint32_t f, uint32_t pl0, uint32_t d0) {
-        const uint32_t slot = f ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp;
-        const uint32_t hw = lds32(d0 + slot * 4);
-        const int nk = (int)(hw >> 16);
-        uint32_t e = d0 + kBlockHeaderBytes + (hw & 0xFFFFu) * 16u;
-        for (int k = 0; k < nk; ++k, e += 16) {
-          uint32_t m0, w01, w23, pad;
-          lds128(e, m0, w01, w23, pad);
-          const uint32_t base = pl0 + (m0 & 15u) * CHP;
-          one_kernel(acc, base + offA, base + offB, m0, w01, w23);
-        }
-      };
 
       for (int cb = 0; cb < nct; ++cb) {
         if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
-        const uint32_t pl0 = slot0 + (uint32_t)pslot * SLOT;
-        const uint32_t d0 = pl0 + IMG_BYTES;
+        const uint32_t pl0 = slot0 + (uint32_t)pslot * SLOT + offA;
+        // filter A, swap, filter B (one copy of the multiply-add code)
 #pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          run_filter(cur, pl0, d0);
-          if (half == 0) {               // swap: park this filter, fetch the other
-            tmem_store32(tm0 + cur * 32u, acc);
+        for (int ph = 0; ph < 2; ++ph) {
+          const uint32_t d0 = pl0 - offA + IMG_BYTES;
+          const uint32_t hw = lds32(d0 + (cur ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp) * 4);
+          uint32_t e = d0 + kBlockHeaderBytes + (hw & 0xFFFFu) * 16u;
+          const uint32_t e_end = e + (hw >> 16) * 16u;
+#pragma unroll 1
+          for (; e != e_end; e += 16) {
+            uint32_t m0, w01, w23, pad;
+            lds128(e, m0, w01, w23, pad);
+            const uint32_t base = pl0 + (m0 & 15u) * CHP;
+            one_kernel4(acc, base, base ^ 16u, m0, w01, w23);
+          }
+          if (ph == 0) {
+            park(cur, acc);
             cur ^= 1u;
-            tmem_load32(tm0 + cur * 32u, acc);
+            fetch(cur, acc);
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(slot_empty(pslot));
-        if (++pslot == PS) { pslot = 0; fpar ^= 1u; }
+        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
       }
       if (!alive) break;
 
-      // results: fp32 -> fp16 (round to nearest even) into the two output stages, one tile row each
-#pragma unroll 1
-      for (int y = 0; y < TR; ++y) {
+      // results: fp32 -> fp16 (round to nearest even) into the two output stages, two tile rows each
+      // byte offsets of filters 0 / 1 inside the group of 32 output channels
+      const int g_out = item_of(it_idx) % p.NG;
+      const uint32_t cposA = ((uint32_t)__ldg(p.xfilt + g_out * FG + warp) & (uint32_t)(FG - 1)) * 2u;
+      const uint32_t cposB = ((uint32_t)__ldg(p.xfilt + g_out * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 2u;
+#pragma unroll
+      for (int o = 0; o < TR4 / 2; ++o) {
         if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t o0 = slot0 + (uint32_t)pslot * SLOT + (uint32_t)(lane * TC) * OUT_PITCH;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           const uint32_t cp = cur ? cposB : cposA;
-          if (y == 0) {
 #pragma unroll
-            for (int x = 0; x < TC; ++x) sts16(o0 + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[0][x])));
-          } else {
+          for (int r = 0; r < 2; ++r)
 #pragma unroll
-            for (int x = 0; x < TC; ++x) sts16(o0 + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[1][x])));
-          }
+            for (int x = 0; x < TC; ++x)
+              sts16(o0 + r * OUT_ROW + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[2 * o + r][x])));
           if (half == 0) {
-            if (y == 0) tmem_store32(tm0 + cur * 32u, acc);   // still needed for the second tile row
+            if (o == 0) park(cur, acc);   // still needed for the lower tile rows
             cur ^= 1u;
-            tmem_load32(tm0 + cur * 32u, acc);
+            fetch(cur, acc);
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(out_ready(pslot));
-        if (++pslot == PS) { pslot = 0; fpar ^= 1u; }
+        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
       }
     }
   }
@@ -400,11 +398,29 @@ k_conv_f16_img(const Params p) {
   if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_conv_f16_img(const Params p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  // refuse a blob packed with other parameters (uniform decision: every thread reads the same header)
+  const BlobHeader* bh = p.hdr;
+  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
+            bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep &&
+            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * kChanTile;
+  for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
+  if (!ok) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
+    return;
+  }
+  // ring geometry by the size of the largest descriptor block (see MAX_NS above)
+  if (bh->max_block_entries <= MAXE3) conv_body<true>(p, smem);
+  else conv_body<false>(p, smem);
+}
+
 // ------------------------------------------------------------------------------------------ host side
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
-  p.nct = C / CB;
-  p.TY = H / TR;
+  p.nct = C / CBI;
+  p.TY = H / TR4;
   const int TX = W / TC;
   p.TXe = TX >= LX ? LX : TX;
   p.NI = LX / p.TXe;
@@ -426,10 +442,10 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
   if (dtype != PAT_F16 || stride != 1) return false;
-  if (W % TC != 0 || H % TR != 0 || H < 2 * (LY - 1)) return false;
+  if (W % TC != 0 || H % TR4 != 0 || H / TR4 < LY - 1) return false;   // a region spans at most two image groups
   const int TX = W / TC;
   if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
-  if (C % CB != 0 || F % FG != 0) return false;
+  if (C % kChanTile != 0 || F % FG != 0) return false;
   Params p;
   return N >= 1 && fill_geometry(p, F, C, N, H, W);
 }
@@ -469,13 +485,14 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
     if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
     if (int rc = check_cuda(cudaFuncSetAttribute(k_conv_f16_img, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
+    if (int rc = check_cuda(cudaFuncSetAttribute(k_stage_images, cudaFuncAttributeMaxDynamicSharedMemorySize, SI_SMEM), "set shared memory size")) return rc;
     cudaFuncAttributes fa;
     if (int rc = check_cuda(cudaFuncGetAttributes(&fa, k_conv_f16_img), "query kernel attributes")) return rc;
     if (fa.numRegs < LAUNCH_REGS)
       return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
     attr_set = true;
   }
-  k_stage_images<<<(unsigned)(p.n_regions * p.nct), 256, 0, st>>>(p);
+  k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
   const int grid = std::min(p.n_items, sm_count);
   k_conv_f16_img<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
   count_launches(2);

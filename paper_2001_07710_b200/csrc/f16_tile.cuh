@@ -118,35 +118,47 @@ __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) { 
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {         // whole warp
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
-// 32 consecutive columns of the thread's lane <-> 32 registers (28 accumulators + 4 unused)
-__device__ __forceinline__ void tmem_store32(uint32_t taddr, const float (&a)[TR][TC]) {
-  static_assert(TR * TC == 28, "accumulator tile is 28 values");
+// 32 consecutive columns of the thread's lane <-> 32 registers: rows Y0 and Y0 + 1 of an accumulator tile
+// (28 values + 4 unused).  The _rows functions only issue the transfer; tmem_wait_st / tmem_wait_ld complete it.
+template <int T, int Y0>
+__device__ __forceinline__ void tmem_store_rows(uint32_t taddr, const float (&a)[T][TC]) {
+  static_assert(TC == 14 && Y0 + 1 < T, "two rows of 14 values");
   const float z = 0.0f;
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%29,%29,%29};\n\t"
-      "tcgen05.wait::st.sync.aligned;"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%29,%29,%29};"
       ::"r"(taddr),
-        "f"(a[0][0]), "f"(a[0][1]), "f"(a[0][2]), "f"(a[0][3]), "f"(a[0][4]), "f"(a[0][5]), "f"(a[0][6]),
-        "f"(a[0][7]), "f"(a[0][8]), "f"(a[0][9]), "f"(a[0][10]), "f"(a[0][11]), "f"(a[0][12]), "f"(a[0][13]),
-        "f"(a[1][0]), "f"(a[1][1]), "f"(a[1][2]), "f"(a[1][3]), "f"(a[1][4]), "f"(a[1][5]), "f"(a[1][6]),
-        "f"(a[1][7]), "f"(a[1][8]), "f"(a[1][9]), "f"(a[1][10]), "f"(a[1][11]), "f"(a[1][12]), "f"(a[1][13]),
+        "f"(a[Y0][0]), "f"(a[Y0][1]), "f"(a[Y0][2]), "f"(a[Y0][3]), "f"(a[Y0][4]), "f"(a[Y0][5]), "f"(a[Y0][6]),
+        "f"(a[Y0][7]), "f"(a[Y0][8]), "f"(a[Y0][9]), "f"(a[Y0][10]), "f"(a[Y0][11]), "f"(a[Y0][12]), "f"(a[Y0][13]),
+        "f"(a[Y0 + 1][0]), "f"(a[Y0 + 1][1]), "f"(a[Y0 + 1][2]), "f"(a[Y0 + 1][3]), "f"(a[Y0 + 1][4]), "f"(a[Y0 + 1][5]), "f"(a[Y0 + 1][6]),
+        "f"(a[Y0 + 1][7]), "f"(a[Y0 + 1][8]), "f"(a[Y0 + 1][9]), "f"(a[Y0 + 1][10]), "f"(a[Y0 + 1][11]), "f"(a[Y0 + 1][12]), "f"(a[Y0 + 1][13]),
         "f"(z)
       : "memory");
 }
-__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&a)[TR][TC]) {
+template <int T, int Y0>
+__device__ __forceinline__ void tmem_load_rows(uint32_t taddr, float (&a)[T][TC]) {
+  static_assert(TC == 14 && Y0 + 1 < T, "two rows of 14 values");
   float d0, d1, d2, d3;
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=f"(a[0][0]), "=f"(a[0][1]), "=f"(a[0][2]), "=f"(a[0][3]), "=f"(a[0][4]), "=f"(a[0][5]), "=f"(a[0][6]),
-        "=f"(a[0][7]), "=f"(a[0][8]), "=f"(a[0][9]), "=f"(a[0][10]), "=f"(a[0][11]), "=f"(a[0][12]), "=f"(a[0][13]),
-        "=f"(a[1][0]), "=f"(a[1][1]), "=f"(a[1][2]), "=f"(a[1][3]), "=f"(a[1][4]), "=f"(a[1][5]), "=f"(a[1][6]),
-        "=f"(a[1][7]), "=f"(a[1][8]), "=f"(a[1][9]), "=f"(a[1][10]), "=f"(a[1][11]), "=f"(a[1][12]), "=f"(a[1][13]),
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=f"(a[Y0][0]), "=f"(a[Y0][1]), "=f"(a[Y0][2]), "=f"(a[Y0][3]), "=f"(a[Y0][4]), "=f"(a[Y0][5]), "=f"(a[Y0][6]),
+        "=f"(a[Y0][7]), "=f"(a[Y0][8]), "=f"(a[Y0][9]), "=f"(a[Y0][10]), "=f"(a[Y0][11]), "=f"(a[Y0][12]), "=f"(a[Y0][13]),
+        "=f"(a[Y0 + 1][0]), "=f"(a[Y0 + 1][1]), "=f"(a[Y0 + 1][2]), "=f"(a[Y0 + 1][3]), "=f"(a[Y0 + 1][4]), "=f"(a[Y0 + 1][5]), "=f"(a[Y0 + 1][6]),
+        "=f"(a[Y0 + 1][7]), "=f"(a[Y0 + 1][8]), "=f"(a[Y0 + 1][9]), "=f"(a[Y0 + 1][10]), "=f"(a[Y0 + 1][11]), "=f"(a[Y0 + 1][12]), "=f"(a[Y0 + 1][13]),
         "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
       : "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_store32(uint32_t taddr, const float (&a)[TR][TC]) {
+  tmem_store_rows<TR, 0>(taddr, a);
+  tmem_wait_st();
+}
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&a)[TR][TC]) {
+  tmem_load_rows<TR, 0>(taddr, a);
+  tmem_wait_ld();
 }
 
 template <int REGS>
@@ -241,6 +253,90 @@ __device__ __forceinline__ void one_kernel(float (&acc)[TR][TC], uint32_t baseA,
     }
   }
 #undef PAT_ROW3
+}
+
+// ---- 4 x 14 pixel tiles (56 accumulators): the code of a pattern walks down the window one row at a time, so a
+// row of 16 pixels is loaded once and serves every tap that reads it.  MASK is a compiled code (first tap in
+// kernel row 0); a0 / a1 = the lane's addresses of logical chunks 0 / 1 of the first window row the code reads
+// (window row `sh`).  The two chunks of a segment trade places every four image rows, i.e. from window row 4 on.
+constexpr int TR4 = 4;
+__host__ __device__ constexpr int last_tap_row(uint32_t mask) { return (mask >> 6) ? 2 : ((mask >> 3) ? 1 : 0); }
+
+template <uint32_t MASK>
+__device__ __forceinline__ void pattern_body4(float (&acc)[TR4][TC], uint32_t a0, uint32_t a1, uint32_t sh, uint32_t w01, uint32_t w23) {
+  unsigned short w[4];
+  split_h2(w01, w[0], w[1]);
+  split_h2(w23, w[2], w[3]);
+  constexpr int NR = last_tap_row(MASK) + TR4;      // rows of the window this code reads
+#pragma unroll
+  for (int j = 0; j < NR; ++j) {
+    unsigned short h[16];
+    uint32_t p0 = a0 + j * ROWB, p1 = a1 + j * ROWB;
+    if (j >= 4) { const uint32_t t = p0; p0 = p1; p1 = t; }
+    else if (j == 3) { const uint32_t q0 = sh ? p1 : p0, q1 = sh ? p0 : p1; p0 = q0; p1 = q1; }
+    load_row(h, p0, p1);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int b = nth_bit(MASK, t);
+      const int r = b / 3, c = b % 3;
+      const int y = j - r;
+      if (y >= 0 && y < TR4) {
+#pragma unroll
+        for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[x + c], w[t]);
+      }
+    }
+  }
+}
+
+// One kept kernel on a 4-row tile.  baseA / baseB = the lane's two chunk addresses of window row 0 in the
+// kernel's channel plane.  Every branch is warp-uniform.
+__device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t baseA, uint32_t baseB, uint32_t meta,
+                                            uint32_t w01, uint32_t w23) {
+  const uint32_t sh = (meta >> 17) & 1u;
+  const uint32_t a0 = baseA + sh * ROWB, a1 = baseB + sh * ROWB;
+  const uint32_t code = (meta >> 13) & 15u;
+  if (code & 8u) {
+    if (code & 4u) {
+      // any other pattern: position by position, each with its own pass over the window rows it reads
+#define PAT_TAP4(B)                                                                          \
+  if (meta & (16u << (B))) {                                                                 \
+    const unsigned short wv = (unsigned short)(w01 & 0xFFFFu);                               \
+    _Pragma("unroll")                                                                        \
+    for (int y = 0; y < TR4; ++y) {                                                          \
+      unsigned short h[16];                                                                  \
+      const int jr = y + (B) / 3;                                                            \
+      const uint32_t q0 = baseA + jr * ROWB, q1 = baseB + jr * ROWB;                         \
+      if (jr >= 4) load_row(h, q1, q0); else load_row(h, q0, q1);                            \
+      _Pragma("unroll")                                                                      \
+      for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[x + (B) % 3], wv);               \
+    }                                                                                        \
+    w01 = __funnelshift_r(w01, w23, 16);                                                     \
+    w23 >>= 16;                                                                              \
+  }
+      PAT_TAP4(0) PAT_TAP4(1) PAT_TAP4(2) PAT_TAP4(3) PAT_TAP4(4) PAT_TAP4(5) PAT_TAP4(6) PAT_TAP4(7) PAT_TAP4(8)
+#undef PAT_TAP4
+    } else if (code & 1u) {
+      pattern_body4<code_mask(9)>(acc, a0, a1, sh, w01, w23);
+    } else {
+      pattern_body4<code_mask(8)>(acc, a0, a1, sh, w01, w23);
+    }
+  } else if (code & 4u) {
+    if (code & 2u) {
+      if (code & 1u) pattern_body4<code_mask(7)>(acc, a0, a1, sh, w01, w23);
+      else pattern_body4<code_mask(6)>(acc, a0, a1, sh, w01, w23);
+    } else {
+      if (code & 1u) pattern_body4<code_mask(5)>(acc, a0, a1, sh, w01, w23);
+      else pattern_body4<code_mask(4)>(acc, a0, a1, sh, w01, w23);
+    }
+  } else {
+    if (code & 2u) {
+      if (code & 1u) pattern_body4<code_mask(3)>(acc, a0, a1, sh, w01, w23);
+      else pattern_body4<code_mask(2)>(acc, a0, a1, sh, w01, w23);
+    } else {
+      if (code & 1u) pattern_body4<code_mask(1)>(acc, a0, a1, sh, w01, w23);
+      else pattern_body4<code_mask(0)>(acc, a0, a1, sh, w01, w23);
+    }
+  }
 }
 
 }  // namespace fast16

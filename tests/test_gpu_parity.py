@@ -145,6 +145,11 @@ TUNED_CASES = [
     (1, 224, 224, 16, 32, 8, 1, 8),
     (7, 16, 14, 16, 32, 8, 1, 1),
     (2, 14, 28, 256, 32, 8, 1, 8),
+    # heights that are multiples of 4 (>= 28) also take the workspace kernels (4-row thread tiles)
+    (5, 28, 14, 64, 32, 8, 1, 8),
+    (2, 32, 112, 48, 64, 8, 3, 10),
+    (3, 44, 28, 32, 32, 4, 1, 2),
+    (9, 28, 28, 16, 32, 12, 1, 1),
 ]
 
 
@@ -153,7 +158,7 @@ TUNED_CASES = [
 def test_conv_tuned_f16_matches_oracle(case, use_workspace):
     """Both tuned fp16 kernels: pat_conv3x3_ws (stage images in a workspace) and pat_conv3x3 (no workspace)."""
     N, H, W, C, F, K, num, den = case
-    assert (pc.pat_conv3x3_workspace(F, C, "f16", N, H, W, 1) > 0)
+    assert (pc.pat_conv3x3_workspace(F, C, "f16", N, H, W, 1) > 0) == (H % 4 == 0 and H >= 28)
     rng = np.random.default_rng(hash(case) % (2 ** 32))
     w = workloads.make_weights(rng, F, C)
     x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
@@ -170,9 +175,9 @@ def test_conv_tuned_f16_matches_oracle(case, use_workspace):
     check_close(out, ref, "f16")
 
 
-def test_conv_workspace_entry_point_is_bit_identical():
-    """pat_conv3x3_ws adds the products of a filter in the same order as pat_conv3x3: identical fp16 results; a
-    caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
+def test_conv_workspace_entry_point_agrees_with_plain_entry_point():
+    """pat_conv3x3_ws and pat_conv3x3 add the kernels of a filter in different orders: fp16 results agree to a
+    rounding step; a caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
     N, H, W, C, F, K = 6, 28, 28, 128, 96, 8
     rng = np.random.default_rng(5)
     w = workloads.make_weights(rng, F, C)
@@ -184,7 +189,8 @@ def test_conv_workspace_entry_point_is_bit_identical():
     y0 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1, use_workspace=False)
     y1 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1, workspace=ws)
     assert pc.pat_query_status() == 0
-    assert torch.equal(y0.view(torch.int16), y1.view(torch.int16))
+    assert bool(torch.isfinite(y1).all())
+    assert torch.allclose(y0.float(), y1.float(), rtol=2e-3, atol=2e-4)
 
 
 @pytest.mark.parametrize("use_workspace", [True, False], ids=["workspace", "no_workspace"])
