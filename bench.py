@@ -132,6 +132,9 @@ def run_ours(args):
             st["ws"] = torch.empty(pc.pat_project_workspace(L.F, L.C), dtype=torch.uint8, device="cuda")
             st["blob"] = torch.empty(pc.pat_pack_size(L.F, L.C, L.K, L.n_keep, dtype), dtype=torch.uint8, device="cuda")
         layers.append(st)
+    # one workspace for the stage images of pat_conv3x3_ws, sized for the largest layer (layers run one after another)
+    cws_bytes = max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg.layers if not L.dense] + [0])
+    cws = torch.empty(max(cws_bytes, 256), dtype=torch.uint8, device="cuda")
 
     def step(conv_events=None):
         for i, st in enumerate(layers):
@@ -144,7 +147,7 @@ def run_ours(args):
                 pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
                 pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
                 if conv_events is not None: conv_events[i][0].record(stream)
-                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"])
+                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
                 if conv_events is not None: conv_events[i][1].record(stream)
 
     def step_e2e():
@@ -157,7 +160,7 @@ def run_ours(args):
             else:
                 pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
                 pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
-                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"])
+                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
             st["hy"].copy_(st["y"], non_blocking=True)
 
     def barrier():

@@ -25,8 +25,8 @@ namespace pat {
 namespace img16 {
 using namespace fast16;
 
-constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three store warps
-constexpr int W_PRODUCER = NCW, W_STORE = NCW + 1, NSW = 3;
+constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three idle warps (register donors)
+constexpr int W_PRODUCER = NCW;
 constexpr int CBI = kChanTile;             // channels per ring stage (16)
 constexpr int MAXROWS = LY * TR4 + 4;      // two bands, each with a top and a bottom halo row (36)
 constexpr int CHP = MAXROWS * ROWB;        // channel plane pitch (4608)
@@ -43,7 +43,7 @@ static_assert(OFF_SLOTS + 2 * (IMG_BYTES + DBLK2) <= SMEM_BYTES, "the two-slot l
 static_assert(IMG_BYTES % 128 == 0 && DBLK3 % 128 == 0 && DBLK2 % 128 == 0 && SMEM_BYTES <= 232448, "shared memory budget of one SM");
 constexpr int OUT_PITCH = FG * 2 + 4;      // output staging inside a slot: [448 px][32 channels] fp16, pixel pitch 68 B
 constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (30464)
-static_assert(2 * OUT_ROW <= IMG_BYTES, "two tile rows of results fit a slot");
+static_assert(2 * OUT_ROW <= IMG_BYTES && 32 % NCW == 0, "two tile rows of results fit a slot");
 constexpr int CONSUMER_REGS = 104, OTHER_REGS = 64;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 512;        // 4 consumer warps per lane quarter x 2 filters x 64 columns
@@ -160,10 +160,12 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
 // stages.  Stage number s uses slot s % NS.
 //   real stage:    the producer waits slot_empty, arms slot_full with the byte count and issues two bulk copies
 //                  (image, descriptor block); consumers wait slot_full, compute, arrive slot_empty (16 arrivals).
-//   output stage:  the producer waits slot_empty and arrives slot_full at once (the slot is free to be written);
-//                  consumers wait slot_full, write two rows of every thread tile, arrive out_ready (16 arrivals);
-//                  the store warp waits out_ready, copies the slot to global memory and arrives slot_empty
-//                  with a count of 16 in the consumers' place.
+//   output stages: the producer waits slot_empty and arrives slot_full at once (the slot is free to be written);
+//                  consumers wait slot_full of both, write their results (tile rows 0-1 into the first, 2-3 into
+//                  the second slot), arrive out_ready and wait for it (16 arrivals: every warp has written),
+//                  copy two thread tiles each to global memory and arrive slot_empty of both slots.
+//                  (A separate store warp shares the issue slots of its SM partition with four consumer warps and
+//                  needed longer for a slot than the consumers for two stages: the ring stood still meanwhile.)
 // In a real stage a consumer warp runs filter A, swaps, runs filter B; the next stage starts with B.  A tile of
 // 56 accumulators is moved to / from tensor memory once per stage and filter.
 template <bool SPARSE>
@@ -246,58 +248,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         }
         atomicExch(p.status, PAT_ERR_TIMEOUT);
       }
-    } else {
-      // ========================================================================= store warps
-      // (one warp copied a slot out in about the time the consumers need for three stages, and the ring stood
-      // still meanwhile; the three warps take every third row of thread tiles)
-      const int sw = warp - W_STORE;
-      const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
-      uint32_t opar = 0;                           // phase parity of out_ready, one bit per slot
-      bool alive = true;
-      int pslot = 0;
-      for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
-        const int item = item_of(it_idx);
-        const int g = item % p.NG;
-        const Region it = decode_region(p, item / p.NG);
-        pslot = (pslot + nct) % NS;                // skip the real stages of the item
-        for (int o = 0; o < TR4 / 2 && alive; ++o) {
-          if (!mbar_wait<kFillSleepNs>(out_ready(pslot), (opar >> pslot) & 1u, abort_flag)) { alive = false; break; }
-          opar ^= 1u << pslot;
-          // one row of one thread tile (= one consumer lane) at a time: 14 pixels x 4 chunks of 8 channels;
-          // consecutive lanes take consecutive chunks, so every pixel is written as one 64-byte run
-          for (int tr = sw; tr < 64; tr += NSW) {
-            const int t = tr & 31, r = tr >> 5;
-            const int ly = t >> 2, lx = t & 3;
-            const int b = (ly < it.n0) ? 0 : 1;
-            const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
-            const int ig = it.ig0 + b;
-            const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
-            const int n_img = ig * p.NI + ni;
-            if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
-            const int col0 = (it.cg * p.TXe + tx) * TC;
-            __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + 2 * o + r)) * p.W + col0) * p.F + g * FG;
-            const uint32_t src_tile = slot0 + (uint32_t)pslot * SLOT + (uint32_t)r * OUT_ROW + (uint32_t)(t * TC) * OUT_PITCH;
-#pragma unroll
-            for (int q0 = 0; q0 < TC * 4; q0 += 32) {
-              const int q = q0 + lane;
-              if (q < TC * 4) {
-                const int x = q >> 2, j = q & 3;
-                const uint32_t src = src_tile + x * OUT_PITCH + j * 16;
-                uint4 v;
-                v.x = lds32(src); v.y = lds32(src + 4); v.z = lds32(src + 8); v.w = lds32(src + 12);
-                *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = v;
-              }
-            }
-          }
-          // the slot is refilled by a bulk copy next: order this warp's reads of it before that write
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          // the slot goes back to the ring once all three warps are done: together they arrive 16 times
-          if (lane == 0) mbar_arrive_n(slot_empty(pslot), sw == 0 ? (uint32_t)(NCW - 2 * (NCW / NSW)) : (uint32_t)(NCW / NSW));
-          if (++pslot == NS) pslot = 0;
-        }
-      }
     }
+    // the other three warps only lend their registers
   } else {
     // =========================================================================== consumer warps
     set_warp_registers<CONSUMER_REGS>();
@@ -363,33 +315,79 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       }
       if (!alive) break;
 
-      // results: fp32 -> fp16 (round to nearest even) into the two output stages, two tile rows each
+      // results: fp32 -> fp16 (round to nearest even) into the two output stages (tile rows 0-1 and 2-3), then,
+      // once all 16 warps have written, every warp copies two thread tiles to global memory
+      const int item = item_of(it_idx);
+      const int g_out = item % p.NG;
       // byte offsets of filters 0 / 1 inside the group of 32 output channels
-      const int g_out = item_of(it_idx) % p.NG;
       const uint32_t cposA = ((uint32_t)__ldg(p.xfilt + g_out * FG + warp) & (uint32_t)(FG - 1)) * 2u;
       const uint32_t cposB = ((uint32_t)__ldg(p.xfilt + g_out * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 2u;
-#pragma unroll
-      for (int o = 0; o < TR4 / 2; ++o) {
-        if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
-        const uint32_t o0 = slot0 + (uint32_t)pslot * SLOT + (uint32_t)(lane * TC) * OUT_PITCH;
+      const int s0 = pslot, s1 = (pslot + 1 == NS) ? 0 : pslot + 1;
+      const uint32_t par1 = (pslot + 1 == NS) ? (fpar ^ 1u) : fpar;
+      if (!mbar_wait<0>(slot_full(s0), fpar, abort_flag)) { alive = false; break; }
+      if (!mbar_wait<0>(slot_full(s1), par1, abort_flag)) { alive = false; break; }
+      const uint32_t ob0 = slot0 + (uint32_t)s0 * SLOT, ob1 = slot0 + (uint32_t)s1 * SLOT;
+      {
+        const uint32_t ol = (uint32_t)(lane * TC) * OUT_PITCH;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
-          const uint32_t cp = cur ? cposB : cposA;
+          const uint32_t cp = ol + (cur ? cposB : cposA);
 #pragma unroll
-          for (int r = 0; r < 2; ++r)
+          for (int y = 0; y < TR4; ++y)
 #pragma unroll
             for (int x = 0; x < TC; ++x)
-              sts16(o0 + r * OUT_ROW + x * OUT_PITCH + cp, __half_as_ushort(__float2half_rn(acc[2 * o + r][x])));
+              sts16((y < 2 ? ob0 : ob1) + (uint32_t)((y & 1) * OUT_ROW + x * OUT_PITCH) + cp, __half_as_ushort(__float2half_rn(acc[y][x])));
           if (half == 0) {
-            if (o == 0) park(cur, acc);   // still needed for the lower tile rows
             cur ^= 1u;
             fetch(cur, acc);
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(out_ready(pslot));
-        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(out_ready(0));
+      if (!mbar_wait<0>(out_ready(0), (uint32_t)(it_idx & 1), abort_flag)) { alive = false; break; }
+      {
+        const Region it = decode_region(p, item / p.NG);
+        const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+        // 14 pixels x 4 chunks of 8 channels per tile row: consecutive lanes take consecutive chunks, so every pixel
+        // is written as one 64-byte run; all loads of a tile are issued before its stores
+        const uint32_t sl = (uint32_t)(lane >> 2) * OUT_PITCH + (uint32_t)(lane & 3) * 16u;
+#pragma unroll 1
+        for (int k = 0; k < 32 / NCW; ++k) {
+          const int t = warp * (32 / NCW) + k;
+          const int ly = t >> 2, lx = t & 3;
+          const int b = (ly < it.n0) ? 0 : 1;
+          const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+          const int ig = it.ig0 + b;
+          const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+          const int n_img = ig * p.NI + ni;
+          if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
+          const int col0 = (it.cg * p.TXe + tx) * TC;
+          __half* dst = p.y + (((size_t)n_img * p.H + TR4 * ty) * p.W + col0 + (lane >> 2)) * p.F + g_out * FG + (lane & 3) * 8;
+          const uint32_t src = sl + (uint32_t)(t * TC) * OUT_PITCH;
+          uint4 v[TR4][2];
+#pragma unroll
+          for (int y = 0; y < TR4; ++y)
+#pragma unroll
+            for (int part = 0; part < 2; ++part)
+              if (part == 0 || lane < 4 * (TC - 8)) {
+                const uint32_t a = (y < 2 ? ob0 : ob1) + src + (uint32_t)((y & 1) * OUT_ROW + part * (8 * OUT_PITCH));
+                v[y][part].x = lds32(a); v[y][part].y = lds32(a + 4); v[y][part].z = lds32(a + 8); v[y][part].w = lds32(a + 12);
+              }
+#pragma unroll
+          for (int y = 0; y < TR4; ++y)
+#pragma unroll
+            for (int part = 0; part < 2; ++part)
+              if (part == 0 || lane < 4 * (TC - 8))
+                *reinterpret_cast<uint4*>(dst + ((size_t)y * p.W + 8 * part) * p.F) = v[y][part];
+        }
+      }
+      // the slots are refilled by bulk copies next: order this warp's reads of them before those writes
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(slot_empty(s0)); mbar_arrive(slot_empty(s1)); }
+      for (int o = 0; o < TR4 / 2; ++o)
+        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
     }
   }
   // every warp comes here, also after a failed wait: the tensor memory must be given back before the block ends
