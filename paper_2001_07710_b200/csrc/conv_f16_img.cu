@@ -44,7 +44,7 @@ static_assert(IMG_BYTES % 128 == 0 && DBLK3 % 128 == 0 && DBLK2 % 128 == 0 && SM
 constexpr int OUT_PITCH = FG * 2 + 4;      // output staging inside a slot: [448 px][32 channels] fp16, pixel pitch 68 B
 constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (30464)
 static_assert(2 * OUT_ROW <= IMG_BYTES && 32 % NCW == 0, "two tile rows of results fit a slot");
-constexpr int CONSUMER_REGS = 104, OTHER_REGS = 64;
+constexpr int CONSUMER_REGS = 112, OTHER_REGS = 32;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 512;        // 4 consumer warps per lane quarter x 2 filters x 64 columns
 
@@ -64,6 +64,12 @@ struct Params {
   int CG, NIG;             // column groups per image, image groups
   int NG;                  // filter groups (F / 32)
   int n_regions, n_items;  // n_items = n_regions * NG
+  // Tail balancing: items [0, n_whole) are processed whole, one per block and round.  Each of the n_split items
+  // that would start another, mostly idle round is cut along the input channels into `parts` pieces that run on
+  // different blocks and write fp32 partial sums (`partials`: [piece][32 filters][56 values][32 lanes]);
+  // k_reduce_parts adds them up in a fixed order.  parts == 1: no cutting.
+  int n_whole, n_split, parts;
+  float* partials;
   uint16_t masks[256];     // the library (checked against the blob header)
 };
 
@@ -195,9 +201,19 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
   volatile int* abort_flag = &s_abort;
   const uint32_t tmem_base = s_tmem;
 
-  const int n_my_items = (p.n_items > (int)blockIdx.x) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  // work units of this block: whole items (item = region * NG + filter group), then at most one piece of a cut item
+  const int n_my_whole = (p.n_whole > (int)blockIdx.x) ? (p.n_whole - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int n_my_items = n_my_whole + ((p.parts > 1 && (int)blockIdx.x < p.n_split * p.parts) ? 1 : 0);
   const int nct = p.nct;
-  auto item_of = [&](int it_idx) { return (int)blockIdx.x + it_idx * (int)gridDim.x; };   // item = region * NG + filter group
+  auto item_of = [&](int it_idx) {
+    return it_idx < n_my_whole ? (int)blockIdx.x + it_idx * (int)gridDim.x : p.n_whole + (int)blockIdx.x / p.parts;
+  };
+  auto piece_of = [&](int it_idx, int& c0, int& c1) {   // channel blocks [c0, c1) of the unit; true for a piece
+    if (it_idx < n_my_whole) { c0 = 0; c1 = nct; return false; }
+    const int q = (int)blockIdx.x % p.parts;
+    c0 = q * nct / p.parts; c1 = (q + 1) * nct / p.parts;
+    return true;
+  };
 
   if (warp >= NCW) {
     set_warp_registers<OTHER_REGS>();
@@ -212,8 +228,10 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         const int g = item % p.NG, reg = item / p.NG;
         const char* img = p.images + (size_t)reg * nct * IMG_BYTES;
         const uint32_t* bo = p.dboff + (size_t)g * nct;
-        uint32_t o0 = __ldg(bo);
-        for (int cb = 0; cb < nct && alive; ++cb) {
+        int c0, c1;
+        const bool piece = piece_of(it_idx, c0, c1);
+        uint32_t o0 = __ldg(bo + c0);
+        for (int cb = c0; cb < c1 && alive; ++cb) {
           const uint32_t o1 = __ldg(bo + cb + 1);
           if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
           if (lane == 0) {
@@ -228,8 +246,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           o0 = o1;
           if (++pslot == NS) { pslot = 0; epar ^= 1u; }
         }
-        // output stages: hand the next two slots to the consumers as they become free
-        for (int o = 0; o < TR4 / 2 && alive; ++o) {
+        // output stages: hand the next two slots to the consumers as they become free (a piece has none)
+        for (int o = 0; o < TR4 / 2 && alive && !piece; ++o) {
           if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
           if (lane == 0) mbar_arrive(slot_full(pslot));
           armed &= ~(1u << pslot);
@@ -286,7 +304,9 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       park(1u, acc);                     // filter 1 starts from zero in tensor memory, filter 0 in registers
       uint32_t cur = 0u;                 // which of the two filters the registers hold
 
-      for (int cb = 0; cb < nct; ++cb) {
+      int c0, c1;
+      const bool piece = piece_of(it_idx, c0, c1);
+      for (int cb = c0; cb < c1; ++cb) {
         if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
         const uint32_t pl0 = slot0 + (uint32_t)pslot * SLOT + offA;
         // filter A, swap, filter B (one copy of the multiply-add code)
@@ -314,6 +334,24 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
       }
       if (!alive) break;
+
+      if (piece) {
+        // partial sums of a cut item: fp32, one 128-byte line per value and warp
+        float* dst = p.partials + (size_t)blockIdx.x * (FG * TR4 * TC * 32) + lane;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          float* d = dst + (size_t)(cur ? FG - 1 - warp : warp) * (TR4 * TC * 32);
+#pragma unroll
+          for (int y = 0; y < TR4; ++y)
+#pragma unroll
+            for (int x = 0; x < TC; ++x) d[(y * TC + x) * 32] = acc[y][x];
+          if (half == 0) {
+            cur ^= 1u;
+            fetch(cur, acc);
+          }
+        }
+        continue;
+      }
 
       // results: fp32 -> fp16 (round to nearest even) into the two output stages (tile rows 0-1 and 2-3), then,
       // once all 16 warps have written, every warp copies two thread tiles to global memory
@@ -414,6 +452,53 @@ k_conv_f16_img(const Params p) {
   else conv_body<false>(p, smem);
 }
 
+// ------------------------------------------------------------------------------------------ cut items
+// Adds the partial sums of the pieces of a cut item (piece 0 first) and writes the fp16 results.  One block per
+// (cut item, row of the thread tiles): the sums go through shared memory as [448 px][32 channels] and leave as
+// 64-byte runs, like the results of a whole item.
+constexpr int MAX_PIECES = 256;            // pieces in flight (the workspace holds that many partial tiles)
+constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
+constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
+__global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
+  __shared__ __align__(16) unsigned char stage[OUT_ROW];
+  const int li = (int)blockIdx.x / TR4, y = (int)blockIdx.x % TR4;
+  const int item = p.n_whole + li;
+  const int g = item % p.NG;
+  const Region it = decode_region(p, item / p.NG);
+  const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS;
+  for (int idx = threadIdx.x; idx < FG * TC * 32; idx += RP_THREADS) {
+    const int lane = idx & 31, x = (idx >> 5) % TC, slot = idx / (32 * TC);
+    const size_t e = ((size_t)slot * (TR4 * TC) + (size_t)(y * TC + x)) * 32 + lane;
+    float v[MAX_PARTS];
+#pragma unroll
+    for (int q = 0; q < MAX_PARTS; ++q) v[q] = (q < p.parts) ? __ldg(src + (size_t)q * PIECE_FLOATS + e) : 0.0f;   // all loads in flight
+    float sum = 0.0f;
+#pragma unroll
+    for (int q = 0; q < MAX_PARTS; ++q) sum += v[q];                                                           // piece 0 first
+    const int cpos = (__ldg(p.xfilt + g * FG + slot) & (FG - 1)) * 2;
+    *reinterpret_cast<__half*>(stage + (lane * TC + x) * OUT_PITCH + cpos) = __float2half_rn(sum);
+  }
+  __syncthreads();
+  const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = warp; t < 32; t += RP_THREADS / 32) {
+    const int ly = t >> 2, lx = t & 3;
+    const int b = (ly < it.n0) ? 0 : 1;
+    const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+    const int ig = it.ig0 + b;
+    const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+    const int n_img = ig * p.NI + ni;
+    if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
+    const int col0 = (it.cg * p.TXe + tx) * TC;
+    __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
+    for (int qq = lane; qq < TC * 4; qq += 32) {
+      const int x = qq >> 2, j = qq & 3;
+      const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + x) * OUT_PITCH + j * 16);
+      *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------ host side
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
@@ -431,6 +516,7 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   if (items > 0x7FFFFFFFll || regions * p.nct > 0x7FFFFFFFll) return false;
   p.n_regions = (int)regions;
   p.n_items = (int)items;
+  p.n_whole = p.n_items; p.n_split = 0; p.parts = 1; p.partials = nullptr;
   return true;
 }
 
@@ -454,7 +540,7 @@ size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
   if (!conv_f16_img_supported(F, C, dtype, N, H, W, stride)) return 0;
   Params p;
   fill_geometry(p, F, C, N, H, W);
-  return (size_t)p.n_regions * p.nct * IMG_BYTES;
+  return align256((size_t)p.n_regions * p.nct * IMG_BYTES) + MAX_PIECES * PIECE_FLOATS * sizeof(float);
 }
 
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
@@ -490,10 +576,23 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
       return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
     attr_set = true;
   }
-  k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
   const int grid = std::min(p.n_items, sm_count);
+  // the items of a last, mostly idle round are cut into up to eight pieces (see Params)
+  const int left = p.n_items % grid;
+  if (left > 0) {
+    const int parts = std::min(std::min(MAX_PARTS, p.nct), std::min(grid, MAX_PIECES) / left);
+    if (parts >= 2) {
+      p.n_whole = p.n_items - left; p.n_split = left; p.parts = parts;
+      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nct * IMG_BYTES));
+    }
+  }
+  k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
   k_conv_f16_img<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
   count_launches(2);
+  if (p.parts > 1) {
+    k_reduce_parts<<<(unsigned)(p.n_split * TR4), RP_THREADS, 0, st>>>(p);
+    count_launches(1);
+  }
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
 }
 

@@ -48,8 +48,8 @@ def test_sizes_are_pure_functions(lib):
     assert lib.pat_pack_size(64, 64, 8, 10, 2) == 0
     assert lib.pat_project_workspace(64, 64) >= 64 * 64 * 9
     assert lib.pat_project_workspace(0, 64) == 0
-    # stage images of the workspace path: 28 regions x 32 channel blocks x 36864 bytes; none for other layer kinds
-    assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 1) == 28 * 32 * 36864
+    # workspace path: stage images (28 regions x 16 channel blocks x 73728 bytes) + 256 partial tiles of cut items
+    assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 1) == 28 * 16 * 73728 + 256 * 32 * 56 * 32 * 4
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 14, 14, 1) == 0
     assert lib.pat_conv3x3_workspace(256, 256, 0, 16, 56, 56, 1) == 0
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 2) == 0
@@ -86,6 +86,6 @@ def test_argument_validation_launches_nothing(lib):
     assert lib.pat_conv3x3(fake, 4, 4, mp, 4, 2, 5, fake, fake, 1, 8, 8, 1, None) == E["dtype"]
     assert lib.pat_conv3x3_ws(fake, 4, 4, mp, 4, 2, 0, fake, fake, 1, 8, 8, 3, fake, 1 << 20, None) == E["arg"]
     assert lib.pat_conv3x3_ws(fake, 32, 16, mp, 4, 2, 1, fake, fake, 1, 28, 14, 1, fake, 16, None) == E["ws"]
-    assert lib.pat_conv3x3_ws(fake, 32, 16, mp, 4, 2, 1, fake, fake, 1, 28, 14, 1, mis, 1 << 20, None) == E["align"]
+    assert lib.pat_conv3x3_ws(fake, 32, 16, mp, 4, 2, 1, fake, fake, 1, 28, 14, 1, mis, 1 << 30, None) == E["align"]
     assert lib.pat_conv3x3_dense(fake, 8, 17, 0, fake, fake, 1, 8, 8, 1, None) == E["shape"]
     assert lib.pat_strerror(E["align"]) == b"misaligned pointer"

@@ -193,6 +193,30 @@ def test_conv_workspace_entry_point_agrees_with_plain_entry_point():
     assert torch.allclose(y0.float(), y1.float(), rtol=2e-3, atol=2e-4)
 
 
+def test_conv_workspace_cut_items():
+    """More work items than SMs with a remainder: the items of the last round are cut along the input channels,
+    run as pieces on different blocks and are added up by the reduce kernel; sampled against the oracle."""
+    N, H, W, C, F, K = 24, 56, 56, 64, 128, 8
+    rng = np.random.default_rng(77)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
+    masks = oracle.library(K)
+    n_keep = F * C // 8
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    y = torch.full((N, H, W, F), float("nan"), dtype=torch.float16, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, y=y)
+    assert pc.pat_query_status() == 0
+    assert bool(torch.isfinite(y).all())
+    coords = np.stack([rng.integers(0, N, 8000), rng.integers(0, H, 8000), rng.integers(0, W, 8000), rng.integers(0, F, 8000)], axis=1).astype(np.int32)
+    coords[:2000, 0] = rng.integers(20, 24, 2000)          # the last images belong to the cut items
+    ref = oracle.conv3x3_at(stored_weights(wm_o, "f16"), x, coords, 1)
+    out = y[coords[:, 0], coords[:, 1], coords[:, 2], coords[:, 3]].float().cpu().numpy()
+    check_close(out, ref, "f16")
+    y2 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", torch.from_numpy(x).cuda(), 1, use_workspace=False)
+    assert torch.allclose(y.float(), y2.float(), rtol=2e-3, atol=2e-4)
+
+
 @pytest.mark.parametrize("use_workspace", [True, False], ids=["workspace", "no_workspace"])
 def test_conv_tuned_f16_many_regions_dense_keep(use_workspace):
     """Several work items per thread block (672 regions) and up to 16 kernels per filter and 16-channel block
