@@ -59,7 +59,7 @@ struct Params {
   int* status;
   int N, H, W, C, F, K, nct;  // nct = channel blocks of 16
   long long n_keep;
-  int TY;                  // tile rows per image (H / 4)
+  int TY;                  // tile rows per image (ceil(H / 4))
   int TXe, NI;             // tile columns per region, images side by side
   int CG, NIG;             // column groups per image, image groups
   int NG;                  // filter groups (F / 32)
@@ -416,7 +416,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           for (int y = 0; y < TR4; ++y)
 #pragma unroll
             for (int part = 0; part < 2; ++part)
-              if (part == 0 || lane < 4 * (TC - 8))
+              if ((part == 0 || lane < 4 * (TC - 8)) && TR4 * ty + y < p.H)
                 *reinterpret_cast<uint4*>(dst + ((size_t)y * p.W + 8 * part) * p.F) = v[y][part];
         }
       }
@@ -488,7 +488,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
     const int ig = it.ig0 + b;
     const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
     const int n_img = ig * p.NI + ni;
-    if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
+    if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || TR4 * ty + y >= p.H) continue;
     const int col0 = (it.cg * p.TXe + tx) * TC;
     __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
     for (int qq = lane; qq < TC * 4; qq += 32) {
@@ -503,7 +503,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
   p.nct = C / CBI;
-  p.TY = H / TR4;
+  p.TY = (H + TR4 - 1) / TR4;   // a last, partly empty tile row when H is not a multiple of 4
   const int TX = W / TC;
   p.TXe = TX >= LX ? LX : TX;
   p.NI = LX / p.TXe;
@@ -526,7 +526,8 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
   if (dtype != PAT_F16 || stride != 1) return false;
-  if (W % TC != 0 || H % TR4 != 0 || H / TR4 < LY - 1) return false;   // a region spans at most two image groups
+  const int TY = (H + TR4 - 1) / TR4;
+  if (W % TC != 0 || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
   const int TX = W / TC;
   if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
   if (C % kChanTile != 0 || F % FG != 0) return false;

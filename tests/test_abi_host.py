@@ -50,7 +50,7 @@ def test_sizes_are_pure_functions(lib):
     assert lib.pat_project_workspace(0, 64) == 0
     # workspace path: stage images (28 regions x 16 channel blocks x 73728 bytes) + 256 partial tiles of cut items
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 1) == 28 * 16 * 73728 + 256 * 32 * 56 * 32 * 4
-    assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 14, 14, 1) == 0
+    assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 20, 14, 1) == 0
     assert lib.pat_conv3x3_workspace(256, 256, 0, 16, 56, 56, 1) == 0
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 2) == 0
     assert lib.pat_conv3x3_workspace(256, 250, 1, 16, 56, 56, 1) == 0
