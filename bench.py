@@ -178,15 +178,20 @@ def run_ours(args):
 
     # ---- the step as a CUDA graph: the ~200 small launches of a step (projection and packing kernels of twelve
     # layers) are then issued by the GPU front end without a host round trip each
-    gstream = torch.cuda.Stream()
-    graph = torch.cuda.CUDAGraph()
     launches0 = pc.pat_launch_count()
-    with torch.cuda.stream(gstream):
-        with torch.cuda.graph(graph, stream=gstream):
-            step()
+    if args.no_graph:                  # plain launches (for profilers, which see one kernel per launch that way)
+        step()
+        run_step = step
+    else:
+        gstream = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gstream):
+            with torch.cuda.graph(graph, stream=gstream):
+                step()
+        run_step = graph.replay
     launches_per_step = pc.pat_launch_count() - launches0
     for _ in range(2):
-        graph.replay()
+        run_step()
     barrier()
 
     # ---- timed region: device-resident inputs, K replays of the step
@@ -196,7 +201,7 @@ def run_ours(args):
     sampler.start()
     e0.record(stream)
     for k in range(args.steps):
-        graph.replay()
+        run_step()
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -252,7 +257,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 storage, f32 accumulate" if dtype == "f16" else "f32", "data": "synthetic",
         "config": {"workload": f"config {cfg.number}: {cfg.name}", "batch_per_gpu": N,
-                   "layers": len(layers), "step": "project + pack + conv for every layer, replayed as one CUDA graph",
+                   "layers": len(layers), "step": "project + pack + conv for every layer" + ("" if args.no_graph else ", replayed as one CUDA graph"),
                    "l2": "inputs larger than L2 (about 3.4 GB touched per step)", "seed": workloads.BASE_SEED},
         "effective_gflops": round(total_flop * world * args.steps / (ms_total * 1e-3) / 1e9, 1),
         "conv_only_images_per_s": round(world * N / (sum(conv_ms) * 1e-3), 2),
@@ -381,6 +386,7 @@ def main():
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="workload number (3 = VGG-16 batch 64 fp16 storage)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch size (profiling small cases)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()
     if args.impl == "reference":

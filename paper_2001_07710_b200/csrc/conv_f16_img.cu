@@ -455,47 +455,57 @@ k_conv_f16_img(const Params p) {
 // ------------------------------------------------------------------------------------------ cut items
 // Adds the partial sums of the pieces of a cut item (piece 0 first) and writes the fp16 results.  One block per
 // (cut item, row of the thread tiles): the sums go through shared memory as [448 px][32 channels] and leave as
-// 64-byte runs, like the results of a whole item.
+// 64-byte runs, like the results of a whole item.  One block per (cut item, row of the thread tiles, half of the
+// tile columns).
 constexpr int MAX_PIECES = 256;            // pieces in flight (the workspace holds that many partial tiles)
 constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
-constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
+constexpr int RP_THREADS = 1024, MAX_PARTS = 8, RP_XH = TC / 2;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   __shared__ __align__(16) unsigned char stage[OUT_ROW];
-  const int li = (int)blockIdx.x / TR4, y = (int)blockIdx.x % TR4;
+  // block = (cut item, row of the thread tiles, left or right half of the tile columns)
+  const int xh = (int)blockIdx.x & 1, y = ((int)blockIdx.x >> 1) % TR4, li = (int)blockIdx.x / (2 * TR4);
   const int item = p.n_whole + li;
   const int g = item % p.NG;
   const Region it = decode_region(p, item / p.NG);
   const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS;
-  for (int idx = threadIdx.x; idx < FG * TC * 32; idx += RP_THREADS) {
-    const int lane = idx & 31, x = (idx >> 5) % TC, slot = idx / (32 * TC);
-    const size_t e = ((size_t)slot * (TR4 * TC) + (size_t)(y * TC + x)) * 32 + lane;
-    float v[MAX_PARTS];
+  constexpr int PER_THREAD = FG * RP_XH * 32 / RP_THREADS;   // 7
+  static_assert(FG * RP_XH * 32 % RP_THREADS == 0, "elements per thread");
+  float v[PER_THREAD][MAX_PARTS];
 #pragma unroll
-    for (int q = 0; q < MAX_PARTS; ++q) v[q] = (q < p.parts) ? __ldg(src + (size_t)q * PIECE_FLOATS + e) : 0.0f;   // all loads in flight
+  for (int i = 0; i < PER_THREAD; ++i) {                      // all loads in flight
+    const int idx = (int)threadIdx.x + i * RP_THREADS;
+    const int lane = idx & 31, x = xh * RP_XH + (idx >> 5) % RP_XH, slot = idx / (32 * RP_XH);
+    const size_t e = ((size_t)slot * (TR4 * TC) + (size_t)(y * TC + x)) * 32 + lane;
+#pragma unroll
+    for (int q = 0; q < MAX_PARTS; ++q) v[i][q] = (q < p.parts) ? __ldg(src + (size_t)q * PIECE_FLOATS + e) : 0.0f;
+  }
+#pragma unroll
+  for (int i = 0; i < PER_THREAD; ++i) {
+    const int idx = (int)threadIdx.x + i * RP_THREADS;
+    const int lane = idx & 31, x = xh * RP_XH + (idx >> 5) % RP_XH, slot = idx / (32 * RP_XH);
     float sum = 0.0f;
 #pragma unroll
-    for (int q = 0; q < MAX_PARTS; ++q) sum += v[q];                                                           // piece 0 first
+    for (int q = 0; q < MAX_PARTS; ++q) sum += v[i][q];       // piece 0 first
     const int cpos = (__ldg(p.xfilt + g * FG + slot) & (FG - 1)) * 2;
     *reinterpret_cast<__half*>(stage + (lane * TC + x) * OUT_PITCH + cpos) = __float2half_rn(sum);
   }
   __syncthreads();
   const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int t = warp; t < 32; t += RP_THREADS / 32) {
-    const int ly = t >> 2, lx = t & 3;
-    const int b = (ly < it.n0) ? 0 : 1;
-    const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
-    const int ig = it.ig0 + b;
-    const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
-    const int n_img = ig * p.NI + ni;
-    if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || TR4 * ty + y >= p.H) continue;
-    const int col0 = (it.cg * p.TXe + tx) * TC;
-    __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
-    for (int qq = lane; qq < TC * 4; qq += 32) {
-      const int x = qq >> 2, j = qq & 3;
-      const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + x) * OUT_PITCH + j * 16);
-      *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
-    }
+  const int t = threadIdx.x >> 5, lane = threadIdx.x & 31;    // one warp per thread tile
+  static_assert(RP_THREADS == 32 * 32 && RP_XH * 4 <= 32, "one warp per tile, one lane per 16-byte chunk");
+  const int ly = t >> 2, lx = t & 3;
+  const int b = (ly < it.n0) ? 0 : 1;
+  const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+  const int ig = it.ig0 + b;
+  const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+  const int n_img = ig * p.NI + ni;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || TR4 * ty + y >= p.H) return;
+  const int col0 = (it.cg * p.TXe + tx) * TC;
+  __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
+  if (lane < RP_XH * 4) {
+    const int x = xh * RP_XH + (lane >> 2), j = lane & 3;
+    const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + x) * OUT_PITCH + j * 16);
+    *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
   }
 }
 
@@ -591,7 +601,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   k_conv_f16_img<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
   count_launches(2);
   if (p.parts > 1) {
-    k_reduce_parts<<<(unsigned)(p.n_split * TR4), RP_THREADS, 0, st>>>(p);
+    k_reduce_parts<<<(unsigned)(p.n_split * TR4 * 2), RP_THREADS, 0, st>>>(p);
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
