@@ -32,9 +32,9 @@ UNIT = "images/s"
 SM_COUNT, FMA_LANES, SM_MAX_MHZ = 148, 128, 1965.0
 FMA_PEAK_TFLOPS = 2 * FMA_LANES * SM_COUNT * SM_MAX_MHZ * 1e6 / 1e12     # 74.45: fp32 FMA, no tensor cores
 DEFAULT_CONFIG = 3
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_conv_f16_s1 launch (conv6 shape, batch 16), from
-# profiles/k_conv_f16_s1_conv6_b16.md
-CONV6_DRAM_BYTES_B16 = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_conv_f16_img launch (conv6 shape, batch 32), from
+# profiles/k_conv_f16_img_conv6_b32.md
+CONV6_DRAM_BYTES_B32 = 68.72e6 + 18.20e6
 
 
 def measured_peaks():
@@ -118,7 +118,8 @@ def run_ours(args):
 
     # ---- seeded host tensors (pinned: they are also the source of the end-to-end copies)
     layers = []
-    for L in cfg.layers:
+    cfg_layers = [L for L in cfg.layers if args.layers is None or L.name in args.layers.split(",")]
+    for L in cfg_layers:
         w_np, x_np = workloads.make_layer_tensors(cfg.number, L, N)
         hw = torch.from_numpy(w_np).pin_memory()
         hx = torch.from_numpy(x_np).to(tdt).pin_memory()
@@ -133,7 +134,7 @@ def run_ours(args):
             st["blob"] = torch.empty(pc.pat_pack_size(L.F, L.C, L.K, L.n_keep, dtype), dtype=torch.uint8, device="cuda")
         layers.append(st)
     # one workspace for the stage images of pat_conv3x3_ws, sized for the largest layer (layers run one after another)
-    cws_bytes = max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg.layers if not L.dense] + [0])
+    cws_bytes = max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg_layers if not L.dense] + [0])
     cws = torch.empty(max(cws_bytes, 256), dtype=torch.uint8, device="cuda")
 
     def step(conv_events=None):
@@ -261,17 +262,16 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (about 3.4 GB touched per step)", "seed": workloads.BASE_SEED},
         "effective_gflops": round(total_flop * world * args.steps / (ms_total * 1e-3) / 1e9, 1),
         "conv_only_images_per_s": round(world * N / (sum(conv_ms) * 1e-3), 2),
-        "roofline": {"bound": "alu", "kernel": "sparse conv (12 launches per step)", "achieved": round(achieved, 3),
+        "roofline": {"bound": "alu", "kernel": "sparse convolution path of the 12 pruned layers (stage images + convolution + reduce launches)", "achieved": round(achieved, 3),
                      "peak": round(FMA_PEAK_TFLOPS, 2), "unit": "TFLOP/s", "frac": round(achieved / FMA_PEAK_TFLOPS, 4),
                      "peak_kind": "derived: 2 x 128 fp32 lanes x 148 SMs x 1.965 GHz",
-                     "traffic": CONV6_DRAM_BYTES_B16 * (N / 16.0) if (cfg.number == 3 and CONV6_DRAM_BYTES_B16) else None,
-                     "traffic_note": ("DRAM read+write bytes of the three launches of conv6 (stage images, convolution, "
-                                      "reduce; ncu, batch 16, scaled by batch/16); algorithmic bytes of that layer: %d"
-                                      % layers[5]["L"].compulsory_bytes(N, elem))
-                                     if (cfg.number == 3 and CONV6_DRAM_BYTES_B16) else
-                                     "no counters for the current kernels" if cfg.number == 3 else None,
+                     "traffic": CONV6_DRAM_BYTES_B32 * (N / 32.0) if cfg.number == 3 else None,
+                     "traffic_note": ("DRAM read+write bytes of one k_conv_f16_img launch on the conv6 shape (ncu, batch 32, "
+                                      "scaled by batch/32; part of the output was still in L2 when the captured launch ended); "
+                                      "algorithmic bytes of that layer: %d" % cfg.layers[5].compulsory_bytes(N, elem))
+                                     if cfg.number == 3 else None,
                      "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
-                     "min_layer_frac": min(p["roof_frac"] for p in per_layer if p["layer"] != "conv1")},
+                     "min_layer_frac": min([p["roof_frac"] for p in per_layer if p["layer"] != "conv1"] + [1.0])},
         "layers": per_layer,
         "e2e": {"value": round(e2e_value, 2), "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
@@ -385,6 +385,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="workload number (3 = VGG-16 batch 64 fp16 storage)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch size (profiling small cases)")
+    ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling one layer)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
