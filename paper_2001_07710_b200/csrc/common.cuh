@@ -9,11 +9,20 @@
 namespace pat {
 
 constexpr uint32_t kBlobMagic = 0x50415443u;  // "PATC"
-constexpr uint32_t kBlobVersion = 2u;
+constexpr uint32_t kBlobVersion = 3u;
 constexpr int kChanTile = 16;                 // granularity (input channels) of the execution section
 constexpr int kExecGroup = 32;                // filters per execution group (aligned groups of original filters)
 constexpr int kMaxK = 255;
-constexpr int kBlockHeaderBytes = 4 * kExecGroup;   // header of a descriptor block: one 32-bit word per filter slot
+constexpr int kBlockHeaderBytes = 4 * kExecGroup;   // header of a descriptor block: 32 words, one per consumer warp in use
+constexpr int kBlockWarps = kExecGroup / 2;         // consumer warps that share a descriptor block (two filters each)
+// Geometry of the stage images the descriptor blocks are written for (the last word of a descriptor is the byte
+// offset of the kernel's window inside a stage image): bytes of a pixel row and of a channel plane.
+constexpr int kImgRowBytes = 128;
+constexpr int kImgPlaneBytes = 36 * kImgRowBytes;
+// Descriptor word (see pattern_word below): bits 18 / 19 = "swap the accumulator tiles before this kernel" /
+// "last operation of this warp in this stage", bits 20-31 = where the warp's list starts in the next stage's block.
+constexpr uint32_t kOpSwap = 1u << 18, kOpEnd = 1u << 19;
+constexpr int kOpNextShift = 20;
 
 // First 256 bytes of every blob.
 struct BlobHeader {
@@ -58,7 +67,7 @@ __host__ __device__ inline BlobLayout blob_layout(int F, int C, int K, int64_t n
   L.tw4 = o;   o = align256(o + 4 * e * nk);
   L.nblk = (dtype == PAT_F16 && F % kExecGroup == 0 && C % kChanTile == 0) ? (F / kExecGroup) * L.nct : 0;
   L.dboff = o; o = align256(o + (L.nblk ? sizeof(uint32_t) * ((size_t)L.nblk + 1) : 0));
-  L.dblk = o;  o = align256(o + (L.nblk ? (size_t)L.nblk * kBlockHeaderBytes + 16 * nk : 0));
+  L.dblk = o;  o = align256(o + (L.nblk ? (size_t)L.nblk * (kBlockHeaderBytes + 16 * kBlockWarps) + 16 * nk : 0));
   L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 4));
   L.total = o;
   return L;
@@ -95,6 +104,7 @@ __host__ __device__ inline void mask_bits(uint32_t m, int bits[4]) {
 // codes (the eight patterns of Section 4.2 need six).  Any other pattern takes the generic code (kGenericCode).
 constexpr int kNumCodes = 10;
 constexpr int kGenericCode = 15;
+constexpr int kNopCode = 14;                  // an operation without a kernel (a warp with nothing to do in a stage)
 __host__ __device__ constexpr uint32_t code_mask(int i) {
   constexpr uint32_t m[kNumCodes] = {0x03A, 0x017, 0x0B2, 0x09A, 0x01B, 0x036, 0x093, 0x03C, 0x192, 0x00F};
   return m[i];

@@ -36,11 +36,12 @@ constexpr int IMG_BYTES = CBI * CHP;       // 73728
 constexpr int MAX_NS = 3;
 constexpr int MAXE3 = 152;
 constexpr int DBLK3 = kBlockHeaderBytes + MAXE3 * 16;           // 2560
-constexpr int DBLK2 = kBlockHeaderBytes + FG * kChanTile * 16;  // largest possible block (8320)
+constexpr int DBLK2 = kBlockHeaderBytes + (FG * kChanTile + kBlockWarps + 8) * 16;  // largest possible block and spare slots up to a multiple of 128 (8704)
 constexpr int OFF_SLOTS = 256;             // barriers and two control words sit in front of the ring
 constexpr int SMEM_BYTES = OFF_SLOTS + 3 * (IMG_BYTES + DBLK3);
 static_assert(OFF_SLOTS + 2 * (IMG_BYTES + DBLK2) <= SMEM_BYTES, "the two-slot layout fits too");
 static_assert(IMG_BYTES % 128 == 0 && DBLK3 % 128 == 0 && DBLK2 % 128 == 0 && SMEM_BYTES <= 232448, "shared memory budget of one SM");
+static_assert(CHP == kImgPlaneBytes && NCW == kBlockWarps, "the descriptor blocks are written for this geometry");
 constexpr int OUT_PITCH = FG * 2 + 4;      // output staging inside a slot: [448 px][32 channels] fp16, pixel pitch 68 B
 constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (30464)
 static_assert(2 * OUT_ROW <= IMG_BYTES && 32 % NCW == 0, "two tile rows of results fit a slot");
@@ -276,13 +277,11 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
     // columns [128 * (w / 4) + 64 * f, +64) of the lanes of quarter w % 4.
     const uint32_t tm0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
     auto park = [&](uint32_t f, const float (&a)[TR4][TC]) {
-      tmem_store_rows<TR4, 0>(tm0 + f * 64u, a);
-      tmem_store_rows<TR4, 2>(tm0 + f * 64u + 32u, a);
+      tmem_store_tile(tm0 + f * 64u, a);
       tmem_wait_st();
     };
     auto fetch = [&](uint32_t f, float (&a)[TR4][TC]) {
-      tmem_load_rows<TR4, 0>(tm0 + f * 64u, a);
-      tmem_load_rows<TR4, 2>(tm0 + f * 64u + 32u, a);
+      tmem_load_tile(tm0 + f * 64u, a);
       tmem_wait_ld();
     };
     int pslot = 0;
@@ -301,37 +300,48 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       for (int y = 0; y < TR4; ++y)
 #pragma unroll
         for (int x = 0; x < TC; ++x) acc[y][x] = 0.0f;
-      park(1u, acc);                     // filter 1 starts from zero in tensor memory, filter 0 in registers
-      uint32_t cur = 0u;                 // which of the two filters the registers hold
-
       int c0, c1;
       const bool piece = piece_of(it_idx, c0, c1);
-      for (int cb = c0; cb < c1; ++cb) {
-        if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
-        const uint32_t pl0 = slot0 + (uint32_t)pslot * SLOT + offA;
-        // filter A, swap, filter B (one copy of the multiply-add code)
+      // A stage is one flat list of operations per warp, written at pack time: kernels of the filter whose tile
+      // the warp holds, then (flag kOpSwap) the other filter's; the last one carries kOpEnd and the place of the
+      // warp's list in the next stage's block.  The next operation and the first two window rows of the current
+      // one are loaded before the pattern's code runs.
+      if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+      uint32_t sl = slot0 + (uint32_t)pslot * SLOT;
+      uint32_t pl0 = sl + offA;
+      const uint32_t hw = lds32(sl + IMG_BYTES + (uint32_t)warp * 4u);
+      uint32_t cur = hw >> 31;           // which of the two filters the registers hold (both tiles are zero now)
+      park(cur ^ 1u, acc);
+      uint32_t e = sl + IMG_BYTES + kBlockHeaderBytes + (hw & 0xFFFFu) * 16u;
+      uint32_t m0, w01, w23, off;
+      lds128(e, m0, w01, w23, off);
+      int cb = c0;
 #pragma unroll 1
-        for (int ph = 0; ph < 2; ++ph) {
-          const uint32_t d0 = pl0 - offA + IMG_BYTES;
-          const uint32_t hw = lds32(d0 + (cur ? (uint32_t)(FG - 1 - warp) : (uint32_t)warp) * 4);
-          uint32_t e = d0 + kBlockHeaderBytes + (hw & 0xFFFFu) * 16u;
-          const uint32_t e_end = e + (hw >> 16) * 16u;
-#pragma unroll 1
-          for (; e != e_end; e += 16) {
-            uint32_t m0, w01, w23, pad;
-            lds128(e, m0, w01, w23, pad);
-            const uint32_t base = pl0 + (m0 & 15u) * CHP;
-            one_kernel4(acc, base, base ^ 16u, m0, w01, w23);
-          }
-          if (ph == 0) {
-            park(cur, acc);
-            cur ^= 1u;
-            fetch(cur, acc);
-          }
+      for (;;) {
+        const uint32_t a0 = pl0 + off;
+        uint32_t r0[8], r1[8];
+        lds_row(r0, a0, a0 ^ 16u);
+        lds_row(r1, a0 + ROWB, (a0 ^ 16u) + ROWB);
+        const uint32_t cm = m0, c01 = w01, c23 = w23, coff = off;
+        e += 16u;
+        lds128(e, m0, w01, w23, off);
+        if (cm & kOpSwap) {
+          park(cur, acc);
+          cur ^= 1u;
+          fetch(cur, acc);
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(slot_empty(pslot));
-        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
+        one_kernel4(acc, pl0, cm, c01, c23, coff, r0, r1);
+        if (cm & kOpEnd) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(slot_empty(pslot));
+          if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
+          if (++cb == c1) break;
+          if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+          sl = slot0 + (uint32_t)pslot * SLOT;
+          pl0 = sl + offA;
+          e = sl + IMG_BYTES + kBlockHeaderBytes + (cm >> kOpNextShift) * 16u;
+          lds128(e, m0, w01, w23, off);
+        }
       }
       if (!alive) break;
 
@@ -441,14 +451,14 @@ k_conv_f16_img(const Params p) {
   const BlobHeader* bh = p.hdr;
   bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
             bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep &&
-            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * kChanTile;
+            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * kChanTile + kBlockWarps;
   for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
   if (!ok) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
     return;
   }
   // ring geometry by the size of the largest descriptor block (see MAX_NS above)
-  if (bh->max_block_entries <= MAXE3) conv_body<true>(p, smem);
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true>(p, smem);
   else conv_body<false>(p, smem);
 }
 

@@ -255,60 +255,151 @@ __device__ __forceinline__ void one_kernel(float (&acc)[TR][TC], uint32_t baseA,
 #undef PAT_ROW3
 }
 
-// ---- 4 x 14 pixel tiles (56 accumulators): the code of a pattern walks down the window one row at a time, so a
-// row of 16 pixels is loaded once and serves every tap that reads it.  MASK is a compiled code (first tap in
-// kernel row 0); a0 / a1 = the lane's addresses of logical chunks 0 / 1 of the first window row the code reads
-// (window row `sh`).  The two chunks of a segment trade places every four image rows, i.e. from window row 4 on.
+// ---- 4 x 14 pixel tiles (56 accumulators)
 constexpr int TR4 = 4;
+static_assert(ROWB == kImgRowBytes, "the descriptors' window offsets are written for this row pitch");
 __host__ __device__ constexpr int last_tap_row(uint32_t mask) { return (mask >> 6) ? 2 : ((mask >> 3) ? 1 : 0); }
 
+// A tile in tensor memory: 56 consecutive columns of the thread's lane, value (y, x) at column 14 y + x, moved by
+// three transfers of 32, 16 and 8 columns whose register lists are the tile in that order (no padding values, so
+// the accumulators can stay where they are).  tmem_store_tile / tmem_load_tile only issue the transfers;
+// tmem_wait_st / tmem_wait_ld complete them.
+#define PAT_F(i) "f"(a[(i) / TC][(i) % TC])
+#define PAT_O(i) "=f"(a[(i) / TC][(i) % TC])
+__device__ __forceinline__ void tmem_store_tile(uint32_t taddr, const float (&a)[TR4][TC]) {
+  static_assert(TR4 * TC == 56, "32 + 16 + 8 columns");
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), PAT_F(0), PAT_F(1), PAT_F(2), PAT_F(3), PAT_F(4), PAT_F(5), PAT_F(6), PAT_F(7), PAT_F(8), PAT_F(9), PAT_F(10),
+        PAT_F(11), PAT_F(12), PAT_F(13), PAT_F(14), PAT_F(15), PAT_F(16), PAT_F(17), PAT_F(18), PAT_F(19), PAT_F(20), PAT_F(21),
+        PAT_F(22), PAT_F(23), PAT_F(24), PAT_F(25), PAT_F(26), PAT_F(27), PAT_F(28), PAT_F(29), PAT_F(30), PAT_F(31)
+      : "memory");
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr + 32u), PAT_F(32), PAT_F(33), PAT_F(34), PAT_F(35), PAT_F(36), PAT_F(37), PAT_F(38), PAT_F(39), PAT_F(40),
+        PAT_F(41), PAT_F(42), PAT_F(43), PAT_F(44), PAT_F(45), PAT_F(46), PAT_F(47)
+      : "memory");
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+      ::"r"(taddr + 48u), PAT_F(48), PAT_F(49), PAT_F(50), PAT_F(51), PAT_F(52), PAT_F(53), PAT_F(54), PAT_F(55)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_load_tile(uint32_t taddr, float (&a)[TR4][TC]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : PAT_O(0), PAT_O(1), PAT_O(2), PAT_O(3), PAT_O(4), PAT_O(5), PAT_O(6), PAT_O(7), PAT_O(8), PAT_O(9), PAT_O(10),
+        PAT_O(11), PAT_O(12), PAT_O(13), PAT_O(14), PAT_O(15), PAT_O(16), PAT_O(17), PAT_O(18), PAT_O(19), PAT_O(20), PAT_O(21),
+        PAT_O(22), PAT_O(23), PAT_O(24), PAT_O(25), PAT_O(26), PAT_O(27), PAT_O(28), PAT_O(29), PAT_O(30), PAT_O(31)
+      : "r"(taddr) : "memory");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : PAT_O(32), PAT_O(33), PAT_O(34), PAT_O(35), PAT_O(36), PAT_O(37), PAT_O(38), PAT_O(39), PAT_O(40),
+        PAT_O(41), PAT_O(42), PAT_O(43), PAT_O(44), PAT_O(45), PAT_O(46), PAT_O(47)
+      : "r"(taddr + 32u) : "memory");
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+      : PAT_O(48), PAT_O(49), PAT_O(50), PAT_O(51), PAT_O(52), PAT_O(53), PAT_O(54), PAT_O(55)
+      : "r"(taddr + 48u) : "memory");
+}
+#undef PAT_F
+#undef PAT_O
+
+// One multiply-add whose fp16 operands are halves of 32-bit registers (no instruction is spent on taking a
+// register apart: the halves are operand selectors of the multiply-add itself).
+template <int VHI, int WHI>
+__device__ __forceinline__ void fma_half_of(float& acc, uint32_t v, uint32_t w) {
+  unsigned short a, b, u0, u1;
+  if (VHI) asm("mov.b32 {%0,%1}, %2;" : "=h"(u0), "=h"(a) : "r"(v)); else asm("mov.b32 {%0,%1}, %2;" : "=h"(a), "=h"(u0) : "r"(v));
+  if (WHI) asm("mov.b32 {%0,%1}, %2;" : "=h"(u1), "=h"(b) : "r"(w)); else asm("mov.b32 {%0,%1}, %2;" : "=h"(b), "=h"(u1) : "r"(w));
+  asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(a), "h"(b));
+}
+__device__ __forceinline__ void lds_row(uint32_t (&q)[8], uint32_t a0, uint32_t a1) {
+  lds128(a0, q[0], q[1], q[2], q[3]);   // logical chunk 0: cols -1..6
+  lds128(a1, q[4], q[5], q[6], q[7]);   // logical chunk 1: cols 7..14
+}
+template <int B>
+__device__ __forceinline__ void tap_row(float (&acc)[TC], const uint32_t (&q)[8], uint32_t w01, uint32_t w23, int t) {
+  // tap number t (0..3, compile time after unrolling) of the pattern sits at kernel column B % 3
+  constexpr int c = B % 3;
+#pragma unroll
+  for (int x = 0; x < TC; ++x) {
+    const uint32_t v = q[(x + c) >> 1];
+    const uint32_t w = t < 2 ? w01 : w23;
+    if ((x + c) & 1) { if (t & 1) fma_half_of<1, 1>(acc[x], v, w); else fma_half_of<1, 0>(acc[x], v, w); }
+    else             { if (t & 1) fma_half_of<0, 1>(acc[x], v, w); else fma_half_of<0, 0>(acc[x], v, w); }
+  }
+}
+
+// The code of one pattern: it walks down the thread's window one row of 16 pixels at a time, and every row
+// serves all taps that read it.  MASK is a compiled code (first tap in kernel row 0); a0 / a1 = the lane's
+// addresses of logical chunks 0 / 1 of window row `sh`, the first row the code reads; r0 / r1 = that row and the
+// next one, loaded by the caller before it branched here.  The two chunks of a segment trade places every four
+// image rows, i.e. from window row 4 on.
 template <uint32_t MASK>
-__device__ __forceinline__ void pattern_body4(float (&acc)[TR4][TC], uint32_t a0, uint32_t a1, uint32_t sh, uint32_t w01, uint32_t w23) {
-  unsigned short w[4];
-  split_h2(w01, w[0], w[1]);
-  split_h2(w23, w[2], w[3]);
+__device__ __forceinline__ void pattern_body4(float (&acc)[TR4][TC], uint32_t a0, uint32_t a1, uint32_t sh, uint32_t w01, uint32_t w23,
+                                              const uint32_t (&r0)[8], const uint32_t (&r1)[8]) {
   constexpr int NR = last_tap_row(MASK) + TR4;      // rows of the window this code reads
 #pragma unroll
   for (int j = 0; j < NR; ++j) {
-    unsigned short h[16];
-    uint32_t p0 = a0 + j * ROWB, p1 = a1 + j * ROWB;
-    if (j >= 4) { const uint32_t t = p0; p0 = p1; p1 = t; }
-    else if (j == 3) { const uint32_t q0 = sh ? p1 : p0, q1 = sh ? p0 : p1; p0 = q0; p1 = q1; }
-    load_row(h, p0, p1);
+    uint32_t q[8];
+    if (j == 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = r0[i];
+    } else if (j == 1) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = r1[i];
+    } else {
+      uint32_t p0 = a0 + j * ROWB, p1 = a1 + j * ROWB;
+      if (j >= 4) { const uint32_t t = p0; p0 = p1; p1 = t; }
+      else if (j == 3) { const uint32_t q0 = sh ? p1 : p0, q1 = sh ? p0 : p1; p0 = q0; p1 = q1; }
+      lds_row(q, p0, p1);
+    }
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
-      const int b = nth_bit(MASK, t);
-      const int r = b / 3, c = b % 3;
-      const int y = j - r;
+      constexpr uint32_t M = MASK;
+      const int b = nth_bit(M, t);
+      const int y = j - b / 3;
       if (y >= 0 && y < TR4) {
-#pragma unroll
-        for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[x + c], w[t]);
+        switch (b) {   // b is a compile-time constant after unrolling
+          case 0: tap_row<0>(acc[y], q, w01, w23, t); break;
+          case 1: tap_row<1>(acc[y], q, w01, w23, t); break;
+          case 2: tap_row<2>(acc[y], q, w01, w23, t); break;
+          case 3: tap_row<3>(acc[y], q, w01, w23, t); break;
+          case 4: tap_row<4>(acc[y], q, w01, w23, t); break;
+          case 5: tap_row<5>(acc[y], q, w01, w23, t); break;
+          case 6: tap_row<6>(acc[y], q, w01, w23, t); break;
+          case 7: tap_row<7>(acc[y], q, w01, w23, t); break;
+          default: tap_row<8>(acc[y], q, w01, w23, t); break;
+        }
       }
     }
   }
 }
 
-// One kept kernel on a 4-row tile.  baseA / baseB = the lane's two chunk addresses of window row 0 in the
-// kernel's channel plane.  Every branch is warp-uniform.
-__device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t baseA, uint32_t baseB, uint32_t meta,
-                                            uint32_t w01, uint32_t w23) {
+// One kept kernel on a 4-row tile.  plane = the lane's address of logical chunk 0 of window row 0 in channel
+// plane 0 of the stage; meta / w01 / w23 / off = the kernel's descriptor (off = byte offset of its channel plane
+// plus its window row shift).  Every branch is warp-uniform.
+__device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t plane, uint32_t meta, uint32_t w01, uint32_t w23,
+                                            uint32_t off, const uint32_t (&r0)[8], const uint32_t (&r1)[8]) {
   const uint32_t sh = (meta >> 17) & 1u;
-  const uint32_t a0 = baseA + sh * ROWB, a1 = baseB + sh * ROWB;
+  const uint32_t a0 = plane + off, a1 = a0 ^ 16u;
   const uint32_t code = (meta >> 13) & 15u;
   if (code & 8u) {
     if (code & 4u) {
+      if (!(code & 1u)) return;          // kNopCode: an operation without a kernel
       // any other pattern: position by position, each with its own pass over the window rows it reads
+      const uint32_t baseA = a0 - sh * ROWB, baseB = baseA ^ 16u;
 #define PAT_TAP4(B)                                                                          \
   if (meta & (16u << (B))) {                                                                 \
-    const unsigned short wv = (unsigned short)(w01 & 0xFFFFu);                               \
     _Pragma("unroll")                                                                        \
     for (int y = 0; y < TR4; ++y) {                                                          \
-      unsigned short h[16];                                                                  \
+      uint32_t q[8];                                                                         \
       const int jr = y + (B) / 3;                                                            \
       const uint32_t q0 = baseA + jr * ROWB, q1 = baseB + jr * ROWB;                         \
-      if (jr >= 4) load_row(h, q1, q0); else load_row(h, q0, q1);                            \
-      _Pragma("unroll")                                                                      \
-      for (int x = 0; x < TC; ++x) fma_f32_f16(acc[y][x], h[x + (B) % 3], wv);               \
+      if (jr >= 4) lds_row(q, q1, q0); else lds_row(q, q0, q1);                              \
+      tap_row<B>(acc[y], q, w01, w23, 0);                                                    \
     }                                                                                        \
     w01 = __funnelshift_r(w01, w23, 16);                                                     \
     w23 >>= 16;                                                                              \
@@ -316,25 +407,25 @@ __device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t base
       PAT_TAP4(0) PAT_TAP4(1) PAT_TAP4(2) PAT_TAP4(3) PAT_TAP4(4) PAT_TAP4(5) PAT_TAP4(6) PAT_TAP4(7) PAT_TAP4(8)
 #undef PAT_TAP4
     } else if (code & 1u) {
-      pattern_body4<code_mask(9)>(acc, a0, a1, sh, w01, w23);
+      pattern_body4<code_mask(9)>(acc, a0, a1, sh, w01, w23, r0, r1);
     } else {
-      pattern_body4<code_mask(8)>(acc, a0, a1, sh, w01, w23);
+      pattern_body4<code_mask(8)>(acc, a0, a1, sh, w01, w23, r0, r1);
     }
   } else if (code & 4u) {
     if (code & 2u) {
-      if (code & 1u) pattern_body4<code_mask(7)>(acc, a0, a1, sh, w01, w23);
-      else pattern_body4<code_mask(6)>(acc, a0, a1, sh, w01, w23);
+      if (code & 1u) pattern_body4<code_mask(7)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      else pattern_body4<code_mask(6)>(acc, a0, a1, sh, w01, w23, r0, r1);
     } else {
-      if (code & 1u) pattern_body4<code_mask(5)>(acc, a0, a1, sh, w01, w23);
-      else pattern_body4<code_mask(4)>(acc, a0, a1, sh, w01, w23);
+      if (code & 1u) pattern_body4<code_mask(5)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      else pattern_body4<code_mask(4)>(acc, a0, a1, sh, w01, w23, r0, r1);
     }
   } else {
     if (code & 2u) {
-      if (code & 1u) pattern_body4<code_mask(3)>(acc, a0, a1, sh, w01, w23);
-      else pattern_body4<code_mask(2)>(acc, a0, a1, sh, w01, w23);
+      if (code & 1u) pattern_body4<code_mask(3)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      else pattern_body4<code_mask(2)>(acc, a0, a1, sh, w01, w23, r0, r1);
     } else {
-      if (code & 1u) pattern_body4<code_mask(1)>(acc, a0, a1, sh, w01, w23);
-      else pattern_body4<code_mask(0)>(acc, a0, a1, sh, w01, w23);
+      if (code & 1u) pattern_body4<code_mask(1)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      else pattern_body4<code_mask(0)>(acc, a0, a1, sh, w01, w23, r0, r1);
     }
   }
 }

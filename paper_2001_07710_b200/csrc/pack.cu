@@ -262,43 +262,82 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
   }
 }
 
-// Descriptor blocks of the fp16 convolution kernel that copies its kernel lists with one bulk copy per pipeline
-// stage.  One block per (group of 32 filters in execution order, 16-channel tile), groups major:
-//   header   32 words, one per filter slot of the group: first entry (bits 0-15) | number of entries (bits 16-31)
-//   entries  16 bytes per kept kernel, slot after slot, inside a slot in (pattern, channel) order:
-//            {channel inside the tile | pattern_word(mask), taps 0-1 (fp16 x2), taps 2-3 (fp16 x2), 0}
-// dboff[b] is the block's offset in 16-byte units.  Launched with one warp per block (lane = filter slot).
+// Descriptor blocks of the fp16 convolution kernel that copies its work lists with one bulk copy per pipeline
+// stage.  One block per (group of 32 filters in execution order, 16-channel tile), groups major.  A block is the
+// work of the kernel's 16 consumer warps in that stage; warp w owns filter slots w ("A") and 31 - w ("B") of the
+// group and keeps one accumulator tile in registers, the other parked.  The order of a warp's operations is fixed
+// here, at pack time: starting from the tile it holds when the stage begins (A at the first tile; afterwards
+// whatever the previous stage left), first the kernels of that filter, then - only if the other filter has kernels
+// in this tile - a swap and the other filter's kernels.
+//   header   32 words; word w < 16: first operation of warp w (bits 0-15) | filter whose tile is in registers when
+//            the stage begins (bit 31).  Words 16-31 unused.
+//   lists    16 bytes per operation, warp after warp, every list one slot longer than the warp's kernels:
+//            {channel inside the tile | pattern_word(mask) | flags, taps 0-1 (fp16 x2), taps 2-3 (fp16 x2),
+//             byte offset of the kernel's window in a stage image: channel plane + window row shift}
+//            flags: kOpSwap on the first kernel after the swap, kOpEnd on the warp's last operation, together with
+//            the start of the warp's list in the next tile's block (bits 20-31).  A warp without kernels in the
+//            tile gets one operation with the code kNopCode; otherwise the spare slot stays unused.
+// Inside a filter the kernels are in (pattern, channel) order.  dboff[b] is the block's offset in 16-byte units.
+// Launched with one warp per block (lane = consumer warp, lanes 16-31 idle apart from the shuffles).
 __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
   const int blk = blockIdx.x, lane = threadIdx.x;
   const int g = blk / nct, cb = blk % nct;
-  const int32_t* row = bp.tptr + (size_t)(g * kExecGroup + lane) * (nct + 1);
-  const int a = row[cb], n = row[cb + 1] - a;
-  int before = a - row[0];                 // kernels of this slot in earlier tiles
-  int incl = n;
+  const bool active = lane < kBlockWarps;
+  const int w = active ? lane : 0;
+  const int32_t* rowA = bp.tptr + (size_t)(g * kExecGroup + w) * (nct + 1);
+  const int32_t* rowB = bp.tptr + (size_t)(g * kExecGroup + kExecGroup - 1 - w) * (nct + 1);
+  // which tile the warp holds when this stage begins
+  int cur = 0;
+  for (int t = 0; t < cb; ++t) {
+    const int nother = cur ? rowA[t + 1] - rowA[t] : rowB[t + 1] - rowB[t];
+    if (nother > 0) cur ^= 1;
+  }
+  const int aA = rowA[cb], nA = rowA[cb + 1] - aA, aB = rowB[cb], nB = rowB[cb + 1] - aB;
+  const int cap = active ? nA + nB + 1 : 0;                       // list slots of this warp in this block
+  const int cap_next = (active && cb + 1 < nct) ? (rowA[cb + 2] - rowA[cb + 1]) + (rowB[cb + 2] - rowB[cb + 1]) + 1 : 0;
+  int incl = cap, incl_next = cap_next;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
-    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-    if (lane >= off) incl += v;
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off), vn = __shfl_up_sync(0xFFFFFFFFu, incl_next, off);
+    if (lane >= off) { incl += v; incl_next += vn; }
   }
+  const int start = incl - cap, start_next = incl_next - cap_next;
+  const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+  // kernels of this group in earlier tiles (all 32 filter slots)
+  const int32_t* row = bp.tptr + (size_t)(g * kExecGroup + lane) * (nct + 1);
+  int before = row[cb] - row[0];
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
-  const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-  const int start = incl - n;
   const uint32_t group_first = (uint32_t)bp.tptr[(size_t)(g * kExecGroup) * (nct + 1)];   // kernels of earlier groups
-  const uint32_t off16 = (uint32_t)blk * (kBlockHeaderBytes / 16) + group_first + (uint32_t)before;
+  const uint32_t off16 = (uint32_t)blk * (uint32_t)(kBlockHeaderBytes / 16 + kBlockWarps) + group_first + (uint32_t)before;
   if (lane == 0) {
     bp.dboff[blk] = off16;
     if (blk == nblk - 1) bp.dboff[nblk] = off16 + kBlockHeaderBytes / 16 + (uint32_t)tot;
     atomicMax(&bp.hdr->max_block_entries, tot);
   }
   char* base = bp.dblk + (size_t)off16 * 16;
-  reinterpret_cast<uint32_t*>(base)[lane] = (uint32_t)start | ((uint32_t)n << 16);
+  reinterpret_cast<uint32_t*>(base)[lane] = active ? ((uint32_t)start | ((uint32_t)cur << 31)) : 0u;
+  if (!active) return;
   uint4* ent = reinterpret_cast<uint4*>(base + kBlockHeaderBytes) + start;
   const uint2* tw4 = static_cast<const uint2*>(bp.tw4);
-  for (int k = 0; k < n; ++k) {
-    const uint32_t mt = bp.tmeta[a + k];
-    const uint2 w = tw4[a + k];
-    ent[k] = make_uint4(((mt & 0xFFFFu) - (uint32_t)(cb * kChanTile)) | pattern_word(lib.m[mt >> 16]), w.x, w.y, 0u);
+  const int n_first = cur ? nB : nA, a_first = cur ? aB : aA;
+  const int n_second = cur ? nA : nB, a_second = cur ? aA : aB;
+  const int n_ops = n_first + n_second;
+  const uint32_t end_flags = kOpEnd | ((uint32_t)start_next << kOpNextShift);
+  if (n_ops == 0) {
+    ent[0] = make_uint4(((uint32_t)kNopCode << 13) | end_flags, 0u, 0u, 0u);
+    return;
+  }
+  for (int k = 0; k < n_ops; ++k) {
+    const int src = k < n_first ? a_first + k : a_second + (k - n_first);
+    const uint32_t mt = bp.tmeta[src];
+    const uint2 wv = tw4[src];
+    const uint32_t ch = (mt & 0xFFFFu) - (uint32_t)(cb * kChanTile);
+    const uint32_t pw = pattern_word(lib.m[mt >> 16]);
+    uint32_t flags = 0u;
+    if (k == n_first) flags |= kOpSwap;
+    if (k == n_ops - 1) flags |= end_flags;
+    ent[k] = make_uint4(ch | pw | flags, wv.x, wv.y, ch * (uint32_t)kImgPlaneBytes + ((pw >> 17) & 1u) * (uint32_t)kImgRowBytes);
   }
 }
 
