@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
 //                  needed longer for a slot than the consumers for two stages: the ring stood still meanwhile.)
 // In a real stage a consumer warp runs filter A, swaps, runs filter B; the next stage starts with B.  A tile of
 // 56 accumulators is moved to / from tensor memory once per stage and filter.
-template <bool SPARSE>
+template <bool SPARSE, int NCODES, bool GENERIC>
 __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
   constexpr int NS = SPARSE ? 3 : 2;
   constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
@@ -330,7 +330,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           cur ^= 1u;
           fetch(cur, acc);
         }
-        one_kernel4(acc, pl0, cm, c01, c23, coff, r0, r1);
+        one_kernel4<NCODES, GENERIC>(acc, pl0, cm, c01, c23, coff, r0, r1);
         if (cm & kOpEnd) {
           __syncwarp();
           if (lane == 0) mbar_arrive(slot_empty(pslot));
@@ -444,6 +444,9 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
   if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+// NCODES / GENERIC: the pattern codes the kernel carries code for (see one_kernel4); the host picks the smallest
+// set that covers the library.
+template <int NCODES, bool GENERIC>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f16_img(const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -458,8 +461,8 @@ k_conv_f16_img(const Params p) {
     return;
   }
   // ring geometry by the size of the largest descriptor block (see MAX_NS above)
-  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true>(p, smem);
-  else conv_body<false>(p, smem);
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC>(p, smem);
+  else conv_body<false, NCODES, GENERIC>(p, smem);
 }
 
 // ------------------------------------------------------------------------------------------ cut items
@@ -583,18 +586,29 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.K = K; p.n_keep = n_keep;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
+  // the smallest set of compiled pattern codes that covers the library
+  int variant = 0;
+  for (int j = 0; j < K; ++j) {
+    const int code = (int)((pattern_word(masks[j]) >> 13) & 15u);
+    variant = std::max(variant, code == kGenericCode ? 2 : (code >= 6 ? 1 : 0));
+  }
+  using KernelFn = void (*)(const Params);
+  static const KernelFn kernels[3] = {k_conv_f16_img<6, false>, k_conv_f16_img<kNumCodes, false>, k_conv_f16_img<kNumCodes, true>};
+
   static thread_local int sm_count = 0;
   static thread_local bool attr_set = false;
   if (!attr_set) {
     int dev = 0;
     if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
     if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
-    if (int rc = check_cuda(cudaFuncSetAttribute(k_conv_f16_img, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
     if (int rc = check_cuda(cudaFuncSetAttribute(k_stage_images, cudaFuncAttributeMaxDynamicSharedMemorySize, SI_SMEM), "set shared memory size")) return rc;
-    cudaFuncAttributes fa;
-    if (int rc = check_cuda(cudaFuncGetAttributes(&fa, k_conv_f16_img), "query kernel attributes")) return rc;
-    if (fa.numRegs < LAUNCH_REGS)
-      return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
+    for (KernelFn fn : kernels) {
+      if (int rc = check_cuda(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
+      cudaFuncAttributes fa;
+      if (int rc = check_cuda(cudaFuncGetAttributes(&fa, fn), "query kernel attributes")) return rc;
+      if (fa.numRegs < LAUNCH_REGS)
+        return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
+    }
     attr_set = true;
   }
   const int grid = std::min(p.n_items, sm_count);
@@ -608,7 +622,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     }
   }
   k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
-  k_conv_f16_img<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
+  kernels[variant]<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
   count_launches(2);
   if (p.parts > 1) {
     k_reduce_parts<<<(unsigned)(p.n_split * TR4 * 2), RP_THREADS, 0, st>>>(p);

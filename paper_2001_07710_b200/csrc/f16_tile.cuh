@@ -380,17 +380,23 @@ __device__ __forceinline__ void pattern_body4(float (&acc)[TR4][TC], uint32_t a0
 
 // One kept kernel on a 4-row tile.  plane = the lane's address of logical chunk 0 of window row 0 in channel
 // plane 0 of the stage; meta / w01 / w23 / off = the kernel's descriptor (off = byte offset of its channel plane
-// plus its window row shift).  Every branch is warp-uniform.
+// plus its window row shift).  Every branch is warp-uniform.  NCODES = number of compiled pattern codes the
+// library can produce (6 for the eight patterns of Section 4.2, 10 for the twelve), GENERIC = the library holds
+// patterns without compiled code: a kernel compiled for a smaller set carries less code and fewer live registers.
+template <int NCODES, bool GENERIC>
 __device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t plane, uint32_t meta, uint32_t w01, uint32_t w23,
                                             uint32_t off, const uint32_t (&r0)[8], const uint32_t (&r1)[8]) {
+  static_assert(NCODES == 6 || NCODES == kNumCodes, "code sets with compiled dispatch trees");
+  static_assert(kGenericCode == 15 && kNopCode == 14, "codes 14 and 15 share the last branch of the tree");
   const uint32_t sh = (meta >> 17) & 1u;
   const uint32_t a0 = plane + off, a1 = a0 ^ 16u;
   const uint32_t code = (meta >> 13) & 15u;
   if (code & 8u) {
     if (code & 4u) {
-      if (!(code & 1u)) return;          // kNopCode: an operation without a kernel
-      // any other pattern: position by position, each with its own pass over the window rows it reads
-      const uint32_t baseA = a0 - sh * ROWB, baseB = baseA ^ 16u;
+      if (!GENERIC || !(code & 1u)) return;          // kNopCode: an operation without a kernel
+      if constexpr (GENERIC) {
+        // any other pattern: position by position, each with its own pass over the window rows it reads
+        const uint32_t baseA = a0 - sh * ROWB, baseB = baseA ^ 16u;
 #define PAT_TAP4(B)                                                                          \
   if (meta & (16u << (B))) {                                                                 \
     _Pragma("unroll")                                                                        \
@@ -404,17 +410,19 @@ __device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t plan
     w01 = __funnelshift_r(w01, w23, 16);                                                     \
     w23 >>= 16;                                                                              \
   }
-      PAT_TAP4(0) PAT_TAP4(1) PAT_TAP4(2) PAT_TAP4(3) PAT_TAP4(4) PAT_TAP4(5) PAT_TAP4(6) PAT_TAP4(7) PAT_TAP4(8)
+        PAT_TAP4(0) PAT_TAP4(1) PAT_TAP4(2) PAT_TAP4(3) PAT_TAP4(4) PAT_TAP4(5) PAT_TAP4(6) PAT_TAP4(7) PAT_TAP4(8)
 #undef PAT_TAP4
-    } else if (code & 1u) {
-      pattern_body4<code_mask(9)>(acc, a0, a1, sh, w01, w23, r0, r1);
-    } else {
-      pattern_body4<code_mask(8)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      }
+    } else if constexpr (NCODES > 8) {
+      if (code & 1u) pattern_body4<code_mask(9)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      else pattern_body4<code_mask(8)>(acc, a0, a1, sh, w01, w23, r0, r1);
     }
   } else if (code & 4u) {
-    if (code & 2u) {
-      if (code & 1u) pattern_body4<code_mask(7)>(acc, a0, a1, sh, w01, w23, r0, r1);
-      else pattern_body4<code_mask(6)>(acc, a0, a1, sh, w01, w23, r0, r1);
+    if (NCODES > 6 && (code & 2u)) {
+      if constexpr (NCODES > 6) {
+        if (code & 1u) pattern_body4<code_mask(7)>(acc, a0, a1, sh, w01, w23, r0, r1);
+        else pattern_body4<code_mask(6)>(acc, a0, a1, sh, w01, w23, r0, r1);
+      }
     } else {
       if (code & 1u) pattern_body4<code_mask(5)>(acc, a0, a1, sh, w01, w23, r0, r1);
       else pattern_body4<code_mask(4)>(acc, a0, a1, sh, w01, w23, r0, r1);
