@@ -19,10 +19,11 @@ constexpr int kBlockWarps = kExecGroup / 2;         // consumer warps that share
 // offset of the kernel's window inside a stage image): bytes of a pixel row and of a channel plane.
 constexpr int kImgRowBytes = 128;
 constexpr int kImgPlaneBytes = 36 * kImgRowBytes;
-// Descriptor word (see pattern_word below): bits 18 / 19 = "swap the accumulator tiles before this kernel" /
-// "last operation of this warp in this stage", bits 20-31 = where the warp's list starts in the next stage's block.
-constexpr uint32_t kOpSwap = 1u << 18, kOpEnd = 1u << 19;
-constexpr int kOpNextShift = 20;
+// Descriptor word (see pattern_word below): bits 18 / 19 / 20 = "swap the accumulator tiles before this kernel" /
+// "last operation of this warp in this stage" / "no kernel: the warp has nothing to do in this stage",
+// bits 21-31 = where the warp's list starts in the next stage's block.
+constexpr uint32_t kOpSwap = 1u << 18, kOpEnd = 1u << 19, kOpNop = 1u << 20;
+constexpr int kOpNextShift = 21;
 
 // First 256 bytes of every blob.
 struct BlobHeader {
@@ -104,7 +105,6 @@ __host__ __device__ inline void mask_bits(uint32_t m, int bits[4]) {
 // codes (the eight patterns of Section 4.2 need six).  Any other pattern takes the generic code (kGenericCode).
 constexpr int kNumCodes = 10;
 constexpr int kGenericCode = 15;
-constexpr int kNopCode = 14;                  // an operation without a kernel (a warp with nothing to do in a stage)
 __host__ __device__ constexpr uint32_t code_mask(int i) {
   constexpr uint32_t m[kNumCodes] = {0x03A, 0x017, 0x0B2, 0x09A, 0x01B, 0x036, 0x093, 0x03C, 0x192, 0x00F};
   return m[i];

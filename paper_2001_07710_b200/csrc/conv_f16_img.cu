@@ -325,12 +325,14 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         const uint32_t cm = m0, c01 = w01, c23 = w23, coff = off;
         e += 16u;
         lds128(e, m0, w01, w23, off);
-        if (cm & kOpSwap) {
+        if (cm & (kOpSwap | kOpNop)) {   // one test for the two rare cases
+          if (cm & kOpNop) goto stage_end;
           park(cur, acc);
           cur ^= 1u;
           fetch(cur, acc);
         }
         one_kernel4<NCODES, GENERIC>(acc, pl0, cm, c01, c23, coff, r0, r1);
+      stage_end:
         if (cm & kOpEnd) {
           __syncwarp();
           if (lane == 0) mbar_arrive(slot_empty(pslot));

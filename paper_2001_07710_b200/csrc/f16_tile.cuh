@@ -387,13 +387,12 @@ template <int NCODES, bool GENERIC>
 __device__ __forceinline__ void one_kernel4(float (&acc)[TR4][TC], uint32_t plane, uint32_t meta, uint32_t w01, uint32_t w23,
                                             uint32_t off, const uint32_t (&r0)[8], const uint32_t (&r1)[8]) {
   static_assert(NCODES == 6 || NCODES == kNumCodes, "code sets with compiled dispatch trees");
-  static_assert(kGenericCode == 15 && kNopCode == 14, "codes 14 and 15 share the last branch of the tree");
+  static_assert(kGenericCode == 15, "the generic code is the last leaf of the tree");
   const uint32_t sh = (meta >> 17) & 1u;
   const uint32_t a0 = plane + off, a1 = a0 ^ 16u;
   const uint32_t code = (meta >> 13) & 15u;
-  if (code & 8u) {
+  if ((NCODES > 8 || GENERIC) && (code & 8u)) {
     if (code & 4u) {
-      if (!GENERIC || !(code & 1u)) return;          // kNopCode: an operation without a kernel
       if constexpr (GENERIC) {
         // any other pattern: position by position, each with its own pass over the window rows it reads
         const uint32_t baseA = a0 - sh * ROWB, baseB = baseA ^ 16u;

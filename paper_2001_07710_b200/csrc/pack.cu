@@ -275,8 +275,8 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
 //            {channel inside the tile | pattern_word(mask) | flags, taps 0-1 (fp16 x2), taps 2-3 (fp16 x2),
 //             byte offset of the kernel's window in a stage image: channel plane + window row shift}
 //            flags: kOpSwap on the first kernel after the swap, kOpEnd on the warp's last operation, together with
-//            the start of the warp's list in the next tile's block (bits 20-31).  A warp without kernels in the
-//            tile gets one operation with the code kNopCode; otherwise the spare slot stays unused.
+//            the start of the warp's list in the next tile's block (bits 21-31).  A warp without kernels in the
+//            tile gets one operation with the flag kOpNop; otherwise the spare slot stays unused.
 // Inside a filter the kernels are in (pattern, channel) order.  dboff[b] is the block's offset in 16-byte units.
 // Launched with one warp per block (lane = consumer warp, lanes 16-31 idle apart from the shuffles).
 __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable
   const int n_ops = n_first + n_second;
   const uint32_t end_flags = kOpEnd | ((uint32_t)start_next << kOpNextShift);
   if (n_ops == 0) {
-    ent[0] = make_uint4(((uint32_t)kNopCode << 13) | end_flags, 0u, 0u, 0u);
+    ent[0] = make_uint4(kOpNop | end_flags, 0u, 0u, 0u);
     return;
   }
   for (int k = 0; k < n_ops; ++k) {
