@@ -346,6 +346,11 @@ int conv_generic(const void* blob, int F, int C, const uint16_t* masks, int K, i
 
 }  // namespace pat
 
+namespace pat {
+bool conv_dense_c3_mma_supported(int F, int C, int dtype, int stride);
+int conv_dense_c3_mma(const float* w, const void* x, void* y, int N, int H, int W, cudaStream_t st);
+}
+
 using namespace pat;
 
 extern "C" int pat_conv3x3_dense(const float* w, int F, int C, int dtype, const void* x, void* y,
@@ -362,6 +367,7 @@ extern "C" int pat_conv3x3_dense(const float* w, int F, int C, int dtype, const 
   a.tiles_x = (a.Wo + TW - 1) / TW; a.tiles_y = (a.Ho + TH - 1) / TH;
   if ((size_t)N * a.tiles_x * a.tiles_y > 0x7FFFFFFFull) return set_error(PAT_ERR_SHAPE, "pat_conv3x3_dense: too many tiles");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (conv_dense_c3_mma_supported(F, C, dtype, stride)) return conv_dense_c3_mma(w, x, y, N, H, W, st);
   if (C == 3 && stride == 1 && F % 8 == 0 && (size_t)F * 27 * 4 <= 48 * 1024) {
     const long long npix = (long long)N * H * W;
     const unsigned blocks = (unsigned)((npix + 255) / 256);
