@@ -7,7 +7,8 @@
 // Exactness: squares of fp32 values are exact in fp64 and are added in ascending bit order, so the energies
 // are the same bits on any IEEE machine.  The n_keep-th largest energy is found with a 4-pass, 16-bit radix
 // select over the (monotone) bit pattern of the non-negative doubles; ties at the threshold are resolved by
-// index with a block scan.
+// index with a block scan.  Six launches per layer: the step after each histogram (and after the tie counts)
+// that needs all blocks' results is done by the block that finishes last.
 #include "common.cuh"
 
 namespace pat {
@@ -24,7 +25,8 @@ struct SelectState {
 // workspace layout
 constexpr int kCoarse = 256;                 // coarse histogram: the upper 8 bits of a 16-bit digit
 constexpr int kPasses = 4;                   // 64-bit keys, 16 bits per pass
-constexpr size_t kHistWords = (size_t)kPasses * (kBins + kCoarse);   // one fine + one coarse histogram per pass
+constexpr size_t kHistWords = (size_t)kPasses * (kBins + kCoarse) + 4;   // one fine + one coarse histogram per pass, then the block tickets
+constexpr size_t kTicketWord = (size_t)kPasses * (kBins + kCoarse);     // hist[kTicketWord]: blocks of the running kernel that are done
 
 struct ProjWs {
   unsigned long long* key;     // [FC] energy bit patterns
@@ -54,55 +56,32 @@ inline ProjWs carve(void* base, int64_t FC) {
   return w;
 }
 
-// One thread per kernel: energies of all masks, argmax (lowest id on ties).
-__global__ void k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
-                                 unsigned long long* __restrict__ key, unsigned char* __restrict__ pid,
-                                 SelectState* st, long long n_keep) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
-  if (i >= FC) return;
-  double sq[9];
-#pragma unroll
-  for (int b = 0; b < 9; ++b) {
-    const double v = (double)w[i * 9 + b];
-    sq[b] = v * v;
-  }
-  double best_e = -1.0;
-  int best = 0;
-  for (int j = 0; j < lib.K; ++j) {
-    const unsigned m = lib.m[j];
-    double e = 0.0;
-#pragma unroll
-    for (int b = 0; b < 9; ++b)
-      if (m & (1u << b)) e += sq[b];
-    if (e > best_e) { best_e = e; best = j; }
-  }
-  key[i] = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
-  pid[i] = (unsigned char)best;
+// The selection kernels end with a step that needs the work of all their blocks (choosing the digit from the
+// complete histogram, scanning the per-block tie counts).  Instead of a launch of its own that step is done by
+// whichever block finishes last: every block publishes its results, takes a ticket, and the block that draws the
+// last ticket (which also puts the counter back to zero for the next kernel) goes on.  Returns true in every thread
+// of that block; its reads of the other blocks' results must bypass L1 (__ldcg).
+__device__ inline bool last_block_done(unsigned int* ticket) {
+  __shared__ bool s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1;
+  __syncthreads();
+  if (s_last) __threadfence();
+  return s_last;
 }
 
-// Histogram of the current 16-bit digit over the keys that match the decided prefix (fine: all 16 bits,
-// coarse: its upper 8 bits).  Identical digits inside a warp are merged into one atomic.
-__global__ void k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
-                           const SelectState* __restrict__ st, unsigned int* __restrict__ hist) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int shift = 48 - 16 * pass;
-  bool in = i < FC;
-  unsigned d = 0;
-  if (in) {
-    const unsigned long long k = key[i];
-    in = (pass == 0) || ((k >> (shift + 16)) == st->prefix);
-    d = (unsigned)((k >> shift) & 0xFFFFull);
-  }
-  unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
-  unsigned int* coarse = fine + kBins;
+// Histogram of one 16-bit digit (fine: all 16 bits, coarse: its upper 8 bits).  Identical digits inside a warp are
+// merged into one atomic.  Called by all threads of a warp; `in` = this thread takes part.
+__device__ inline void hist_add(unsigned int* fine, unsigned int* coarse, bool in, unsigned d) {
   const unsigned active = __ballot_sync(0xFFFFFFFFu, in);
-  if (!in) return;
-  const unsigned same = __match_any_sync(active, d);
-  const int lane = threadIdx.x & 31;
-  if ((int)(__ffs(same) - 1) == lane) atomicAdd(&fine[d], (unsigned)__popc(same));
-  const unsigned same_c = __match_any_sync(active, d >> 8);
-  if ((int)(__ffs(same_c) - 1) == lane) atomicAdd(&coarse[d >> 8], (unsigned)__popc(same_c));
+  if (in) {
+    const int lane = threadIdx.x & 31;
+    const unsigned same = __match_any_sync(active, d);
+    if ((int)(__ffs(same) - 1) == lane) atomicAdd(&fine[d], (unsigned)__popc(same));
+    const unsigned same_c = __match_any_sync(active, d >> 8);
+    if ((int)(__ffs(same_c) - 1) == lane) atomicAdd(&coarse[d >> 8], (unsigned)__popc(same_c));
+  }
 }
 
 // Inclusive scan over the 256 threads of a block, thread 0 first.
@@ -123,17 +102,18 @@ __device__ inline unsigned long long block_scan_256(unsigned long long v, unsign
 
 // One block of 256 threads: find the digit d with  count(digit > d) < remaining <= count(digit >= d), first in
 // the coarse histogram, then among the 256 fine bins of the coarse bin found.  Thread 0 owns the highest bin.
-__global__ void __launch_bounds__(256) k_sel_pick(SelectState* st, const unsigned int* __restrict__ hist, int pass) {
+__device__ inline void pick_digit(SelectState* st, const unsigned int* hist, int pass) {
   __shared__ unsigned long long warp_tot[8];
   __shared__ int s_coarse;
   __shared__ unsigned long long s_above;
   const unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
   const unsigned int* coarse = fine + kBins;
   const int t = threadIdx.x;
-  const unsigned long long rem = (unsigned long long)st->remaining;
+  const unsigned long long rem = (unsigned long long)__ldcg(&st->remaining);
+  const unsigned long long prefix = __ldcg(&st->prefix);
   {
     const int bin = kCoarse - 1 - t;
-    const unsigned long long c = coarse[bin];
+    const unsigned long long c = __ldcg(coarse + bin);
     const unsigned long long incl = block_scan_256(c, warp_tot);
     if (rem > incl - c && rem <= incl) { s_coarse = bin; s_above = incl - c; }
   }
@@ -142,44 +122,96 @@ __global__ void __launch_bounds__(256) k_sel_pick(SelectState* st, const unsigne
   const unsigned long long above = s_above;
   {
     const int bin = cb * 256 + (255 - t);
-    const unsigned long long c = fine[bin];
+    const unsigned long long c = __ldcg(fine + bin);
     const unsigned long long incl = above + block_scan_256(c, warp_tot);
     if (rem > incl - c && rem <= incl) {
-      st->prefix = (st->prefix << 16) | (unsigned long long)bin;
+      st->prefix = (prefix << 16) | (unsigned long long)bin;
       st->remaining = (long long)(rem - (incl - c));
     }
   }
 }
 
-// Ties at the threshold: count per block of 1024 consecutive kernels.
+// One thread per kernel: energies of all masks, argmax (lowest id on ties); histogram of the first digit of the
+// energies' bit patterns; the last block picks that digit.  do_select = false (everything or nothing is kept):
+// pattern ids only.
+__global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
+                                                        unsigned long long* __restrict__ key, unsigned char* __restrict__ pid,
+                                                        SelectState* st, long long n_keep, unsigned int* hist, bool do_select) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
+  const bool in = i < FC;
+  unsigned long long k = 0ull;
+  if (in) {
+    double sq[9];
+#pragma unroll
+    for (int b = 0; b < 9; ++b) {
+      const double v = (double)w[i * 9 + b];
+      sq[b] = v * v;
+    }
+    double best_e = -1.0;
+    int best = 0;
+    for (int j = 0; j < lib.K; ++j) {
+      const unsigned m = lib.m[j];
+      double e = 0.0;
+#pragma unroll
+      for (int b = 0; b < 9; ++b)
+        if (m & (1u << b)) e += sq[b];
+      if (e > best_e) { best_e = e; best = j; }
+    }
+    k = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
+    key[i] = k;
+    pid[i] = (unsigned char)best;
+  }
+  if (!do_select) return;
+  hist_add(hist, hist + kBins, in, (unsigned)(k >> 48));
+  if (last_block_done(hist + kTicketWord)) pick_digit(st, hist, 0);
+}
+
+// Histogram of the current 16-bit digit over the keys that match the decided prefix; the last block picks the digit.
+__global__ void __launch_bounds__(256) k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
+                                                  SelectState* st, unsigned int* hist) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int shift = 48 - 16 * pass;
+  bool in = i < FC;
+  unsigned d = 0;
+  if (in) {
+    const unsigned long long k = key[i];
+    in = (k >> (shift + 16)) == st->prefix;
+    d = (unsigned)((k >> shift) & 0xFFFFull);
+  }
+  unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
+  hist_add(fine, fine + kBins, in, d);
+  if (last_block_done(hist + kTicketWord)) pick_digit(st, hist, pass);
+}
+
+// Ties at the threshold: count per block of 1024 consecutive kernels; the last block turns the counts into
+// exclusive offsets (sequential over chunks of 1024 blocks).
 __global__ void __launch_bounds__(kSelBlock) k_tie_count(const unsigned long long* __restrict__ key, int64_t FC,
-                                                         const SelectState* __restrict__ st, unsigned int* __restrict__ blk) {
+                                                         const SelectState* __restrict__ st, unsigned int* blk, int nblk,
+                                                         unsigned int* ticket) {
+  __shared__ unsigned int part[kSelBlock];
+  __shared__ unsigned int carry;
   const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
   const int tie = (i < FC && key[i] == st->prefix) ? 1 : 0;
   const int n = __syncthreads_count(tie);
   if (threadIdx.x == 0) blk[blockIdx.x] = (unsigned)n;
-}
-
-// One block: exclusive scan of the per-block tie counts (sequential over chunks of 1024 blocks).
-__global__ void __launch_bounds__(1024) k_tie_scan(unsigned int* blk, int nblk) {
-  __shared__ unsigned int part[1024];
-  __shared__ unsigned int carry;
+  if (!last_block_done(ticket)) return;
   if (threadIdx.x == 0) carry = 0u;
   __syncthreads();
-  for (int base = 0; base < nblk; base += 1024) {
-    const int i = base + threadIdx.x;
-    const unsigned int v = (i < nblk) ? blk[i] : 0u;
+  for (int base = 0; base < nblk; base += kSelBlock) {
+    const int q = base + threadIdx.x;
+    const unsigned int v = (q < nblk) ? __ldcg(blk + q) : 0u;
     part[threadIdx.x] = v;
     __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
+    for (int off = 1; off < kSelBlock; off <<= 1) {
       unsigned int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0u;
       __syncthreads();
       part[threadIdx.x] += a;
       __syncthreads();
     }
-    if (i < nblk) blk[i] = carry + part[threadIdx.x] - v;
+    if (q < nblk) blk[q] = carry + part[threadIdx.x] - v;
     __syncthreads();
-    if (threadIdx.x == 1023) carry += part[1023];
+    if (threadIdx.x == kSelBlock - 1) carry += part[kSelBlock - 1];
     __syncthreads();
   }
 }
@@ -250,21 +282,19 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   lib.K = K;
   const int nb256 = (int)((FC + 255) / 256);
   const int nblk = (int)((FC + kSelBlock - 1) / kSelBlock);
-  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep);
   int mode = -1;
   if (n_keep == FC) mode = 1;
   else if (n_keep == 0) mode = 0;
   if (mode < 0) {
     if (int rc = check_cuda(cudaMemsetAsync(ws.hist, 0, 4 * kHistWords, st), "pat_project memset")) return rc;
-    for (int pass = 0; pass < kPasses; ++pass) {
-      k_sel_hist<<<nb256, 256, 0, st>>>(ws.key, FC, pass, ws.st, ws.hist);
-      k_sel_pick<<<1, 256, 0, st>>>(ws.st, ws.hist, pass);
-    }
-    k_tie_count<<<nblk, kSelBlock, 0, st>>>(ws.key, FC, ws.st, ws.blk);
-    k_tie_scan<<<1, 1024, 0, st>>>(ws.blk, nblk);
+  }
+  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0);
+  if (mode < 0) {
+    for (int pass = 1; pass < kPasses; ++pass) k_sel_hist<<<nb256, 256, 0, st>>>(ws.key, FC, pass, ws.st, ws.hist);
+    k_tie_count<<<nblk, kSelBlock, 0, st>>>(ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord);
   }
   k_finalize<<<nblk, kSelBlock, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
-  count_launches(mode < 0 ? 12 : 2);
+  count_launches(mode < 0 ? 6 : 2);
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
 
