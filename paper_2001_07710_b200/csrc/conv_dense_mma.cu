@@ -45,7 +45,7 @@ __device__ __forceinline__ int channel_of(int jt, int col) {
   return (jt < 4 ? 0 : 32) + 8 * (col >> 1) + 2 * (jt & 3) + (col & 1);
 }
 
-__global__ void __launch_bounds__(NTHREADS) k_conv_dense_c3_mma(const Args a) {
+__global__ void __launch_bounds__(NTHREADS, 4) k_conv_dense_c3_mma(const Args a) {
   __shared__ __align__(16) __half tile[(TH + 2) * ROWP];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
