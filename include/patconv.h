@@ -169,6 +169,8 @@ int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K,
 /* Dense 3x3 convolution for layers that are not pruned (the first layer of VGG-16, C = 3).
  *   w   dev, [F][C][3][3] fp32 (converted to the activation type on the fly)
  *   x   dev NHWC [N][H][W][C]; y dev NHWC [N][Ho][Wo][F]; dtype of x and y = `dtype`
+ * The case C = 3, F = 64, PAT_F16, stride 1 runs on the tensor cores (fp16 products, fp32 sums, like every
+ * other path); all other cases run FMA kernels.
  * Restrictions: C <= 16, F a multiple of 8, F <= 512. */
 int pat_conv3x3_dense(const float *w, int F, int C, int dtype, const void *x, void *y,
                       int N, int H, int W, int stride, void *stream);
