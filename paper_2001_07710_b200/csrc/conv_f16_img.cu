@@ -45,6 +45,7 @@ static_assert(CHP == kImgPlaneBytes && NCW == kBlockWarps, "the descriptor block
 constexpr int OUT_PITCH = FG * 2 + 4;      // output staging inside a slot: [448 px][32 channels] fp16, pixel pitch 68 B
 constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (30464)
 static_assert(2 * OUT_ROW <= IMG_BYTES && 32 % NCW == 0, "two tile rows of results fit a slot");
+static_assert(OUT_PITCH - FG * 2 >= 4, "the last pixel's padding takes the one-word shift of tiles 16-31");
 constexpr int CONSUMER_REGS = 112, OTHER_REGS = 32;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 512;        // 4 consumer warps per lane quarter x 2 filters x 64 columns
@@ -378,7 +379,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       if (!mbar_wait<0>(slot_full(s1), par1, abort_flag)) { alive = false; break; }
       const uint32_t ob0 = slot0 + (uint32_t)s0 * SLOT, ob1 = slot0 + (uint32_t)s1 * SLOT;
       {
-        const uint32_t ol = (uint32_t)(lane * TC) * OUT_PITCH;
+        // tiles 16-31 sit one word further on: lanes l and l + 16 would otherwise store to the same banks
+        const uint32_t ol = (uint32_t)(lane * TC) * OUT_PITCH + (uint32_t)(lane >> 4) * 4u;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           const uint32_t cp = ol + (cur ? cposB : cposA);
@@ -414,7 +416,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
           const int col0 = (it.cg * p.TXe + tx) * TC;
           __half* dst = p.y + (((size_t)n_img * p.H + TR4 * ty) * p.W + col0 + (lane >> 2)) * p.F + g_out * FG + (lane & 3) * 8;
-          const uint32_t src = sl + (uint32_t)(t * TC) * OUT_PITCH;
+          const uint32_t src = sl + (uint32_t)(t * TC) * OUT_PITCH + (uint32_t)(t >> 4) * 4u;
           uint4 v[TR4][2];
 #pragma unroll
           for (int y = 0; y < TR4; ++y)
