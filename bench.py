@@ -213,15 +213,17 @@ def run_ours(args):
                 step()
         run_step = graph.replay
     launches_per_step = pc.pat_launch_count() - launches0
+    # clocks are sampled from here on (two more untimed steps, then the timed region): nvidia-smi needs some tens of
+    # milliseconds before its first sample, more than a short timed region lasts
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(2):
         run_step()
     barrier()
 
     # ---- timed region: device-resident inputs, K replays of the step
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
     e0.record(stream)
     for k in range(args.steps):
         run_step()
@@ -406,7 +408,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="workload number (3 = VGG-16 batch 64 fp16 storage)")
