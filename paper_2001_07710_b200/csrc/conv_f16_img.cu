@@ -112,6 +112,9 @@ constexpr int SI_PITCH = CHP + 8;          // the two channel octets a warp writ
 constexpr int SI_SMEM = CBI * SI_PITCH;
 __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
   extern __shared__ __align__(16) unsigned char img[];
+  // the convolution kernel is launched as a programmatic dependent: its blocks may take over SMs as this grid's
+  // last blocks finish, and wait (griddepcontrol.wait) for the whole grid before they read a stage image
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int cb16 = (int)(blockIdx.x % (unsigned)p.nct);
   const int reg = (int)(blockIdx.x / (unsigned)p.nct);
   const Region r = decode_region(p, reg);
@@ -464,6 +467,8 @@ k_conv_f16_img(const Params p) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
     return;
   }
+  // everything below reads the stage images or writes the output: the stage-image grid must be complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // ring geometry by the size of the largest descriptor block (see MAX_NS above)
   if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC>(p, smem);
   else conv_body<false, NCODES, GENERIC>(p, smem);
@@ -479,6 +484,7 @@ constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
 constexpr int RP_THREADS = 1024, MAX_PARTS = 8, RP_XH = TC / 2;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   __shared__ __align__(16) unsigned char stage[OUT_ROW];
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // launched as a programmatic dependent of the convolution kernel
   // block = (cut item, row of the thread tiles, left or right half of the tile columns)
   const int xh = (int)blockIdx.x & 1, y = ((int)blockIdx.x >> 1) % TR4, li = (int)blockIdx.x / (2 * TR4);
   const int item = p.n_whole + li;
@@ -626,10 +632,19 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     }
   }
   k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
-  kernels[variant]<<<grid, NTHREADS, SMEM_BYTES, st>>>(p);
+  // the two kernels that follow are programmatic dependents of their predecessor: the launch itself overlaps the
+  // predecessor's tail, the kernels wait for its completion before they touch its results
+  cudaLaunchAttribute pdl;
+  pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = st; cfg.attrs = &pdl; cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM_BYTES;
+  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant], p), "pat_conv3x3 launch")) return rc;
   count_launches(2);
   if (p.parts > 1) {
-    k_reduce_parts<<<(unsigned)(p.n_split * TR4 * 2), RP_THREADS, 0, st>>>(p);
+    cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * 2)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
+    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, k_reduce_parts, p), "pat_conv3x3 launch")) return rc;
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
