@@ -86,6 +86,23 @@ int* status_word();
 // Host-side count of kernel launches (see pat_launch_count).
 void count_launches(int n);
 
+// Launch of a kernel that follows another kernel of this library in the same stream and begins with pdl_wait():
+// as a programmatic dependent its launch overlaps the predecessor's tail (the small projection and packing kernels
+// are launch-latency bound), and pdl_wait() holds it until the predecessor has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cfg.attrs = &attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 int set_error(int code, const char* fmt, ...);
 int check_library(const uint16_t* masks, int K);
 int check_cuda(cudaError_t e, const char* what);

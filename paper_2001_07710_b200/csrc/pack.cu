@@ -52,6 +52,7 @@ __host__ __device__ inline BlobPtrs blob_ptrs(void* blob, const BlobLayout& L, i
 
 // One block per original filter: per-pattern counts and kept count.
 __global__ void __launch_bounds__(256) k_pack_count(const uint8_t* __restrict__ pid, int C, int K, BlobPtrs bp, int* status) {
+  pdl_wait();
   extern __shared__ int sh[];   // K counters
   const int f = blockIdx.x;
   for (int j = threadIdx.x; j < K; j += blockDim.x) sh[j] = 0;
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(256) k_pack_count(const uint8_t* __restrict__ 
 // (kept count descending, per-pattern counts lexicographically descending, original index ascending);
 // the threads of the block share the comparisons.
 __global__ void __launch_bounds__(128) k_pack_rank(int F, int K, BlobPtrs bp) {
+  pdl_wait();
   __shared__ int s_rank, s_xrank;
   const int f = blockIdx.x;
   if (threadIdx.x == 0) { s_rank = 0; s_xrank = 0; }
@@ -112,6 +114,7 @@ __global__ void __launch_bounds__(128) k_pack_rank(int F, int K, BlobPtrs bp) {
 // One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
 __global__ void __launch_bounds__(1024) k_pack_ptrs(int F, int C, int K, long long n_keep, int dtype, MaskTable lib,
                                                     unsigned long long total_bytes, BlobPtrs bp, int* status) {
+  pdl_wait();
   __shared__ int part[1024];
   __shared__ int carry;
   if (threadIdx.x == 0) carry = 0;
@@ -187,6 +190,7 @@ template <> __device__ inline __half cvt_weight<__half>(float v) { return __floa
 template <typename T, bool TABLE>
 __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ wm, const uint8_t* __restrict__ pid,
                                                       int C, int K, int nct, MaskTable lib, BlobPtrs bp) {
+  pdl_wait();
   extern __shared__ __align__(16) uint8_t sm_raw[];
   int* tile_pat = reinterpret_cast<int*>(sm_raw);                          // [nct][K] (TABLE only)
   int* tile_start = tile_pat + (TABLE ? nct * K : 0);                      // [nct + 1] kept kernels before tile t
@@ -280,6 +284,7 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
 // Inside a filter the kernels are in (pattern, channel) order.  dboff[b] is the block's offset in 16-byte units.
 // Launched with one warp per block (lane = consumer warp, lanes 16-31 idle apart from the shuffles).
 __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
+  pdl_wait();
   const int blk = blockIdx.x, lane = threadIdx.x;
   const int g = blk / nct, cb = blk % nct;
   const bool active = lane < kBlockWarps;
@@ -404,25 +409,25 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const MaskTable lib = make_table(masks, K);
   const BlobPtrs bp = blob_ptrs(blob, L, F, K);
-  k_pack_count<<<F, 256, K * sizeof(int), st>>>(pattern_id, C, K, bp, status);
-  k_pack_rank<<<F, 128, 0, st>>>(F, K, bp);
-  k_pack_ptrs<<<1, 1024, 0, st>>>(F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
+  launch_dependent(k_pack_count, dim3(F), dim3(256), K * sizeof(int), st, pattern_id, C, K, bp, status);
+  launch_dependent(k_pack_rank, dim3(F), dim3(128), 0, st, F, K, bp);
+  launch_dependent(k_pack_ptrs, dim3(1), dim3(1024), 0, st, F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
   {
     const size_t table = sizeof(int) * (size_t)L.nct * K;
     const bool use_table = table <= 24 * 1024;
     const size_t smem = (use_table ? table : 0) + sizeof(int) * ((size_t)L.nct + 1) + (size_t)C;
     if (smem > 48 * 1024) return set_error(PAT_ERR_SHAPE, "pat_pack: C=%d too large for the packing kernel", C);
     if (dtype == PAT_F16) {
-      if (use_table) k_pack_scatter<__half, true><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
-      else k_pack_scatter<__half, false><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+      if (use_table) launch_dependent(k_pack_scatter<__half, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
+      else launch_dependent(k_pack_scatter<__half, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
     } else {
-      if (use_table) k_pack_scatter<float, true><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
-      else k_pack_scatter<float, false><<<F, 256, smem, st>>>(w_masked, pattern_id, C, K, L.nct, lib, bp);
+      if (use_table) launch_dependent(k_pack_scatter<float, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
+      else launch_dependent(k_pack_scatter<float, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
     }
   }
   count_launches(4);
   if (L.nblk > 0) {
-    k_pack_blocks<<<L.nblk, 32, 0, st>>>(L.nct, L.nblk, lib, bp);
+    launch_dependent(k_pack_blocks, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_pack launch");

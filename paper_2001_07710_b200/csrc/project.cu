@@ -137,6 +137,7 @@ __device__ inline void pick_digit(SelectState* st, const unsigned int* hist, int
 __global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
                                                         unsigned long long* __restrict__ key, unsigned char* __restrict__ pid,
                                                         SelectState* st, long long n_keep, unsigned int* hist, bool do_select) {
+  pdl_wait();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
   const bool in = i < FC;
@@ -170,6 +171,7 @@ __global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict_
 // Histogram of the current 16-bit digit over the keys that match the decided prefix; the last block picks the digit.
 __global__ void __launch_bounds__(256) k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
                                                   SelectState* st, unsigned int* hist) {
+  pdl_wait();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int shift = 48 - 16 * pass;
   bool in = i < FC;
@@ -189,6 +191,7 @@ __global__ void __launch_bounds__(256) k_sel_hist(const unsigned long long* __re
 __global__ void __launch_bounds__(kSelBlock) k_tie_count(const unsigned long long* __restrict__ key, int64_t FC,
                                                          const SelectState* __restrict__ st, unsigned int* blk, int nblk,
                                                          unsigned int* ticket) {
+  pdl_wait();
   __shared__ unsigned int part[kSelBlock];
   __shared__ unsigned int carry;
   const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
@@ -223,6 +226,7 @@ __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t 
                                                         const SelectState* __restrict__ st,
                                                         const unsigned int* __restrict__ blk,
                                                         unsigned char* __restrict__ pid_out, float* wm, int keep_all_or_none) {
+  pdl_wait();
   __shared__ unsigned int warp_cnt[kSelBlock / 32];
   const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
   const bool valid = i < FC;
@@ -288,12 +292,12 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   if (mode < 0) {
     if (int rc = check_cuda(cudaMemsetAsync(ws.hist, 0, 4 * kHistWords, st), "pat_project memset")) return rc;
   }
-  k_select_pattern<<<nb256, 256, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0);
+  launch_dependent(k_select_pattern, dim3(nb256), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0);
   if (mode < 0) {
-    for (int pass = 1; pass < kPasses; ++pass) k_sel_hist<<<nb256, 256, 0, st>>>(ws.key, FC, pass, ws.st, ws.hist);
-    k_tie_count<<<nblk, kSelBlock, 0, st>>>(ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord);
+    for (int pass = 1; pass < kPasses; ++pass) launch_dependent(k_sel_hist, dim3(nb256), dim3(256), 0, st, ws.key, FC, pass, ws.st, ws.hist);
+    launch_dependent(k_tie_count, dim3(nblk), dim3(kSelBlock), 0, st, ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord);
   }
-  k_finalize<<<nblk, kSelBlock, 0, st>>>(w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
+  launch_dependent(k_finalize, dim3(nblk), dim3(kSelBlock), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
   count_launches(mode < 0 ? 6 : 2);
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
