@@ -140,7 +140,7 @@ def run_ours(args):
     # Projection and packing of a layer depend on its weights only, so they run on a second stream while the first
     # stream convolves the layers before it (an event per layer orders the convolution after its own packing): the
     # small projection / packing kernels fill the idle SMs at the ends of the convolution kernels.
-    side = torch.cuda.Stream()
+    side = torch.cuda.Stream(priority=-1)    # its small blocks go first whenever an SM has room
     packed_ev = [torch.cuda.Event() for _ in layers]
 
     def step(conv_events=None, overlap=True):
