@@ -34,7 +34,7 @@ FMA_PEAK_TFLOPS = 2 * FMA_LANES * SM_COUNT * SM_MAX_MHZ * 1e6 / 1e12     # 74.45
 DEFAULT_CONFIG = 3
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_conv_f16_img launch (conv6 shape, batch 32), from
 # profiles/k_conv_f16_img_conv6_b32.md
-CONV6_DRAM_BYTES_B32 = 67.52e6 + 17.59e6
+CONV6_DRAM_BYTES_B32 = 67.53e6 + 17.12e6
 
 
 def measured_peaks():
