@@ -19,6 +19,10 @@ constexpr int kBlockWarps = kExecGroup / 2;         // consumer warps that share
 // offset of the kernel's window inside a stage image): bytes of a pixel row and of a channel plane.
 constexpr int kImgRowBytes = 128;
 constexpr int kImgPlaneBytes = 36 * kImgRowBytes;
+// fp32 blobs: stages of 8 channels (the same bytes per stage), rows and planes twice as large, 32-byte operations
+constexpr int kChanStageF32 = 8;
+constexpr int kImgRowBytesF32 = 256;
+constexpr int kImgPlaneBytesF32 = 36 * kImgRowBytesF32;
 // Descriptor word (see pattern_word below): bits 18 / 19 / 20 = "swap the accumulator tiles before this kernel" /
 // "last operation of this warp in this stage" / "no kernel: the warp has nothing to do in this stage",
 // bits 21-31 = where the warp's list starts in the next stage's block.
@@ -41,8 +45,8 @@ constexpr size_t kHeaderBytes = 768;
 struct BlobLayout {
   size_t perm, fptr, pptr, chan, w4;   // canonical section
   size_t xfilt, tptr, tmeta, tw4;      // execution section (its own filter order, see pack.cu)
-  size_t dboff, dblk;                  // descriptor blocks (fp16 blobs with F % 32 == 0 and C % 16 == 0; else empty)
-  int nblk;                            // number of descriptor blocks = (F / 32) * nct, or 0
+  size_t dboff, dblk;                  // descriptor blocks (blobs with F % 32 == 0 and C % 16 == 0; else empty)
+  int nblk;                            // number of descriptor blocks = (F / 32) * (C / 16) for fp16, (F / 32) * (C / 8) for fp32, or 0
   size_t scratch;                      // pack-time temporaries: hist[F][K], count[F], inv[F], xinv[F], xbase[F]
   size_t total;
   int nct;                             // number of 16-channel tiles = ceil(C / 16)
@@ -66,9 +70,11 @@ __host__ __device__ inline BlobLayout blob_layout(int F, int C, int K, int64_t n
   L.tptr = o;  o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)L.nct + 1));
   L.tmeta = o; o = align256(o + sizeof(uint32_t) * nk);
   L.tw4 = o;   o = align256(o + 4 * e * nk);
-  L.nblk = (dtype == PAT_F16 && F % kExecGroup == 0 && C % kChanTile == 0) ? (F / kExecGroup) * L.nct : 0;
+  const bool has_blocks = F % kExecGroup == 0 && C % kChanTile == 0;
+  const size_t op_bytes = dtype == PAT_F16 ? 16 : 32;          // one operation of a descriptor block
+  L.nblk = !has_blocks ? 0 : (dtype == PAT_F16 ? (F / kExecGroup) * L.nct : (F / kExecGroup) * (C / kChanStageF32));
   L.dboff = o; o = align256(o + (L.nblk ? sizeof(uint32_t) * ((size_t)L.nblk + 1) : 0));
-  L.dblk = o;  o = align256(o + (L.nblk ? (size_t)L.nblk * (kBlockHeaderBytes + 16 * kBlockWarps) + 16 * nk : 0));
+  L.dblk = o;  o = align256(o + (L.nblk ? (size_t)L.nblk * (kBlockHeaderBytes + op_bytes * kBlockWarps) + op_bytes * nk : 0));
   L.scratch = o; o = align256(o + sizeof(int32_t) * (size_t)F * ((size_t)K + 4));
   L.total = o;
   return L;

@@ -11,6 +11,9 @@ bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int st
 size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                  const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st);
+size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
+int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st);
 }
 
 using namespace pat;
@@ -42,17 +45,18 @@ extern "C" int pat_conv3x3(const void* blob, int F, int C, const uint16_t* masks
 
 extern "C" size_t pat_conv3x3_workspace(int F, int C, int dtype, int N, int H, int W, int stride) {
   if (F < 1 || C < 1 || N < 1 || H < 1 || W < 1) return 0;
-  return conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
+  return dtype == PAT_F32 ? conv_f32_img_workspace(F, C, dtype, N, H, W, stride) : conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
 }
 
 extern "C" int pat_conv3x3_ws(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                               int dtype, const void* x, void* y, int N, int H, int W, int stride,
                               void* workspace, size_t workspace_bytes, void* stream) {
   if (int rc = check_conv_args(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride)) return rc;
-  const size_t need = conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
+  const size_t need = pat_conv3x3_workspace(F, C, dtype, N, H, W, stride);
   if (need == 0) return pat_conv3x3(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, stream);
   if (!workspace || workspace_bytes < need)
     return set_error(PAT_ERR_WORKSPACE, "pat_conv3x3_ws: workspace has %zu bytes, needs %zu", workspace_bytes, need);
   if (!aligned(workspace, 256)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3_ws: workspace must be 256-byte aligned");
+  if (dtype == PAT_F32) return conv_f32_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, workspace, reinterpret_cast<cudaStream_t>(stream));
   return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, workspace, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -1,0 +1,654 @@
+// Sparse 3x3 convolution for fp32 storage and accumulation, stride 1 (sm_100a): the workspace path of conv_f16_img.cu
+// for 4-byte activations.  The same three kernels and the same protocol (stage images built once per call, a
+// persistent warp-specialised kernel fed by bulk copies through a ring of shared-memory slots, flat pack-time
+// operation lists, one accumulator tile in registers and one parked in tensor memory, cut items reduced by a third
+// kernel); what differs:
+//  * a stage holds 8 input channels (the same 72 KB): channel-planar [8 ch][36 rows][4 segments][16 px] floats, a
+//    segment = four 16-byte chunks.  Physical chunk = logical chunk ^ (segment / 2 + 2 x parity of the tile row whose
+//    window starts in that row's group of four), so the eight lanes that share a wavefront of a 16-byte load
+//    (four column slots x two tile rows) touch eight different bank groups;
+//  * an operation is 32 bytes (four fp32 taps), a window row is four 16-byte loads and plain fp32 multiply-adds;
+//  * the results leave in two rounds (tile rows 0-1, then 2-3): a slot takes one tile row of fp32 results.
+#include <algorithm>
+#include "f16_tile.cuh"
+
+namespace pat {
+namespace img32 {
+using namespace fast16;
+
+constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three idle warps (register donors)
+constexpr int W_PRODUCER = NCW;
+constexpr int CBI = kChanStageF32;         // channels per ring stage (8)
+constexpr int SEGF = 64;                   // bytes of a segment: 16 px of one channel
+constexpr int ROWF = LX * SEGF;            // 256
+constexpr int MAXROWS = LY * TR4 + 4;      // 36
+constexpr int CHPF = MAXROWS * ROWF;       // channel plane pitch (9216)
+constexpr int IMG_BYTES = CBI * CHPF;      // 73728
+static_assert(ROWF == kImgRowBytesF32 && CHPF == kImgPlaneBytesF32 && NCW == kBlockWarps, "the descriptor blocks are written for this geometry");
+constexpr int MAX_NS = 3;
+constexpr int OPB = 32;                    // bytes of an operation
+constexpr int MAXE3 = 108;                 // operations of a descriptor block that still allow three slots
+constexpr int DBLK3 = kBlockHeaderBytes + MAXE3 * OPB;                       // 3584
+constexpr int DBLK2 = kBlockHeaderBytes + (FG * CBI + kBlockWarps + 4) * OPB; // largest possible block and spare slots (8960)
+constexpr int OFF_SLOTS = 256;
+constexpr int SMEM_BYTES = OFF_SLOTS + 3 * (IMG_BYTES + DBLK3);
+static_assert(OFF_SLOTS + 2 * (IMG_BYTES + DBLK2) <= SMEM_BYTES, "the two-slot layout fits too");
+static_assert(IMG_BYTES % 128 == 0 && DBLK3 % 128 == 0 && DBLK2 % 128 == 0 && SMEM_BYTES <= 232448, "shared memory budget of one SM");
+constexpr int OUT_PITCH = FG * 4 + 4;      // output staging inside a slot: [448 px][32 channels] fp32, pixel pitch 132 B
+constexpr int OUT_ROW = 32 * TC * OUT_PITCH;   // one row of every thread tile (59136)
+static_assert(OUT_ROW <= IMG_BYTES, "one tile row of results fits a slot");
+constexpr int CONSUMER_REGS = 112, OTHER_REGS = 32;
+static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
+constexpr uint32_t TMEM_COLS = 512;
+
+struct Params {
+  const float* x;
+  float* y;
+  char* images;            // stage images: [region][stage of 8 channels][IMG_BYTES]
+  const int32_t* xfilt;    // execution position -> original filter
+  const uint32_t* dboff;   // descriptor block -> offset in 16-byte units
+  const char* dblk;
+  const BlobHeader* hdr;
+  int* status;
+  int N, H, W, C, F, K, nst;  // nst = stages of 8 channels
+  long long n_keep;
+  int TY, TXe, NI, CG, NIG, NG;
+  int n_regions, n_items;
+  int n_whole, n_split, parts;   // cut items: see conv_f16_img.cu
+  float* partials;
+  uint16_t masks[256];
+};
+
+struct Region {
+  int cg, ig0, ta0, n0;
+  bool band1;
+  int nrows;
+};
+__device__ __forceinline__ Region decode_region(const Params& p, int reg) {
+  Region r;
+  r.cg = reg % p.CG;
+  const int gt0 = (reg / p.CG) * LY;
+  r.ig0 = gt0 / p.TY;
+  r.ta0 = gt0 % p.TY;
+  r.n0 = min(LY, p.TY - r.ta0);
+  r.band1 = (r.n0 < LY) && (r.ig0 + 1 < p.NIG);
+  r.nrows = r.band1 ? MAXROWS : TR4 * r.n0 + 2;
+  return r;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------ stage images
+// One block per (region, stage of 8 channels).  Image layout: byte ch * CHPF + row * ROWF + seg * SEGF +
+// ((px >> 2) ^ sw) * 16 + (px & 3) * 4 with px = 0..15 <-> image column 14 * (tile column) - 1 + px and
+// sw = seg / 2 + 2 * (parity of the tile row, counted through both bands, whose window starts in that row's group of four).
+constexpr int SI_THREADS = 256;
+constexpr int SI_PITCH = CHPF + 16;        // the two channel quads a warp writes at once fall into different bank halves
+constexpr int SI_SMEM = CBI * SI_PITCH;
+__global__ void __launch_bounds__(SI_THREADS) k_stage_images_f32(const Params p) {
+  extern __shared__ __align__(16) unsigned char img[];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see conv_f16_img.cu
+  const int st8 = (int)(blockIdx.x % (unsigned)p.nst);
+  const int reg = (int)(blockIdx.x / (unsigned)p.nst);
+  const Region r = decode_region(p, reg);
+  const int rows0 = TR4 * r.n0 + 2;
+  const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+  // a unit = one pixel x one channel quad: one 16-byte load, four 4-byte stores
+  constexpr int UNITS = MAXROWS * LX * 16 * 2, PER_THREAD = UNITS / SI_THREADS;   // 18 per thread
+  static_assert(UNITS % SI_THREADS == 0, "units per thread");
+  uint4 v[PER_THREAD];
+#pragma unroll
+  for (int i = 0; i < PER_THREAD; ++i) {
+    const int u = (int)threadIdx.x + SI_THREADS * i;
+    const int quad = u & 1, k = (u >> 1) & 15, seg = (u >> 5) & 3, pr = u >> 7;
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (pr < r.nrows) {
+      const int b = (pr >= rows0) ? 1 : 0;
+      const int yy = b ? (pr - rows0 - 1) : (TR4 * r.ta0 - 1 + pr);
+      const int ni = seg >> txe_shift, tx = seg & (p.TXe - 1);
+      const int n_img = (r.ig0 + b) * p.NI + ni;
+      const int xx = (r.cg * p.TXe + tx) * TC - 1 + k;
+      if (yy >= 0 && yy < p.H && n_img < p.N && xx >= 0 && xx < p.W)
+        v[i] = __ldg(reinterpret_cast<const uint4*>(p.x + (((size_t)n_img * p.H + yy) * p.W + xx) * p.C + st8 * CBI + quad * 4));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < PER_THREAD; ++i) {
+    const int u = (int)threadIdx.x + SI_THREADS * i;
+    const int quad = u & 1, k = (u >> 1) & 15, seg = (u >> 5) & 3, pr = u >> 7;
+    const int b = (pr >= rows0) ? 1 : 0;
+    const int par = ((((b ? pr - rows0 : pr) >> 2) + (b ? r.n0 : 0)) & 1);
+    const int sw = (seg >> 1) | (par << 1);
+    const uint32_t o = (uint32_t)(pr * ROWF + seg * SEGF + (((k >> 2) ^ sw) << 4) + (k & 3) * 4);
+    *reinterpret_cast<uint32_t*>(img + (quad * 4 + 0) * SI_PITCH + o) = v[i].x;
+    *reinterpret_cast<uint32_t*>(img + (quad * 4 + 1) * SI_PITCH + o) = v[i].y;
+    *reinterpret_cast<uint32_t*>(img + (quad * 4 + 2) * SI_PITCH + o) = v[i].z;
+    *reinterpret_cast<uint32_t*>(img + (quad * 4 + 3) * SI_PITCH + o) = v[i].w;
+  }
+  __syncthreads();
+  uint4* dst = reinterpret_cast<uint4*>(p.images + (size_t)blockIdx.x * IMG_BYTES);
+  for (int i = threadIdx.x; i < IMG_BYTES / 16; i += SI_THREADS) {
+    const int ch = i / (CHPF / 16), w = i % (CHPF / 16);
+    dst[i] = *reinterpret_cast<const uint4*>(img + ch * SI_PITCH + w * 16);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ consumer math
+__device__ __forceinline__ void lds_row_f32(float (&h)[16], uint32_t a, uint32_t x) {
+  // a = address of logical chunk 0 of the row (64-byte aligned), x = the lane's chunk swizzle for this row (bits 4-5)
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t q0, q1, q2, q3;
+    lds128((a + 16u * c) ^ x, q0, q1, q2, q3);
+    h[4 * c] = __uint_as_float(q0); h[4 * c + 1] = __uint_as_float(q1); h[4 * c + 2] = __uint_as_float(q2); h[4 * c + 3] = __uint_as_float(q3);
+  }
+}
+
+// The code of one pattern on a 4 x 14 tile (see pattern_body4 in f16_tile.cuh): a0 = address of logical chunk 0 of
+// window row `sh`, swb = the lane's chunk swizzle (bits 4-5) for window rows 0-3; from window row 4 on the rows
+// belong to the next tile row's group, whose parity bit is the other one.
+template <uint32_t MASK>
+__device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a0, uint32_t sh, uint32_t swb, const float (&w)[4]) {
+  constexpr int NR = last_tap_row(MASK) + TR4;
+#pragma unroll
+  for (int j = 0; j < NR; ++j) {
+    uint32_t x = swb;
+    if (j >= 4) x ^= 32u;
+    else if (j == 3) x ^= sh << 5;
+    float h[16];
+    lds_row_f32(h, a0 + j * ROWF, x);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int b = nth_bit(MASK, t);
+      const int y = j - b / 3, c = b % 3;
+      if (y >= 0 && y < TR4) {
+#pragma unroll
+        for (int xx = 0; xx < TC; ++xx) acc[y][xx] = fmaf(h[xx + c], w[t], acc[y][xx]);
+      }
+    }
+  }
+}
+
+template <int NCODES, bool GENERIC>
+__device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t plane, uint32_t swb, uint32_t meta, uint32_t off,
+                                             float (&w)[4]) {
+  static_assert(NCODES == 6 || NCODES == kNumCodes, "code sets with compiled dispatch trees");
+  const uint32_t sh = (meta >> 17) & 1u;
+  const uint32_t a0 = plane + off;
+  const uint32_t code = (meta >> 13) & 15u;
+  if ((NCODES > 8 || GENERIC) && (code & 8u)) {
+    if (code & 4u) {
+      if constexpr (GENERIC) {
+        // any other pattern: position by position, each with its own pass over the window rows it reads
+        const uint32_t base = a0 - sh * ROWF;
+#define PAT_TAP4F(B)                                                                         \
+  if (meta & (16u << (B))) {                                                                 \
+    _Pragma("unroll")                                                                        \
+    for (int y = 0; y < TR4; ++y) {                                                          \
+      float h[16];                                                                           \
+      const int jr = y + (B) / 3;                                                            \
+      lds_row_f32(h, base + jr * ROWF, jr >= 4 ? (swb ^ 32u) : swb);                         \
+      _Pragma("unroll")                                                                      \
+      for (int xx = 0; xx < TC; ++xx) acc[y][xx] = fmaf(h[xx + (B) % 3], w[0], acc[y][xx]);  \
+    }                                                                                        \
+    w[0] = w[1]; w[1] = w[2]; w[2] = w[3];                                                   \
+  }
+        PAT_TAP4F(0) PAT_TAP4F(1) PAT_TAP4F(2) PAT_TAP4F(3) PAT_TAP4F(4) PAT_TAP4F(5) PAT_TAP4F(6) PAT_TAP4F(7) PAT_TAP4F(8)
+#undef PAT_TAP4F
+      }
+    } else if constexpr (NCODES > 8) {
+      if (code & 1u) pattern_body4f<code_mask(9)>(acc, a0, sh, swb, w);
+      else pattern_body4f<code_mask(8)>(acc, a0, sh, swb, w);
+    }
+  } else if (code & 4u) {
+    if (NCODES > 6 && (code & 2u)) {
+      if constexpr (NCODES > 6) {
+        if (code & 1u) pattern_body4f<code_mask(7)>(acc, a0, sh, swb, w);
+        else pattern_body4f<code_mask(6)>(acc, a0, sh, swb, w);
+      }
+    } else {
+      if (code & 1u) pattern_body4f<code_mask(5)>(acc, a0, sh, swb, w);
+      else pattern_body4f<code_mask(4)>(acc, a0, sh, swb, w);
+    }
+  } else {
+    if (code & 2u) {
+      if (code & 1u) pattern_body4f<code_mask(3)>(acc, a0, sh, swb, w);
+      else pattern_body4f<code_mask(2)>(acc, a0, sh, swb, w);
+    } else {
+      if (code & 1u) pattern_body4f<code_mask(1)>(acc, a0, sh, swb, w);
+      else pattern_body4f<code_mask(0)>(acc, a0, sh, swb, w);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ the convolution
+// Ring protocol as in conv_f16_img.cu: per work item nst stages of 8 channels, then two output stages whose slots
+// the consumers use as staging for the results - here twice (tile rows 0-1, then 2-3), with a block-wide barrier
+// after writing and after copying out the first pair of rows.
+template <bool SPARSE, int NCODES, bool GENERIC>
+__device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
+  constexpr int NS = SPARSE ? 3 : 2;
+  constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
+  const uint32_t sbase = smem_u32(smem);
+  auto slot_full = [&](int s) { return sbase + 8u * s; };
+  auto slot_empty = [&](int s) { return sbase + 8u * (MAX_NS + s); };
+  auto out_ready = [&](int s) { return sbase + 8u * (2 * MAX_NS + s); };   // 0: results written, 1: first rows copied out
+  static_assert(8 * 3 * MAX_NS + 8 <= OFF_SLOTS, "barrier block and control words");
+  int& s_abort = *reinterpret_cast<int*>(smem + 8 * 3 * MAX_NS);
+  uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(smem + 8 * 3 * MAX_NS + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t slot0 = sbase + OFF_SLOTS;
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < MAX_NS; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), NCW); mbar_init(out_ready(s), NCW); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) tmem_alloc(smem_u32(&s_tmem), TMEM_COLS);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  volatile int* abort_flag = &s_abort;
+  const uint32_t tmem_base = s_tmem;
+
+  const int n_my_whole = (p.n_whole > (int)blockIdx.x) ? (p.n_whole - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int n_my_items = n_my_whole + ((p.parts > 1 && (int)blockIdx.x < p.n_split * p.parts) ? 1 : 0);
+  const int nst = p.nst;
+  auto item_of = [&](int it_idx) {
+    return it_idx < n_my_whole ? (int)blockIdx.x + it_idx * (int)gridDim.x : p.n_whole + (int)blockIdx.x / p.parts;
+  };
+  auto piece_of = [&](int it_idx, int& c0, int& c1) {
+    if (it_idx < n_my_whole) { c0 = 0; c1 = nst; return false; }
+    const int q = (int)blockIdx.x % p.parts;
+    c0 = q * nst / p.parts; c1 = (q + 1) * nst / p.parts;
+    return true;
+  };
+
+  if (warp >= NCW) {
+    set_warp_registers<OTHER_REGS>();
+    if (warp == W_PRODUCER) {
+      // ========================================================================= producer warp
+      int pslot = 0;
+      uint32_t epar = 1u;
+      uint32_t armed = 0u, armed_par = 0u;
+      bool alive = true;
+      for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
+        const int item = item_of(it_idx);
+        const int g = item % p.NG, reg = item / p.NG;
+        const char* img = p.images + (size_t)reg * nst * IMG_BYTES;
+        const uint32_t* bo = p.dboff + (size_t)g * nst;
+        int c0, c1;
+        const bool piece = piece_of(it_idx, c0, c1);
+        uint32_t o0 = __ldg(bo + c0);
+        for (int cb = c0; cb < c1 && alive; ++cb) {
+          const uint32_t o1 = __ldg(bo + cb + 1);
+          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
+          if (lane == 0) {
+            const uint32_t dbytes = (o1 - o0) * 16u;
+            const uint32_t dst = slot0 + (uint32_t)pslot * SLOT;
+            mbar_arrive_expect_tx(slot_full(pslot), (uint32_t)IMG_BYTES + dbytes);
+            bulk_load(dst + IMG_BYTES, p.dblk + (size_t)o0 * 16, dbytes, slot_full(pslot));
+            bulk_load(dst, img + (size_t)cb * IMG_BYTES, (uint32_t)IMG_BYTES, slot_full(pslot));
+          }
+          armed |= 1u << pslot;
+          armed_par = (armed_par & ~(1u << pslot)) | ((epar ^ 1u) << pslot);
+          o0 = o1;
+          if (++pslot == NS) { pslot = 0; epar ^= 1u; }
+        }
+        // output stages: hand the next two slots to the consumers as they become free (a piece has none)
+        for (int o = 0; o < 2 && alive && !piece; ++o) {
+          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
+          if (lane == 0) mbar_arrive(slot_full(pslot));
+          armed &= ~(1u << pslot);
+          if (++pslot == NS) { pslot = 0; epar ^= 1u; }
+        }
+      }
+      if (!alive && lane == 0) {
+        const unsigned long long t0 = global_ns();
+        for (int s = 0; s < NS; ++s) {
+          if (!((armed >> s) & 1u)) continue;
+          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+            if (mbar_try_wait(slot_full(s), (armed_par >> s) & 1u)) break;
+            if (global_ns() - t0 > kWaitNs) break;
+          }
+        }
+        atomicExch(p.status, PAT_ERR_TIMEOUT);
+      }
+    }
+  } else {
+    // =========================================================================== consumer warps
+    set_warp_registers<CONSUMER_REGS>();
+    const uint32_t tm0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+    auto park = [&](uint32_t f, const float (&a)[TR4][TC]) {
+      tmem_store_tile(tm0 + f * 64u, a);
+      tmem_wait_st();
+    };
+    auto fetch = [&](uint32_t f, float (&a)[TR4][TC]) {
+      tmem_load_tile(tm0 + f * 64u, a);
+      tmem_wait_ld();
+    };
+    int pslot = 0;
+    uint32_t fpar = 0u;
+    bool alive = true;
+    for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
+      const int item = item_of(it_idx);
+      const Region it = decode_region(p, item / p.NG);
+      const int ly = lane >> 2, lx = lane & 3;
+      const int band = (ly < it.n0) ? 0 : 1;
+      // the lane's address of logical chunk 0 of window row 0, relative to a channel plane, and its chunk swizzle
+      const uint32_t offA = (uint32_t)((TR4 * ly + 2 * band) * ROWF + lx * SEGF);
+      const uint32_t swb = (uint32_t)(((lx >> 1) | ((ly & 1) << 1)) << 4);
+      float acc[TR4][TC];
+#pragma unroll
+      for (int y = 0; y < TR4; ++y)
+#pragma unroll
+        for (int x = 0; x < TC; ++x) acc[y][x] = 0.0f;
+      int c0, c1;
+      const bool piece = piece_of(it_idx, c0, c1);
+      if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+      uint32_t sl = slot0 + (uint32_t)pslot * SLOT;
+      uint32_t pl0 = sl + offA;
+      const uint32_t hw = lds32(sl + IMG_BYTES + (uint32_t)warp * 4u);
+      uint32_t cur = hw >> 31;           // which of the two filters the registers hold (both tiles are zero now)
+      park(cur ^ 1u, acc);
+      uint32_t e = sl + IMG_BYTES + kBlockHeaderBytes + (hw & 0xFFFFu) * 16u;
+      uint32_t m0, off, w0, w1, w2, w3, pad0, pad1;
+      lds128(e, m0, off, w0, w1);
+      lds128(e + 16u, w2, w3, pad0, pad1);
+      int cb = c0;
+#pragma unroll 1
+      for (;;) {
+        const uint32_t cm = m0, coff = off;
+        float w[4] = {__uint_as_float(w0), __uint_as_float(w1), __uint_as_float(w2), __uint_as_float(w3)};
+        e += OPB;
+        lds128(e, m0, off, w0, w1);        // the next operation
+        lds128(e + 16u, w2, w3, pad0, pad1);
+        if (cm & (kOpSwap | kOpNop)) {     // one test for the two rare cases
+          if (cm & kOpNop) goto stage_end;
+          park(cur, acc);
+          cur ^= 1u;
+          fetch(cur, acc);
+        }
+        one_kernel4f<NCODES, GENERIC>(acc, pl0, swb, cm, coff, w);
+      stage_end:
+        if (cm & kOpEnd) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(slot_empty(pslot));
+          if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
+          if (++cb == c1) break;
+          if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+          sl = slot0 + (uint32_t)pslot * SLOT;
+          pl0 = sl + offA;
+          e = sl + IMG_BYTES + kBlockHeaderBytes + (cm >> kOpNextShift) * 16u;
+          lds128(e, m0, off, w0, w1);
+          lds128(e + 16u, w2, w3, pad0, pad1);
+        }
+      }
+      if (!alive) break;
+
+      if (piece) {
+        // partial sums of a cut item: one 128-byte line per value and warp
+        float* dst = p.partials + (size_t)blockIdx.x * (FG * TR4 * TC * 32) + lane;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          float* d = dst + (size_t)(cur ? FG - 1 - warp : warp) * (TR4 * TC * 32);
+#pragma unroll
+          for (int y = 0; y < TR4; ++y)
+#pragma unroll
+            for (int x = 0; x < TC; ++x) d[(y * TC + x) * 32] = acc[y][x];
+          if (half == 0) {
+            cur ^= 1u;
+            fetch(cur, acc);
+          }
+        }
+        continue;
+      }
+
+      // results, two rounds: tile row 2 r into the first output slot, 2 r + 1 into the second, as [pixel][32 channels];
+      // once all 16 warps have written, every warp copies those rows of two thread tiles to global memory
+      const int g_out = item % p.NG;
+      const uint32_t cposA = ((uint32_t)__ldg(p.xfilt + g_out * FG + warp) & (uint32_t)(FG - 1)) * 4u;
+      const uint32_t cposB = ((uint32_t)__ldg(p.xfilt + g_out * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 4u;
+      const int s0 = pslot, s1 = (pslot + 1 == NS) ? 0 : pslot + 1;
+      const uint32_t par1 = (pslot + 1 == NS) ? (fpar ^ 1u) : fpar;
+      if (!mbar_wait<0>(slot_full(s0), fpar, abort_flag)) { alive = false; break; }
+      if (!mbar_wait<0>(slot_full(s1), par1, abort_flag)) { alive = false; break; }
+      const uint32_t ob0 = slot0 + (uint32_t)s0 * SLOT, ob1 = slot0 + (uint32_t)s1 * SLOT;
+      const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+      // tiles 16-31 sit one word further on: lanes l and l + 16 would otherwise store to the same banks
+      const uint32_t ol = (uint32_t)(lane * TC) * OUT_PITCH + (uint32_t)(lane >> 4) * 4u;
+#pragma unroll 1
+      for (int round = 0; round < 2 && alive; ++round) {
+        // this round's two rows of both filters: the one in registers first, then the other one
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t cp = ol + (cur ? cposB : cposA);
+#pragma unroll
+          for (int x = 0; x < TC; ++x) {
+            sts32(ob0 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[2][x] : acc[0][x]));
+            sts32(ob1 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[3][x] : acc[1][x]));
+          }
+          if (half == 0) {
+            if (round == 0) park(cur, acc);     // its rows 2-3 are still to come
+            cur ^= 1u;
+            fetch(cur, acc);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(out_ready(0));
+        if (!mbar_wait<0>(out_ready(0), (uint32_t)round, abort_flag)) { alive = false; break; }
+        // 14 pixels x 8 chunks of 4 channels per tile row: eight consecutive lanes write one pixel's 128 bytes
+        const uint32_t slc = (uint32_t)(lane >> 3) * OUT_PITCH + (uint32_t)(lane & 7) * 16u;
+#pragma unroll 1
+        for (int k = 0; k < 32 / NCW; ++k) {
+          const int t = warp * (32 / NCW) + k;
+          const int tly = t >> 2, tlx = t & 3;
+          const int b = (tly < it.n0) ? 0 : 1;
+          const int ni = tlx >> txe_shift, tx = tlx & (p.TXe - 1);
+          const int ig = it.ig0 + b;
+          const int ty = b ? (tly - it.n0) : (it.ta0 + tly);
+          const int n_img = ig * p.NI + ni;
+          if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
+          const int col0 = (it.cg * p.TXe + tx) * TC;
+          const uint32_t src = slc + (uint32_t)(t * TC) * OUT_PITCH + (uint32_t)(t >> 4) * 4u;
+#pragma unroll
+          for (int yy = 0; yy < 2; ++yy) {
+            const int row = TR4 * ty + 2 * round + yy;
+            float* dst = p.y + (((size_t)n_img * p.H + row) * p.W + col0 + (lane >> 3)) * p.F + g_out * FG + (lane & 7) * 4;
+            uint4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (4 * i + (lane >> 3) < TC) {
+                const uint32_t a = (yy ? ob1 : ob0) + src + (uint32_t)(4 * i) * OUT_PITCH;
+                v[i].x = lds32(a); v[i].y = lds32(a + 4); v[i].z = lds32(a + 8); v[i].w = lds32(a + 12);
+              }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (4 * i + (lane >> 3) < TC && row < p.H)
+                *reinterpret_cast<uint4*>(dst + (size_t)(4 * i) * p.F) = v[i];
+          }
+        }
+        if (round == 0) {
+          // the second pair of rows overwrites the staging: every warp must have copied the first pair out
+          __syncwarp();
+          if (lane == 0) mbar_arrive(out_ready(1));
+          if (!mbar_wait<0>(out_ready(1), (uint32_t)(it_idx & 1), abort_flag)) { alive = false; break; }
+        }
+      }
+      if (!alive) break;
+      // the slots are refilled by bulk copies next: order this warp's accesses to them before those writes
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(slot_empty(s0)); mbar_arrive(slot_empty(s1)); }
+      for (int o = 0; o < 2; ++o)
+        if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+template <int NCODES, bool GENERIC>
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_conv_f32_img(const Params p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const BlobHeader* bh = p.hdr;
+  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
+            bh->K == p.K && bh->dtype == PAT_F32 && bh->n_keep == p.n_keep &&
+            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * CBI + kBlockWarps;
+  for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
+  if (!ok) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
+    return;
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC>(p, smem);
+  else conv_body<false, NCODES, GENERIC>(p, smem);
+}
+
+// ------------------------------------------------------------------------------------------ cut items
+// Adds the partial sums of the pieces of a cut item (piece 0 first) and writes the results.  One block per
+// (cut item, value of the thread tile); thread = (filter position, lane).
+constexpr int MAX_PIECES = 256;
+constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
+constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
+__global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int v = (int)blockIdx.x % (TR4 * TC), li = (int)blockIdx.x / (TR4 * TC);
+  const int item = p.n_whole + li;
+  const int g = item % p.NG;
+  const Region it = decode_region(p, item / p.NG);
+  const int lane = threadIdx.x & 31, slot = threadIdx.x >> 5;
+  const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS + ((size_t)slot * (TR4 * TC) + v) * 32 + lane;
+  float sum = 0.0f;
+  for (int q = 0; q < p.parts; ++q) sum += __ldg(src + (size_t)q * PIECE_FLOATS);   // piece 0 first
+  const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+  const int ly = lane >> 2, lx = lane & 3;
+  const int b = (ly < it.n0) ? 0 : 1;
+  const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+  const int ig = it.ig0 + b;
+  const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+  const int n_img = ig * p.NI + ni;
+  const int row = TR4 * ty + v / TC, col = (it.cg * p.TXe + tx) * TC + v % TC;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H) return;
+  p.y[(((size_t)n_img * p.H + row) * p.W + col) * p.F + __ldg(p.xfilt + g * FG + slot)] = sum;
+}
+
+// ------------------------------------------------------------------------------------------ host side
+static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
+  p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
+  p.nst = C / CBI;
+  p.TY = (H + TR4 - 1) / TR4;
+  const int TX = W / TC;
+  p.TXe = TX >= LX ? LX : TX;
+  p.NI = LX / p.TXe;
+  p.CG = TX / p.TXe;
+  p.NIG = (N + p.NI - 1) / p.NI;
+  p.NG = F / FG;
+  const long long row_blocks = ((long long)p.NIG * p.TY + LY - 1) / LY;
+  const long long regions = row_blocks * p.CG;
+  const long long items = regions * p.NG;
+  if (items > 0x7FFFFFFFll || regions * p.nst > 0x7FFFFFFFll) return false;
+  p.n_regions = (int)regions;
+  p.n_items = (int)items;
+  p.n_whole = p.n_items; p.n_split = 0; p.parts = 1; p.partials = nullptr;
+  return true;
+}
+
+}  // namespace img32
+
+// True when the fp32 stage-image kernels cover this layer.
+bool conv_f32_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
+  using namespace img32;
+  if (dtype != PAT_F32 || stride != 1) return false;
+  const int TY = (H + TR4 - 1) / TR4;
+  if (W % TC != 0 || !(TY >= LY - 1 || 2 * TY == LY)) return false;
+  const int TX = W / TC;
+  if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
+  if (C % kChanTile != 0 || F % FG != 0) return false;
+  Params p;
+  return N >= 1 && fill_geometry(p, F, C, N, H, W);
+}
+
+size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride) {
+  using namespace img32;
+  if (!conv_f32_img_supported(F, C, dtype, N, H, W, stride)) return 0;
+  Params p;
+  if (!fill_geometry(p, F, C, N, H, W)) return 0;
+  return align256((size_t)p.n_regions * p.nst * IMG_BYTES) + MAX_PIECES * PIECE_FLOATS * sizeof(float);
+}
+
+int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st) {
+  using namespace img32;
+  const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F32);
+  const char* b = static_cast<const char*>(blob);
+  Params p;
+  if (!fill_geometry(p, F, C, N, H, W) || L.nblk == 0) return set_error(PAT_ERR_SHAPE, "pat_conv3x3: layer not covered by the stage-image kernels");
+  p.x = static_cast<const float*>(x);
+  p.y = static_cast<float*>(y);
+  p.images = static_cast<char*>(workspace);
+  p.hdr = reinterpret_cast<const BlobHeader*>(b);
+  p.xfilt = reinterpret_cast<const int32_t*>(b + L.xfilt);
+  p.dboff = reinterpret_cast<const uint32_t*>(b + L.dboff);
+  p.dblk = b + L.dblk;
+  p.status = status_word();
+  if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
+  p.K = K; p.n_keep = n_keep;
+  for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
+
+  int variant = 0;
+  for (int j = 0; j < K; ++j) {
+    const int code = (int)((pattern_word(masks[j]) >> 13) & 15u);
+    variant = std::max(variant, code == kGenericCode ? 2 : (code >= 6 ? 1 : 0));
+  }
+  using KernelFn = void (*)(const Params);
+  static const KernelFn kernels[3] = {k_conv_f32_img<6, false>, k_conv_f32_img<kNumCodes, false>, k_conv_f32_img<kNumCodes, true>};
+
+  static thread_local int sm_count = 0;
+  static thread_local bool attr_set = false;
+  if (!attr_set) {
+    int dev = 0;
+    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
+    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
+    if (int rc = check_cuda(cudaFuncSetAttribute(k_stage_images_f32, cudaFuncAttributeMaxDynamicSharedMemorySize, SI_SMEM), "set shared memory size")) return rc;
+    for (KernelFn fn : kernels) {
+      if (int rc = check_cuda(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
+      cudaFuncAttributes fa;
+      if (int rc = check_cuda(cudaFuncGetAttributes(&fa, fn), "query kernel attributes")) return rc;
+      if (fa.numRegs < LAUNCH_REGS)
+        return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
+    }
+    attr_set = true;
+  }
+  const int grid = std::min(p.n_items, sm_count);
+  const int left = p.n_items % grid;
+  if (left > 0) {
+    const int parts = std::min(std::min(MAX_PARTS, p.nst), std::min(grid, MAX_PIECES) / left);
+    if (parts >= 2) {
+      p.n_whole = p.n_items - left; p.n_split = left; p.parts = parts;
+      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nst * IMG_BYTES));
+    }
+  }
+  k_stage_images_f32<<<(unsigned)(p.n_regions * p.nst), SI_THREADS, SI_SMEM, st>>>(p);
+  cudaLaunchAttribute pdl;
+  pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = st; cfg.attrs = &pdl; cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM_BYTES;
+  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant], p), "pat_conv3x3 launch")) return rc;
+  count_launches(2);
+  if (p.parts > 1) {
+    cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * TC)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
+    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, k_reduce_parts_f32, p), "pat_conv3x3 launch")) return rc;
+    count_launches(1);
+  }
+  return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");
+}
+
+}  // namespace pat

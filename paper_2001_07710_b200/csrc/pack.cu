@@ -346,6 +346,88 @@ __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable
   }
 }
 
+// Descriptor blocks of fp32 blobs: the same lists for stages of 8 channels (a tile of 16 channels of the
+// execution section gives two stages: its kernels with channel 0-7 and 8-15, each in (pattern, channel) order) and
+// 32-byte operations:
+//   {channel inside the stage | pattern_word(mask) | flags, byte offset of the window in an fp32 stage image, taps 0-1}
+//   {taps 2-3, 0, 0}
+// Offsets (header words, "next list", dboff) count 16-byte units as in fp16 blobs, so an operation is two units.
+__global__ void __launch_bounds__(32) k_pack_blocks_f32(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
+  pdl_wait();
+  const int blk = blockIdx.x, lane = threadIdx.x;
+  const int nst = 2 * nct;                                   // stages of 8 channels
+  const int g = blk / nst, st8 = blk % nst;
+  const bool active = lane < kBlockWarps;
+  const int w = active ? lane : 0;
+  const int32_t* rowA = bp.tptr + (size_t)(g * kExecGroup + w) * (nct + 1);
+  const int32_t* rowB = bp.tptr + (size_t)(g * kExecGroup + kExecGroup - 1 - w) * (nct + 1);
+  // kernels of a filter slot in stage s: those of tile s / 2 whose channel lies in half s % 2
+  auto count = [&](const int32_t* row, int s) {
+    const int t = s >> 1, half = s & 1;
+    int n = 0;
+    for (int k = row[t]; k < row[t + 1]; ++k) n += ((int)(((bp.tmeta[k] & 0xFFFFu) >> 3) & 1u) == half) ? 1 : 0;
+    return n;
+  };
+  int cur = 0;                                               // which tile the warp holds when this stage begins
+  for (int s = 0; s < st8; ++s)
+    if (count(cur ? rowA : rowB, s) > 0) cur ^= 1;
+  const int nA = count(rowA, st8), nB = count(rowB, st8);
+  const int cap = active ? nA + nB + 1 : 0;
+  const int cap_next = (active && st8 + 1 < nst) ? count(rowA, st8 + 1) + count(rowB, st8 + 1) + 1 : 0;
+  int incl = cap, incl_next = cap_next;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, off), vn = __shfl_up_sync(0xFFFFFFFFu, incl_next, off);
+    if (lane >= off) { incl += v; incl_next += vn; }
+  }
+  const int start = incl - cap, start_next = incl_next - cap_next;
+  const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+  // kernels of this group in earlier stages (all 32 filter slots)
+  const int32_t* row = bp.tptr + (size_t)(g * kExecGroup + lane) * (nct + 1);
+  int before = row[st8 >> 1] - row[0] + ((st8 & 1) ? count(row, st8 - 1) : 0);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, off);
+  const uint32_t group_first = (uint32_t)bp.tptr[(size_t)(g * kExecGroup) * (nct + 1)];
+  const uint32_t off16 = (uint32_t)blk * (uint32_t)(kBlockHeaderBytes / 16 + 2 * kBlockWarps) + 2u * (group_first + (uint32_t)before);
+  if (lane == 0) {
+    bp.dboff[blk] = off16;
+    if (blk == nblk - 1) bp.dboff[nblk] = off16 + kBlockHeaderBytes / 16 + 2u * (uint32_t)tot;
+    atomicMax(&bp.hdr->max_block_entries, tot);
+  }
+  char* base = bp.dblk + (size_t)off16 * 16;
+  reinterpret_cast<uint32_t*>(base)[lane] = active ? ((uint32_t)(2 * start) | ((uint32_t)cur << 31)) : 0u;
+  if (!active) return;
+  uint4* ent = reinterpret_cast<uint4*>(base + kBlockHeaderBytes) + 2 * start;
+  const uint4* tw4 = static_cast<const uint4*>(bp.tw4);       // four fp32 taps per kernel
+  const int n_first = cur ? nB : nA, n_second = cur ? nA : nB;
+  const int n_ops = n_first + n_second;
+  const uint32_t end_flags = kOpEnd | ((uint32_t)(2 * start_next) << kOpNextShift);
+  if (n_ops == 0) {
+    ent[0] = make_uint4(kOpNop | end_flags, 0u, 0u, 0u);
+    ent[1] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const int t16 = st8 >> 1, half = st8 & 1;
+  int k_out = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    const int32_t* r = (pass == 0) == (cur == 0) ? rowA : rowB;   // first the filter whose tile is held
+    for (int k = r[t16]; k < r[t16 + 1]; ++k) {
+      const uint32_t mt = bp.tmeta[k];
+      const uint32_t ch16 = (mt & 0xFFFFu) - (uint32_t)(t16 * kChanTile);
+      if ((int)(ch16 >> 3) != half) continue;
+      const uint32_t ch = ch16 & 7u;
+      const uint32_t pw = pattern_word(lib.m[mt >> 16]);
+      uint32_t flags = 0u;
+      if (k_out == n_first) flags |= kOpSwap;
+      if (k_out == n_ops - 1) flags |= end_flags;
+      const uint4 wv = tw4[k];
+      ent[2 * k_out] = make_uint4(ch | pw | flags, ch * (uint32_t)kImgPlaneBytesF32 + ((pw >> 17) & 1u) * (uint32_t)kImgRowBytesF32, wv.x, wv.y);
+      ent[2 * k_out + 1] = make_uint4(wv.z, wv.w, 0u, 0u);
+      ++k_out;
+    }
+  }
+}
+
 __device__ inline bool header_matches(const BlobHeader* h, int F, int C, int K, long long n_keep, int dtype, const MaskTable& lib) {
   if (h->magic != kBlobMagic || h->version != kBlobVersion) return false;
   if (h->F != F || h->C != C || h->K != K || h->dtype != dtype || h->n_keep != n_keep) return false;
@@ -427,7 +509,8 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   }
   count_launches(4);
   if (L.nblk > 0) {
-    launch_dependent(k_pack_blocks, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
+    if (dtype == PAT_F16) launch_dependent(k_pack_blocks, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
+    else launch_dependent(k_pack_blocks_f32, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_pack launch");

@@ -51,7 +51,9 @@ def test_sizes_are_pure_functions(lib):
     # workspace path: stage images (28 regions x 16 channel blocks x 73728 bytes) + 256 partial tiles of cut items
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 1) == 28 * 16 * 73728 + 256 * 32 * 56 * 32 * 4
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 20, 14, 1) == 0
-    assert lib.pat_conv3x3_workspace(256, 256, 0, 16, 56, 56, 1) == 0
+    # fp32: stages of 8 channels, so twice the stage images
+    assert lib.pat_conv3x3_workspace(256, 256, 0, 16, 56, 56, 1) == 28 * 32 * 73728 + 256 * 32 * 56 * 32 * 4
+    assert lib.pat_conv3x3_workspace(256, 256, 0, 16, 56, 56, 2) == 0
     assert lib.pat_conv3x3_workspace(256, 256, 1, 16, 56, 56, 2) == 0
     assert lib.pat_conv3x3_workspace(256, 250, 1, 16, 56, 56, 1) == 0
     off = (C.c_size_t * 5)()

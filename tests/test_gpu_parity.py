@@ -178,6 +178,54 @@ def test_conv_tuned_f16_matches_oracle(case, use_workspace):
     check_close(out, ref, "f16")
 
 
+@pytest.mark.parametrize("case", TUNED_CASES)
+def test_conv_workspace_f32_matches_oracle(case):
+    """The fp32 workspace kernels (stages of 8 channels, 32-byte operations, results written in two rounds) on the
+    shapes of the tuned fp16 cases: every output element against the oracle, within the fp32 tolerance."""
+    N, H, W, C, F, K, num, den = case
+    tile_rows = (H + 3) // 4
+    assert (pc.pat_conv3x3_workspace(F, C, "f32", N, H, W, 1) > 0) == (tile_rows == 4 or tile_rows >= 7)
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 1)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f32")
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, "f32"), x, 1)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f32")
+    y = torch.full((N, H, W, F), float("nan"), dtype=torch.float32, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f32", torch.from_numpy(x).cuda(), 1, y=y)
+    assert pc.pat_query_status() == 0
+    out = y.cpu().numpy()
+    assert np.isfinite(out).all()                                   # every output element was written
+    check_close(out, ref, "f32")
+
+
+def test_conv_workspace_f32_cut_items_and_arbitrary_library():
+    """fp32 workspace kernels with a remainder of work items (pieces + reduce kernel) and with masks outside the
+    built-in set (position-by-position code); sampled against the oracle, and against the generic kernel."""
+    N, H, W, C, F = 24, 56, 56, 32, 128
+    masks = np.array([0b000001111, 0b111100000, 0b101000101, 0x03A, 0x0D8, 0b100110001], dtype=np.uint16)
+    rng = np.random.default_rng(78)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f32")
+    n_keep = F * C // 4
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f32")
+    xt = torch.from_numpy(x).cuda()
+    y = torch.full((N, H, W, F), float("nan"), dtype=torch.float32, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, "f32", xt, 1, y=y)
+    assert pc.pat_query_status() == 0
+    assert bool(torch.isfinite(y).all())
+    coords = np.stack([rng.integers(0, N, 6000), rng.integers(0, H, 6000), rng.integers(0, W, 6000), rng.integers(0, F, 6000)], axis=1).astype(np.int32)
+    coords[:2000, 0] = rng.integers(20, 24, 2000)          # the last images belong to the cut items
+    ref = oracle.conv3x3_at(stored_weights(wm_o, "f32"), x, coords, 1)
+    out = y[coords[:, 0], coords[:, 1], coords[:, 2], coords[:, 3]].cpu().numpy()
+    check_close(out, ref, "f32")
+    y2 = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f32", xt, 1, use_workspace=False)
+    assert torch.allclose(y, y2, rtol=1e-4, atol=1e-5)
+
+
 def test_conv_workspace_entry_point_agrees_with_plain_entry_point():
     """pat_conv3x3_ws and pat_conv3x3 add the kernels of a filter in different orders: fp16 results agree to a
     rounding step; a caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
