@@ -152,12 +152,13 @@ int pat_unpack(const void *blob, int F, int C, const uint16_t *masks, int K, int
 int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                 int dtype, const void *x, void *y, int N, int H, int W, int stride, void *stream);
 
-/* The same convolution with a caller-supplied device workspace.  For the layer shapes it covers (fp16, stride 1,
- * C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k}, H even and >= 14) the
- * activations are first re-arranged, once per call, into the channel-planar tiles the multiply-add kernel
- * stages in shared memory; the kernel then needs no transposition of its own and runs a deeper pipeline.
- * pat_conv3x3_workspace returns the bytes needed (about 1.3 x the size of x), or 0 for a layer the workspace
- * path does not cover: pat_conv3x3_ws then behaves exactly like pat_conv3x3 and ignores the workspace.
+/* The same convolution with a caller-supplied device workspace.  For the layer shapes it covers (fp16 or fp32,
+ * stride 1, C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k}, ceil(H/4) == 4 or >= 7)
+ * the activations are first re-arranged, once per call, into the channel-planar tiles the multiply-add kernel stages in
+ * shared memory; the kernel then needs no transposition of its own and runs a deeper pipeline.
+ * pat_conv3x3_workspace returns the bytes needed (about 1.3 x the size of x, plus 59 MB for partial sums), or 0 for a
+ * layer the workspace path does not cover: pat_conv3x3_ws then behaves exactly like pat_conv3x3 and ignores the
+ * workspace.
  *   workspace  dev, at least pat_conv3x3_workspace(...) bytes, 256-byte aligned; contents are scratch;
  *              concurrent calls must use different workspaces
  * Results: the same products as pat_conv3x3, added in fp32 in a different order of the kernels of a filter. */
