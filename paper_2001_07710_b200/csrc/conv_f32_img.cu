@@ -625,8 +625,21 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     }
     attr_set = true;
   }
-  const int grid = std::min(p.n_items, sm_count);
-  const int left = p.n_items % grid;
+  int grid = std::min(p.n_items, sm_count);
+  // fewer work items than half the SMs (small batches): every item is cut along the input channels, so that up to
+  // eight blocks share an item; their partial sums are added by the reduce kernel
+  if (2 * p.n_items <= sm_count) {
+    // a piece keeps at least 32 input channels - below that its partial sums cost more than the idle SMs - unless
+    // the items are so few (a single small image) that the partial sums are a few megabytes in all
+    const int min_channels = p.n_items <= 8 ? CBI : 32;
+    const int parts = std::min(std::min(MAX_PARTS, C / min_channels), std::min(sm_count, MAX_PIECES) / p.n_items);
+    if (parts >= 3) {
+      p.n_whole = 0; p.n_split = p.n_items; p.parts = parts;
+      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nst * IMG_BYTES));
+      grid = p.n_items * parts;
+    }
+  }
+  const int left = p.parts > 1 ? 0 : p.n_items % grid;
   if (left > 0) {
     const int parts = std::min(std::min(MAX_PARTS, p.nst), std::min(grid, MAX_PIECES) / left);
     if (parts >= 2) {
