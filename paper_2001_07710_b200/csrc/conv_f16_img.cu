@@ -433,7 +433,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           for (int y = 0; y < TR4; ++y)
 #pragma unroll
             for (int part = 0; part < 2; ++part)
-              if ((part == 0 || lane < 4 * (TC - 8)) && TR4 * ty + y < p.H)
+              if ((part == 0 || lane < 4 * (TC - 8)) && TR4 * ty + y < p.H && col0 + (lane >> 2) + 8 * part < p.W)
                 *reinterpret_cast<uint4*>(dst + ((size_t)y * p.W + 8 * part) * p.F) = v[y][part];
         }
       }
@@ -525,7 +525,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || TR4 * ty + y >= p.H) return;
   const int col0 = (it.cg * p.TXe + tx) * TC;
   __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
-  if (lane < RP_XH * 4) {
+  if (lane < RP_XH * 4 && col0 + xh * RP_XH + (lane >> 2) < p.W) {
     const int x = xh * RP_XH + (lane >> 2), j = lane & 3;
     const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + x) * OUT_PITCH + j * 16);
     *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
@@ -536,8 +536,8 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
   p.nct = C / CBI;
-  p.TY = (H + TR4 - 1) / TR4;   // a last, partly empty tile row when H is not a multiple of 4
-  const int TX = W / TC;
+  p.TY = std::max((H + TR4 - 1) / TR4, LY / 2);   // a last, partly empty tile row when H is not a multiple of 4; small images take four tile rows
+  const int TX = W < TC ? 1 : W / TC;                // an image narrower than a thread tile takes one tile column
   p.TXe = TX >= LX ? LX : TX;
   p.NI = LX / p.TXe;
   p.CG = TX / p.TXe;
@@ -559,9 +559,9 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
   if (dtype != PAT_F16 || stride != 1) return false;
-  const int TY = (H + TR4 - 1) / TR4;
-  if (W % TC != 0 || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
-  const int TX = W / TC;
+  const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
+  if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
+  const int TX = W < TC ? 1 : W / TC;
   if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
   if (C % kChanTile != 0 || F % FG != 0) return false;
   Params p;

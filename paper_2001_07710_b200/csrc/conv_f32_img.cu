@@ -467,7 +467,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
               }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              if (4 * i + (lane >> 3) < TC && row < p.H)
+              if (4 * i + (lane >> 3) < TC && row < p.H && col0 + 4 * i + (lane >> 3) < p.W)
                 *reinterpret_cast<uint4*>(dst + (size_t)(4 * i) * p.F) = v[i];
           }
         }
@@ -534,7 +534,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
   const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
   const int n_img = ig * p.NI + ni;
   const int row = TR4 * ty + v / TC, col = (it.cg * p.TXe + tx) * TC + v % TC;
-  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H) return;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H || col >= p.W) return;
   p.y[(((size_t)n_img * p.H + row) * p.W + col) * p.F + __ldg(p.xfilt + g * FG + slot)] = sum;
 }
 
@@ -542,8 +542,8 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
   p.nst = C / CBI;
-  p.TY = (H + TR4 - 1) / TR4;
-  const int TX = W / TC;
+  p.TY = std::max((H + TR4 - 1) / TR4, LY / 2);   // a last, partly empty tile row when H is not a multiple of 4; small images take four tile rows
+  const int TX = W < TC ? 1 : W / TC;                // an image narrower than a thread tile takes one tile column
   p.TXe = TX >= LX ? LX : TX;
   p.NI = LX / p.TXe;
   p.CG = TX / p.TXe;
@@ -565,9 +565,9 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 bool conv_f32_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img32;
   if (dtype != PAT_F32 || stride != 1) return false;
-  const int TY = (H + TR4 - 1) / TR4;
-  if (W % TC != 0 || !(TY >= LY - 1 || 2 * TY == LY)) return false;
-  const int TX = W / TC;
+  const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
+  if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
+  const int TX = W < TC ? 1 : W / TC;
   if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
   if (C % kChanTile != 0 || F % FG != 0) return false;
   Params p;

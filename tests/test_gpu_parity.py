@@ -226,6 +226,34 @@ def test_conv_workspace_f32_cut_items_and_arbitrary_library():
     assert torch.allclose(y, y2, rtol=1e-4, atol=1e-5)
 
 
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+@pytest.mark.parametrize("case", [(9, 7, 7, 32, 64, 8, 1, 4), (5, 12, 10, 16, 32, 12, 1, 2), (3, 3, 14, 32, 32, 8, 1, 1), (6, 16, 5, 16, 32, 4, 1, 2)])
+def test_conv_workspace_small_images(case, dtype):
+    """Images smaller than a thread tile (fewer than 14 columns) or than four tile rows (fewer than 13 rows) take a
+    whole tile column / four tile rows of the workspace kernels; the pixels outside the image are neither read nor written."""
+    N, H, W, C, F, K, num, den = case
+    assert pc.pat_conv3x3_workspace(F, C, dtype, N, H, W, 1) > 0
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 7)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, dtype), x, 1)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    # the output sits inside a larger buffer filled with a marker: nothing outside it may be written
+    buf = torch.full((N * H * W * F + 4096,), 7.0, dtype=tdt, device="cuda")
+    y = buf[2048:2048 + N * H * W * F].view(N, H, W, F)
+    y.fill_(float("nan"))
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, torch.from_numpy(x).cuda(), 1, y=y)
+    assert pc.pat_query_status() == 0
+    out = y.float().cpu().numpy()
+    assert np.isfinite(out).all()
+    check_close(out, ref, dtype)
+    assert bool((buf[:2048] == 7.0).all()) and bool((buf[2048 + N * H * W * F:] == 7.0).all())
+
+
 def test_conv_workspace_entry_point_agrees_with_plain_entry_point():
     """pat_conv3x3_ws and pat_conv3x3 add the kernels of a filter in different orders: fp16 results agree to a
     rounding step; a caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
