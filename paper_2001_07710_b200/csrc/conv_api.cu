@@ -10,10 +10,10 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride);
 size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st);
+                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
 size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st);
+                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
 }
 
 using namespace pat;
@@ -57,6 +57,6 @@ extern "C" int pat_conv3x3_ws(const void* blob, int F, int C, const uint16_t* ma
   if (!workspace || workspace_bytes < need)
     return set_error(PAT_ERR_WORKSPACE, "pat_conv3x3_ws: workspace has %zu bytes, needs %zu", workspace_bytes, need);
   if (!aligned(workspace, 256)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3_ws: workspace must be 256-byte aligned");
-  if (dtype == PAT_F32) return conv_f32_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, workspace, reinterpret_cast<cudaStream_t>(stream));
-  return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, workspace, reinterpret_cast<cudaStream_t>(stream));
+  if (dtype == PAT_F32) return conv_f32_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, workspace, reinterpret_cast<cudaStream_t>(stream));
+  return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, workspace, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -60,6 +60,7 @@ struct Params {
   const BlobHeader* hdr;
   int* status;
   int N, H, W, C, F, K, nct;  // nct = channel blocks of 16
+  int Ho, Wo, sub;            // output size; sub = stride - 1: with stride 2 only the results at even rows and columns are written
   long long n_keep;
   int TY;                  // tile rows per image (ceil(H / 4))
   int TXe, NI;             // tile columns per region, images side by side
@@ -418,7 +419,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           const int n_img = ig * p.NI + ni;
           if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
           const int col0 = (it.cg * p.TXe + tx) * TC;
-          __half* dst = p.y + (((size_t)n_img * p.H + TR4 * ty) * p.W + col0 + (lane >> 2)) * p.F + g_out * FG + (lane & 3) * 8;
+          const int row0 = TR4 * ty, colp = col0 + (lane >> 2);
+          __half* dst = p.y + (size_t)n_img * p.Ho * p.Wo * p.F + g_out * FG + (lane & 3) * 8;
           const uint32_t src = sl + (uint32_t)(t * TC) * OUT_PITCH + (uint32_t)(t >> 4) * 4u;
           uint4 v[TR4][2];
 #pragma unroll
@@ -433,8 +435,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           for (int y = 0; y < TR4; ++y)
 #pragma unroll
             for (int part = 0; part < 2; ++part)
-              if ((part == 0 || lane < 4 * (TC - 8)) && TR4 * ty + y < p.H && col0 + (lane >> 2) + 8 * part < p.W)
-                *reinterpret_cast<uint4*>(dst + ((size_t)y * p.W + 8 * part) * p.F) = v[y][part];
+              if ((part == 0 || lane < 4 * (TC - 8)) && row0 + y < p.H && colp + 8 * part < p.W && (((row0 + y) | (colp + 8 * part)) & p.sub) == 0)
+                *reinterpret_cast<uint4*>(dst + ((size_t)((row0 + y) >> p.sub) * p.Wo + ((colp + 8 * part) >> p.sub)) * p.F) = v[y][part];
         }
       }
       // the slots are refilled by bulk copies next: order this warp's reads of them before those writes
@@ -524,11 +526,13 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   const int n_img = ig * p.NI + ni;
   if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || TR4 * ty + y >= p.H) return;
   const int col0 = (it.cg * p.TXe + tx) * TC;
-  __half* dst_tile = p.y + (((size_t)n_img * p.H + (TR4 * ty + y)) * p.W + col0) * p.F + g * FG;
+  const int row = TR4 * ty + y;
   if (lane < RP_XH * 4 && col0 + xh * RP_XH + (lane >> 2) < p.W) {
     const int x = xh * RP_XH + (lane >> 2), j = lane & 3;
+    if (((row | (col0 + x)) & p.sub) != 0) return;           // stride 2: even rows and columns only
     const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + x) * OUT_PITCH + j * 16);
-    *reinterpret_cast<uint4*>(dst_tile + (size_t)x * p.F + j * 8) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+    __half* dst = p.y + (((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo + ((col0 + x) >> p.sub)) * p.F + g * FG + j * 8;
+    *reinterpret_cast<uint4*>(dst) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
   }
 }
 
@@ -558,7 +562,7 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 // True when the stage-image kernels cover this layer.
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
-  if (dtype != PAT_F16 || stride != 1) return false;
+  if (dtype != PAT_F16 || (stride != 1 && stride != 2)) return false;   // stride 2: computed like stride 1, one result in four written
   const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
   if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
   const int TX = W < TC ? 1 : W / TC;
@@ -578,7 +582,7 @@ size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
 }
 
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st) {
+                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st) {
   using namespace img16;
   const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F16);
   const char* b = static_cast<const char*>(blob);
@@ -594,6 +598,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.status = status_word();
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
+  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   // the smallest set of compiled pattern codes that covers the library

@@ -51,6 +51,7 @@ struct Params {
   const BlobHeader* hdr;
   int* status;
   int N, H, W, C, F, K, nst;  // nst = stages of 8 channels
+  int Ho, Wo, sub;            // output size; sub = stride - 1: with stride 2 only the results at even rows and columns are written
   long long n_keep;
   int TY, TXe, NI, CG, NIG, NG;
   int n_regions, n_items;
@@ -457,7 +458,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 #pragma unroll
           for (int yy = 0; yy < 2; ++yy) {
             const int row = TR4 * ty + 2 * round + yy;
-            float* dst = p.y + (((size_t)n_img * p.H + row) * p.W + col0 + (lane >> 3)) * p.F + g_out * FG + (lane & 7) * 4;
+            const int colp = col0 + (lane >> 3);
+            float* dst = p.y + ((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo * p.F + g_out * FG + (lane & 7) * 4;
             uint4 v[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -467,8 +469,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
               }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              if (4 * i + (lane >> 3) < TC && row < p.H && col0 + 4 * i + (lane >> 3) < p.W)
-                *reinterpret_cast<uint4*>(dst + (size_t)(4 * i) * p.F) = v[i];
+              if (4 * i + (lane >> 3) < TC && row < p.H && colp + 4 * i < p.W && ((row | (colp + 4 * i)) & p.sub) == 0)
+                *reinterpret_cast<uint4*>(dst + (size_t)((colp + 4 * i) >> p.sub) * p.F) = v[i];
           }
         }
         if (round == 0) {
@@ -534,8 +536,8 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
   const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
   const int n_img = ig * p.NI + ni;
   const int row = TR4 * ty + v / TC, col = (it.cg * p.TXe + tx) * TC + v % TC;
-  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H || col >= p.W) return;
-  p.y[(((size_t)n_img * p.H + row) * p.W + col) * p.F + __ldg(p.xfilt + g * FG + slot)] = sum;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H || col >= p.W || ((row | col) & p.sub) != 0) return;
+  p.y[(((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo + (col >> p.sub)) * p.F + __ldg(p.xfilt + g * FG + slot)] = sum;
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -564,7 +566,7 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 // True when the fp32 stage-image kernels cover this layer.
 bool conv_f32_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img32;
-  if (dtype != PAT_F32 || stride != 1) return false;
+  if (dtype != PAT_F32 || (stride != 1 && stride != 2)) return false;   // stride 2: computed like stride 1, one result in four written
   const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
   if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
   const int TX = W < TC ? 1 : W / TC;
@@ -583,7 +585,7 @@ size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
 }
 
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, void* workspace, cudaStream_t st) {
+                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st) {
   using namespace img32;
   const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F32);
   const char* b = static_cast<const char*>(blob);
@@ -599,6 +601,7 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.status = status_word();
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
+  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   int variant = 0;

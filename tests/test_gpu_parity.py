@@ -254,6 +254,30 @@ def test_conv_workspace_small_images(case, dtype):
     assert bool((buf[:2048] == 7.0).all()) and bool((buf[2048 + N * H * W * F:] == 7.0).all())
 
 
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+@pytest.mark.parametrize("case", [(3, 56, 56, 32, 64, 8, 1, 4), (5, 14, 14, 64, 32, 8, 1, 2), (2, 28, 28, 16, 32, 12, 1, 1), (4, 7, 7, 32, 32, 8, 1, 4),
+                                  (24, 28, 56, 64, 64, 8, 1, 8)])
+def test_conv_workspace_stride2(case, dtype):
+    """Stride 2 on the workspace kernels (computed like stride 1; the results at even rows and columns are written),
+    odd and even sizes, cut items included: every output element against the oracle."""
+    N, H, W, C, F, K, num, den = case
+    assert pc.pat_conv3x3_workspace(F, C, dtype, N, H, W, 2) > 0
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 11)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.conv3x3(stored_weights(wm_o, dtype), x, 2)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, torch.from_numpy(x).cuda(), 2)
+    assert pc.pat_query_status() == 0
+    assert tuple(y.shape) == ref.shape
+    out = y.float().cpu().numpy()
+    assert np.isfinite(out).all()
+    check_close(out, ref, dtype)
+
+
 def test_conv_workspace_entry_point_agrees_with_plain_entry_point():
     """pat_conv3x3_ws and pat_conv3x3 add the kernels of a filter in different orders: fp16 results agree to a
     rounding step; a caller-owned workspace full of NaN bit patterns is overwritten before it is read."""
