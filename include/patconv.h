@@ -153,9 +153,10 @@ int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, in
                 int dtype, const void *x, void *y, int N, int H, int W, int stride, void *stream);
 
 /* The same convolution with a caller-supplied device workspace.  For the layer shapes it covers (fp16 or fp32,
- * stride 1, C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k}, ceil(H/4) == 4 or >= 7)
- * the activations are first re-arranged, once per call, into the channel-planar tiles the multiply-add kernel stages in
- * shared memory; the kernel then needs no transposition of its own and runs a deeper pipeline.
+ * stride 1 or 2, C a multiple of 16, F a multiple of 32, W a multiple of 14 with W/14 in {1, 2, 4k} or W < 14,
+ * max(ceil(H/4), 4) == 4 or >= 7) the activations are first re-arranged, once per call, into the channel-planar tiles
+ * the multiply-add kernel stages in shared memory; the kernel then needs no transposition of its own and runs a deeper
+ * pipeline.  Stride 2 is computed like stride 1 and the results at even rows and columns are written.
  * pat_conv3x3_workspace returns the bytes needed (about 1.3 x the size of x, plus 59 MB for partial sums), or 0 for a
  * layer the workspace path does not cover: pat_conv3x3_ws then behaves exactly like pat_conv3x3 and ignores the
  * workspace.
