@@ -173,18 +173,36 @@ def run_ours(args):
         if overlap:
             main.wait_stream(side)
 
+    # End to end: every step copies its weights and inputs from pinned host memory and reads all outputs back.  The
+    # copies run on streams of their own (host-to-device, device-to-host: the link is full duplex) and overlap the
+    # compute stream layer by layer; events order copy-in -> compute -> copy-out per layer, and a step begins only
+    # when the previous step's kernels no longer read the device buffers it overwrites.
+    h2d, d2h = torch.cuda.Stream(), torch.cuda.Stream()
+    in_ev = [torch.cuda.Event() for _ in layers]
+    out_ev = [torch.cuda.Event() for _ in layers]
+
     def step_e2e():
-        for st in layers:
+        main = torch.cuda.current_stream()
+        h2d.wait_stream(main)                      # the previous step has consumed w and x
+        with torch.cuda.stream(h2d):
+            for i, st in enumerate(layers):
+                st["w"].copy_(st["hw"], non_blocking=True)
+                st["x"].copy_(st["hx"], non_blocking=True)
+                in_ev[i].record(h2d)
+        for i, st in enumerate(layers):
             L = st["L"]
-            st["w"].copy_(st["hw"], non_blocking=True)
-            st["x"].copy_(st["hx"], non_blocking=True)
+            main.wait_event(in_ev[i])
             if L.dense:
                 pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
             else:
                 pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
                 pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
                 pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
-            st["hy"].copy_(st["y"], non_blocking=True)
+            out_ev[i].record(main)
+            with torch.cuda.stream(d2h):
+                d2h.wait_event(out_ev[i])
+                st["hy"].copy_(st["y"], non_blocking=True)
+        main.wait_stream(d2h)                      # the results are on the host before the step counts as done
 
     def barrier():
         torch.cuda.synchronize()
