@@ -151,7 +151,8 @@ __device__ __forceinline__ void lds_row_f32(float (&h)[16], uint32_t a, uint32_t
 // window row `sh`, swb = the lane's chunk swizzle (bits 4-5) for window rows 0-3; from window row 4 on the rows
 // belong to the next tile row's group, whose parity bit is the other one.
 template <uint32_t MASK>
-__device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a0, uint32_t sh, uint32_t swb, const float (&w)[4]) {
+__device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a0, uint32_t sh, uint32_t swb, const float (&w)[4],
+                                               const float (&r0)[16]) {
   constexpr int NR = last_tap_row(MASK) + TR4;
 #pragma unroll
   for (int j = 0; j < NR; ++j) {
@@ -159,7 +160,12 @@ __device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a
     if (j >= 4) x ^= 32u;
     else if (j == 3) x ^= sh << 5;
     float h[16];
-    lds_row_f32(h, a0 + j * ROWF, x);
+    if (j == 0) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) h[i] = r0[i];       // loaded by the caller before it branched here
+    } else {
+      lds_row_f32(h, a0 + j * ROWF, x);
+    }
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const int b = nth_bit(MASK, t);
@@ -174,7 +180,7 @@ __device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a
 
 template <int NCODES, bool GENERIC>
 __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t plane, uint32_t swb, uint32_t meta, uint32_t off,
-                                             float (&w)[4]) {
+                                             float (&w)[4], const float (&r0)[16]) {
   static_assert(NCODES == 6 || NCODES == kNumCodes, "code sets with compiled dispatch trees");
   const uint32_t sh = (meta >> 17) & 1u;
   const uint32_t a0 = plane + off;
@@ -200,26 +206,26 @@ __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t pla
 #undef PAT_TAP4F
       }
     } else if constexpr (NCODES > 8) {
-      if (code & 1u) pattern_body4f<code_mask(9)>(acc, a0, sh, swb, w);
-      else pattern_body4f<code_mask(8)>(acc, a0, sh, swb, w);
+      if (code & 1u) pattern_body4f<code_mask(9)>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(8)>(acc, a0, sh, swb, w, r0);
     }
   } else if (code & 4u) {
     if (NCODES > 6 && (code & 2u)) {
       if constexpr (NCODES > 6) {
-        if (code & 1u) pattern_body4f<code_mask(7)>(acc, a0, sh, swb, w);
-        else pattern_body4f<code_mask(6)>(acc, a0, sh, swb, w);
+        if (code & 1u) pattern_body4f<code_mask(7)>(acc, a0, sh, swb, w, r0);
+        else pattern_body4f<code_mask(6)>(acc, a0, sh, swb, w, r0);
       }
     } else {
-      if (code & 1u) pattern_body4f<code_mask(5)>(acc, a0, sh, swb, w);
-      else pattern_body4f<code_mask(4)>(acc, a0, sh, swb, w);
+      if (code & 1u) pattern_body4f<code_mask(5)>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(4)>(acc, a0, sh, swb, w, r0);
     }
   } else {
     if (code & 2u) {
-      if (code & 1u) pattern_body4f<code_mask(3)>(acc, a0, sh, swb, w);
-      else pattern_body4f<code_mask(2)>(acc, a0, sh, swb, w);
+      if (code & 1u) pattern_body4f<code_mask(3)>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(2)>(acc, a0, sh, swb, w, r0);
     } else {
-      if (code & 1u) pattern_body4f<code_mask(1)>(acc, a0, sh, swb, w);
-      else pattern_body4f<code_mask(0)>(acc, a0, sh, swb, w);
+      if (code & 1u) pattern_body4f<code_mask(1)>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(0)>(acc, a0, sh, swb, w, r0);
     }
   }
 }
@@ -364,6 +370,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       for (;;) {
         const uint32_t cm = m0, coff = off;
         float w[4] = {__uint_as_float(w0), __uint_as_float(w1), __uint_as_float(w2), __uint_as_float(w3)};
+        float r0[16];                      // the first window row of this kernel (window rows 0-3 share the lane's swizzle)
+        lds_row_f32(r0, pl0 + coff, swb);
         e += OPB;
         lds128(e, m0, off, w0, w1);        // the next operation
         lds128(e + 16u, w2, w3, pad0, pad1);
@@ -373,7 +381,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           cur ^= 1u;
           fetch(cur, acc);
         }
-        one_kernel4f<NCODES, GENERIC>(acc, pl0, swb, cm, coff, w);
+        one_kernel4f<NCODES, GENERIC>(acc, pl0, swb, cm, coff, w, r0);
       stage_end:
         if (cm & kOpEnd) {
           __syncwarp();
