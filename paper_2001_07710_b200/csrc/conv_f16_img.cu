@@ -1,9 +1,10 @@
-// Sparse 3x3 convolution for fp16 storage / fp32 accumulation, stride 1 (sm_100a): two kernels.
+// Sparse 3x3 convolution for fp16 storage / fp32 accumulation (sm_100a): three kernels.  Stride 2 is computed like
+// stride 1 and only the results at even rows and columns are written.
 //
 //  1. k_stage_images re-arranges the NHWC activations once per call into "stage images": for every region
-//     (8 tile rows x 4 column slots of 4 x 14 pixel tiles) and every block of 8 input channels one contiguous
-//     36 KB piece laid out exactly as the convolution kernel wants it in shared memory - channel-planar
-//     [8 ch][36 rows][4 segments][16 px], halo pixels duplicated, zero padding written out, the two 16-byte chunks
+//     (8 tile rows x 4 column slots of 4 x 14 pixel tiles) and every block of 16 input channels one contiguous
+//     72 KB piece laid out exactly as the convolution kernel wants it in shared memory - channel-planar
+//     [16 ch][36 rows][4 segments][16 px], halo pixels duplicated, zero padding written out, the two 16-byte chunks
 //     of a segment trading places from one tile row to the next so that the 16-byte window loads of a warp touch
 //     every bank once.  This is plain streaming work (reads the input once, writes 1.3 x its size) and it is done
 //     once per region, whereas a kernel that transposes inside its pipeline repeats it for every group of 32 filters.

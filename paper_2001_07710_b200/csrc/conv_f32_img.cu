@@ -1,5 +1,5 @@
-// Sparse 3x3 convolution for fp32 storage and accumulation, stride 1 (sm_100a): the workspace path of conv_f16_img.cu
-// for 4-byte activations.  The same three kernels and the same protocol (stage images built once per call, a
+// Sparse 3x3 convolution for fp32 storage and accumulation (sm_100a): the workspace path of conv_f16_img.cu for
+// 4-byte activations (stride 2 likewise: computed like stride 1, the results at even rows and columns written).  The same three kernels and the same protocol (stage images built once per call, a
 // persistent warp-specialised kernel fed by bulk copies through a ring of shared-memory slots, flat pack-time
 // operation lists, one accumulator tile in registers and one parked in tensor memory, cut items reduced by a third
 // kernel); what differs:
