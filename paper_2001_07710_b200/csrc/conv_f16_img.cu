@@ -10,15 +10,16 @@
 //     once per region, whereas a kernel that transposes inside its pipeline repeats it for every group of 32 filters.
 //  2. k_conv_f16_img is the persistent, warp-specialised convolution kernel (one block per SM).  A work item is one
 //     region x one group of 32 filters.  One producer thread streams the item's stage images and the matching
-//     kernel-descriptor blocks of the packed weights (both contiguous, one bulk copy each per stage) into a ring of
-//     5 shared-memory slots; 16 consumer warps (two filters each, 4 x 14 pixels per thread, one accumulator tile of
-//     56 values in registers and the other parked in tensor memory) run the per-pattern multiply-add code
-//     (Section 6.2); results leave through four extra ring stages per item and a store warp, as 64-byte runs of
-//     NHWC output.  The tall thread tile is what the multiply-add rate hangs on: a kernel costs about the same
-//     number of other instructions (descriptor, addresses, branch) and 1.5 x the window loads of a 2 x 14 tile
-//     for twice the multiply-adds.  With nothing but two bulk copies per stage on the producer side the ring is
-//     deep, and the consumer warps, whose per-stage work differs (about one kernel per filter and channel block at
-//     12.5 % density), seldom wait for each other.  Every wait is bounded; tensor memory is released on every path.
+//     descriptor blocks of the packed weights (both contiguous, one bulk copy each per stage) into a ring of three
+//     shared-memory slots (two when the blob is dense); 16 consumer warps (two filters each, 4 x 14 pixels per
+//     thread, one accumulator tile of 56 values in registers and the other parked in tensor memory) run the
+//     per-pattern multiply-add code (Section 6.2) over flat operation lists written at pack time; the results leave
+//     through two extra ring stages per item: the consumer warps stage them as [pixel][32 channels] and copy them
+//     out as 64-byte runs of NHWC output.  The tall thread tile is what the multiply-add rate hangs on: a kernel
+//     costs about the same number of other instructions (descriptor, addresses, branch) and 1.5 x the window loads
+//     of a 2 x 14 tile for twice the multiply-adds.  Every wait is bounded; tensor memory is released on every path.
+//  3. k_reduce_parts adds, in a fixed order, the fp32 partial sums of work items that were cut along the input
+//     channels (the items of a last, mostly idle round; every item when there are fewer items than half the SMs).
 #include <algorithm>
 #include "f16_tile.cuh"
 
