@@ -180,8 +180,9 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
 //                  copy two thread tiles each to global memory and arrive slot_empty of both slots.
 //                  (A separate store warp shares the issue slots of its SM partition with four consumer warps and
 //                  needed longer for a slot than the consumers for two stages: the ring stood still meanwhile.)
-// In a real stage a consumer warp runs filter A, swaps, runs filter B; the next stage starts with B.  A tile of
-// 56 accumulators is moved to / from tensor memory once per stage and filter.
+// In a real stage a consumer warp runs the operations of its list in the stage's descriptor block: the kernels of the
+// filter whose tile it holds, a swap of the two accumulator tiles through tensor memory if its other filter has
+// kernels in this stage, and those kernels; the next stage starts with the tile it then holds.
 template <bool SPARSE, int NCODES, bool GENERIC>
 __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
   constexpr int NS = SPARSE ? 3 : 2;
