@@ -32,9 +32,65 @@ UNIT = "images/s"
 SM_COUNT, FMA_LANES, SM_MAX_MHZ = 148, 128, 1965.0
 FMA_PEAK_TFLOPS = 2 * FMA_LANES * SM_COUNT * SM_MAX_MHZ * 1e6 / 1e12     # 74.45: fp32 FMA, no tensor cores
 DEFAULT_CONFIG = 3
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_conv_f16_img launch (conv6 shape, batch 32), from
-# profiles/k_conv_f16_img_conv6_b32.md
-CONV6_DRAM_BYTES_B32 = 67.53e6 + 17.12e6
+# DRAM traffic of the convolution path (ncu counters of a small case), written by `bench.py --write-traffic` and
+# valid only for the kernel sources it was captured from
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_conv_f16_img_conv6_b32.json")
+TRAFFIC_SOURCES = ["conv_f16_img.cu", "f16_tile.cuh", "common.cuh"]
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2001_07710_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def write_traffic(csv_path: str):
+    """Turns an ncu launch list with dram__bytes_read.sum / dram__bytes_write.sum of the three launches of the conv6
+    path (batch 32) into TRAFFIC_FILE.  The bytes the path wrote but that were still in L2 when a launch ended are
+    added from what the launches are known to write (stage images, outputs)."""
+    import csv
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    rows = [r for r in csv.reader(open(csv_path)) if len(r) > 5]
+    hdr = rows[0]
+    ki, mi, ui, vi = hdr.index("Kernel Name"), hdr.index("Metric Name"), hdr.index("Metric Unit"), hdr.index("Metric Value")
+    kernels = {}
+    for r in rows[1:]:
+        name = "stage" if "k_stage_images" in r[ki] else "conv" if "k_conv_f16_img" in r[ki] else "reduce" if "k_reduce_parts" in r[ki] else None
+        if name is None or not r[mi].startswith("dram__bytes_"):
+            continue
+        key = "read" if "read" in r[mi] else "write"
+        kernels.setdefault(name, {})[key] = float(r[vi].replace(",", "")) * unit[r[ui]]
+    cfg = workloads.configs()[3]
+    L = [l for l in cfg.layers if l.name == "conv6"][0]
+    from paper_2001_07710_b200 import binding
+    lib = binding.load()
+    images = lib.pat_conv3x3_workspace(L.F, L.C, 1, 32, L.H, L.W, 1) - 256 * 32 * 56 * 32 * 4     # stage images without the partial tiles
+    known_writes = images + 32 * L.Ho * L.Wo * L.F * 2
+    pending = max(0.0, known_writes - sum(k.get("write", 0.0) for k in kernels.values()))
+    out = {"workload": "config 3 layer conv6 (56x56x256 -> 256, keep 12.5 %), fp16 storage, batch 32",
+           "source_sha16": kernel_source_hash(), "sources": TRAFFIC_SOURCES, "batch": 32, "kernels": kernels,
+           "written_still_in_l2": pending, "algorithmic_bytes": L.compulsory_bytes(32, 2)}
+    json.dump(out, open(TRAFFIC_FILE, "w"), indent=1)
+    print(json.dumps(out))
+
+
+def traffic_field(N: int, cfg_no: int):
+    """roofline.traffic for the benchmark's batch, or None when the counters do not belong to the current kernels."""
+    if cfg_no != 3 or not os.path.exists(TRAFFIC_FILE):
+        return None, "no counters for this workload"
+    t = json.load(open(TRAFFIC_FILE))
+    if t.get("source_sha16") != kernel_source_hash():
+        return None, "the kernel sources changed since the counters in %s were taken" % os.path.basename(TRAFFIC_FILE)
+    scale = N / float(t["batch"])
+    dram = sum(k.get("read", 0.0) + k.get("write", 0.0) for k in t["kernels"].values()) + t.get("written_still_in_l2", 0.0)
+    note = ("DRAM read + write of the three launches of one layer's path (stage images, convolution, reduce) on %s "
+            "(ncu), plus the %.1f MB the launches wrote that were still in L2 when they ended, scaled by batch/%d; "
+            "algorithmic bytes of that layer at this batch: %d (traffic / algorithmic = %.2f)"
+            % (t["workload"], t.get("written_still_in_l2", 0.0) / 1e6, t["batch"], int(t["algorithmic_bytes"] * scale),
+               dram / t["algorithmic_bytes"]))
+    return dram * scale, note
 
 
 def measured_peaks():
@@ -105,6 +161,7 @@ def run_ours(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")     # the communicator's own log (rings, NVLS) goes to stderr
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     pc.load()
 
@@ -278,6 +335,8 @@ def run_ours(args):
     assert pc.pat_query_status() == 0
 
     # ---- roofline of the dominant kernel (the sparse convolution), and per layer
+    traffic, traffic_note = traffic_field(N, cfg.number)
+    fma_measured = pc.pat_measure_fma_peak(1 if dtype == "f16" else 0)
     peaks, peak_kind = measured_peaks()
     hbm = peaks["hbm_gbs"]
     per_layer = []
@@ -311,14 +370,12 @@ def run_ours(args):
                    "l2": l2_note, "seed": workloads.BASE_SEED},
         "effective_gflops": round(total_flop * world * args.steps / (ms_total * 1e-3) / 1e9, 1),
         "conv_only_images_per_s": round(world * N / (sum(conv_ms) * 1e-3), 2),
-        "roofline": {"bound": "alu", "kernel": "sparse convolution path of the 12 pruned layers (stage images + convolution + reduce launches)", "achieved": round(achieved, 3),
+        "roofline": {"bound": "alu", "kernel": "sparse convolution path of the pruned layers (stage images + convolution + reduce launches)", "achieved": round(achieved, 3),
                      "peak": round(FMA_PEAK_TFLOPS, 2), "unit": "TFLOP/s", "frac": round(achieved / FMA_PEAK_TFLOPS, 4),
                      "peak_kind": "derived: 2 x 128 fp32 lanes x 148 SMs x 1.965 GHz",
-                     "traffic": CONV6_DRAM_BYTES_B32 * (N / 32.0) if cfg.number == 3 else None,
-                     "traffic_note": ("DRAM read+write bytes of one k_conv_f16_img launch on the conv6 shape (ncu, batch 32, "
-                                      "scaled by batch/32; part of the output was still in L2 when the captured launch ended); "
-                                      "algorithmic bytes of that layer: %d" % cfg.layers[5].compulsory_bytes(N, elem))
-                                     if cfg.number == 3 else None,
+                     "traffic": traffic, "traffic_note": traffic_note,
+                     "peak_measured": round(fma_measured, 2),
+                     "peak_measured_kind": "fma.rn.f32.f16 chains on all SMs, best of three, this run (pat_measure_fma_peak)",
                      "hbm_peak_gbs": hbm, "hbm_peak_kind": peak_kind,
                      "min_layer_frac": min([p["roof_frac"] for p in per_layer if p["layer"] != "conv1"] + [1.0])},
         "layers": per_layer,
@@ -327,12 +384,88 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if world == 1 and not args.no_other_configs and args.batch is None and args.layers is None:
+        # the other four configurations: short measurements of their own, after the main timed region
+        out["other_configs"] = {str(c): quick_config(pc, torch, c, peaks) for c in range(5) if c != cfg.number}
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_seconds)
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def quick_config(pc, torch, cfg_no: int, peaks, steps: int = 10):
+    """One of the other configurations: the same step (project + pack + convolution of every layer) on one stream,
+    `steps` times after three warm-up steps, CUDA events around the steps and around every convolution call."""
+    cfg = workloads.configs()[cfg_no]
+    N, dtype = cfg.N, cfg.dtype
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    elem = 2 if dtype == "f16" else 4
+    masks = {K: pc.pat_library_builtin(K) for K in (4, 8, 12)}
+    layers = []
+    for L in cfg.layers:
+        w_np, x_np = workloads.make_layer_tensors(cfg.number, L, N)
+        st = dict(L=L, w=torch.from_numpy(w_np).cuda(), x=torch.from_numpy(x_np).to(tdt).cuda(),
+                  y=torch.empty((N, L.Ho, L.Wo, L.F), dtype=tdt, device="cuda"))
+        if not L.dense:
+            st["pid"] = torch.empty((L.F, L.C), dtype=torch.uint8, device="cuda")
+            st["wm"] = torch.empty((L.F, L.C, 3, 3), dtype=torch.float32, device="cuda")
+            st["ws"] = torch.empty(pc.pat_project_workspace(L.F, L.C), dtype=torch.uint8, device="cuda")
+            st["blob"] = torch.empty(pc.pat_pack_size(L.F, L.C, L.K, L.n_keep, dtype), dtype=torch.uint8, device="cuda")
+        layers.append(st)
+    cws = torch.empty(max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg.layers if not L.dense] + [256]),
+                      dtype=torch.uint8, device="cuda")
+    main = torch.cuda.current_stream()
+
+    def step(ev=None):
+        for i, st in enumerate(layers):
+            L = st["L"]
+            if not L.dense:
+                pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
+                pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
+            if ev is not None: ev[i][0].record(main)
+            if L.dense:
+                pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
+            else:
+                pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
+            if ev is not None: ev[i][1].record(main)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(main)
+    for _ in range(steps):
+        step()
+    e1.record(main)
+    torch.cuda.synchronize()
+    ms_step = e0.elapsed_time(e1) / steps
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(3)]
+    for k in range(3):
+        step(ev[k])
+    torch.cuda.synchronize()
+    assert pc.pat_query_status() == 0
+    conv_ms = [float(np.mean([ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(3)])) for i in range(len(layers))]
+    fracs, flop_s, ms_s, roof_s = [], 0.0, 0.0, 0.0
+    for st, ms in zip(layers, conv_ms):
+        L = st["L"]
+        flop = L.useful_flop(N)
+        p_flop = (peaks["bf16_tflops"] if (L.dense and dtype == "f16") else FMA_PEAK_TFLOPS) * 1e12
+        roof_us = max(flop / p_flop, L.compulsory_bytes(N, elem) / (peaks["hbm_gbs"] * 1e9)) * 1e6
+        roof_s += roof_us
+        if not L.dense:
+            fracs.append(roof_us / (ms * 1e3)); flop_s += flop; ms_s += ms
+    touched = sum((st["x"].numel() + st["y"].numel()) * elem for st in layers)
+    res = {"workload": f"config {cfg.number}: {cfg.name}", "batch": N, "dtype": dtype, "steps": steps,
+           "images_per_s": round(N / (ms_step * 1e-3), 1), "ms_per_step": round(ms_step, 4),
+           "conv_ms_per_step": round(sum(conv_ms), 4),
+           "sparse_conv_tflops": round(flop_s / (ms_s * 1e-3) / 1e12, 3),
+           "roof_frac": round(roof_s / (sum(conv_ms) * 1e3), 4), "min_layer_frac": round(min(fracs), 4),
+           "l2": "inputs and outputs larger than L2" if touched > 4 * 126e6 else "warm L2 (working set %.0f MB, no flush between steps)" % (touched / 1e6)}
+    del layers, cws
+    torch.cuda.empty_cache()
+    return res
 
 
 # ----------------------------------------------------------------------------------------------- CPU oracle
@@ -439,11 +572,33 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="projection / packing on the same stream as the convolutions")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the short measurements of the other four configurations")
+    ap.add_argument("--fma-peak", action="store_true", help="only measure and print the device's multiply-add rate")
+    ap.add_argument("--write-traffic", default=None, metavar="NCU_CSV",
+                    help="turn an ncu launch list with the DRAM byte counters of the conv6 path into " + os.path.relpath(TRAFFIC_FILE, ROOT))
     args = ap.parse_args()
+    if args.write_traffic:
+        write_traffic(args.write_traffic)
+        return
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    world = int(os.environ.get("WORLD_SIZE", "0"))
+    if world == 0 and args.gpus > 1:
+        # no launcher around us: start one rank per GPU on this node ourselves
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 2000), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if world > 0 and world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if args.fma_peak:
+        import torch
+        import paper_2001_07710_b200 as pc
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        print(json.dumps({"fma_rn_f32_tflops": round(pc.pat_measure_fma_peak(0), 2), "fma_rn_f32_f16_tflops": round(pc.pat_measure_fma_peak(1), 2),
+                          "derived_tflops": round(FMA_PEAK_TFLOPS, 2)}))
+        return
+    run_ours(args)
 
 
 if __name__ == "__main__":

@@ -133,7 +133,9 @@ int pat_pack(const float *w_masked, const uint8_t *pattern_id, int F, int C,
 int pat_blob_layout(int F, int C, int K, int64_t n_keep, int dtype, size_t offsets[5]);
 
 /* Expand a blob back to dense masked weights [F][C][3][3] fp32 (fp16 entries are widened
- * exactly).  Inverse of pat_pack: for dtype PAT_F32 the result is bit-identical to w_masked. */
+ * exactly).  Inverse of pat_pack: for dtype PAT_F32 the result is bit-identical to w_masked.
+ * (Section 6.2 stores the re-ordered model compactly; this call reads that storage back as the
+ * masked kernels of Section 4.1, mask o kernel, which is how the packed layout is verified.) */
 int pat_unpack(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                int dtype, float *w_dense_out, void *stream);
 
@@ -148,7 +150,8 @@ int pat_unpack(const void *blob, int F, int C, const uint16_t *masks, int K, int
  *   masks    host, the library the blob was packed with (selects the compiled tap code)
  *   x        dev, NHWC [N][H][W][C], 16-byte aligned
  *   y        dev out, NHWC [N][Ho][Wo][F], 16-byte aligned, must not overlap x
- * Restrictions: C a multiple of 8, F a multiple of 8 (PAT_ERR_SHAPE otherwise). */
+ * Any F and C in 1..65535 is accepted; shapes outside the tuned kernels' reach (see pat_conv3x3_ws) run a generic
+ * kernel. */
 int pat_conv3x3(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                 int dtype, const void *x, void *y, int N, int H, int W, int stride, void *stream);
 
@@ -168,16 +171,20 @@ int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K,
                    int dtype, const void *x, void *y, int N, int H, int W, int stride,
                    void *workspace, size_t workspace_bytes, void *stream);
 
-/* Dense 3x3 convolution for layers that are not pruned (the first layer of VGG-16, C = 3).
+/* Dense 3x3 convolution for layers that are not pruned: the first layer of the VGG-16 of Section 7
+ * (C = 3 input channels), which stays dense when the other twelve are pattern-pruned.
  *   w   dev, [F][C][3][3] fp32 (converted to the activation type on the fly)
  *   x   dev NHWC [N][H][W][C]; y dev NHWC [N][Ho][Wo][F]; dtype of x and y = `dtype`
  * The case C = 3, F = 64, PAT_F16, stride 1 runs on the tensor cores (fp16 products, fp32 sums, like every
  * other path); all other cases run FMA kernels.
- * Restrictions: C <= 16, F a multiple of 8, F <= 512. */
+ * Restrictions: 1 <= C <= 16, 1 <= F <= 65535 (PAT_ERR_SHAPE otherwise). */
 int pat_conv3x3_dense(const float *w, int F, int C, int dtype, const void *x, void *y,
                       int N, int H, int W, int stride, void *stream);
 
-/* Synchronises `stream` and returns the device-side status word: PAT_OK, or PAT_ERR_BLOB when a
+/* The kernels never trap and never wait without a limit (the paper's execution scheme, Section 6.2, has no
+ * counterpart: it generates straight-line code per layer); what they cannot do they report in one status word
+ * per device.
+ * Synchronises `stream` and returns the device-side status word: PAT_OK, or PAT_ERR_BLOB when a
  * kernel found a blob header that did not match its arguments (the kernel then wrote nothing),
  * or PAT_ERR_TIMEOUT when a bounded wait inside a kernel expired (its output is then incomplete).
  * The word is cleared by the call. */
@@ -186,6 +193,24 @@ int pat_query_status(void *stream);
 /* Number of CUDA kernels this library has launched from the calling process so far (all threads,
  * all entry points).  Host-side counter; useful to check that work really ran on the GPU. */
 uint64_t pat_launch_count(void);
+
+/* Measures the device's multiply-add rate with the instruction the convolution kernels issue (kind 0: fma.rn.f32,
+ * kind 1: fma.rn.f32.f16 with an fp32 accumulator): the denominator of their roofline, taken at the clock the device
+ * really runs at.  Launches a few short kernels on `stream` and waits for them (this one call synchronises).
+ *   scratch     dev, 256-byte aligned, at least 256 + 4 * 8 * 256 * (number of SMs) bytes (2 MiB always suffices)
+ *   tflops_out  host out: best of three runs, in TFLOP/s (2 flop per multiply-add)
+ * The paper has no counterpart (it reports end-to-end latencies, Section 7.2). */
+int pat_measure_fma_peak(int kind, void *scratch, size_t scratch_bytes, double *tflops_out, void *stream);
+
+/* Test hooks of the convolution kernels' bounded waits (host-side, process-wide, not thread safe).  The paper has
+ * no counterpart.
+ *   what = 0  limit of every device-side wait in nanoseconds (value <= 0: back to the default of 2 s);
+ *   what = 1  workspace kernels (pat_conv3x3_ws): in every thread block the copy of pipeline stage number `value`
+ *             is never issued, so the wait for it runs out after the limit and the kernel ends, with every other
+ *             copy landed and its tensor memory released, leaving PAT_ERR_TIMEOUT in the status word
+ *             (value < 0: off, the default).
+ * Returns PAT_ERR_INVALID_ARG for any other `what`. */
+int pat_debug_set(int what, long long value);
 
 #ifdef __cplusplus
 }

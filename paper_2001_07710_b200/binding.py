@@ -24,7 +24,7 @@ TORCH_DTYPE = {PAT_F32: torch.float32, PAT_F16: torch.float16}
 EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project_workspace", "pat_project",
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
            "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels",
-           "pat_conv3x3_workspace", "pat_conv3x3_ws"]
+           "pat_conv3x3_workspace", "pat_conv3x3_ws", "pat_debug_set", "pat_measure_fma_peak"]
 
 
 class PatError(RuntimeError):
@@ -62,6 +62,8 @@ def load() -> C.CDLL:
     L.pat_launch_count.argtypes = []; L.pat_launch_count.restype = C.c_uint64
     L.pat_project_static.argtypes = [vp, i32, i32, vp, i32, i64, vp, vp, vp]
     L.pat_project_static_max_kernels.argtypes = []; L.pat_project_static_max_kernels.restype = i64
+    L.pat_debug_set.argtypes = [i32, C.c_longlong]
+    L.pat_measure_fma_peak.argtypes = [i32, vp, sz, vp, vp]
     _lib = L
     return L
 
@@ -189,6 +191,18 @@ def pat_query_status(stream=None) -> int:
 
 def pat_launch_count() -> int:
     return int(load().pat_launch_count())
+
+
+def pat_measure_fma_peak(kind: int = 1, stream=None) -> float:
+    """TFLOP/s of fma.rn.f32 (kind 0) or fma.rn.f32.f16 (kind 1) on the current device."""
+    scratch = torch.empty(2 << 20, dtype=torch.uint8, device="cuda")
+    out = C.c_double(0.0)
+    _check(load().pat_measure_fma_peak(int(kind), _ptr(scratch), scratch.numel(), C.byref(out), _stream(stream)))
+    return float(out.value)
+
+
+def pat_debug_set(what: int, value: int) -> None:
+    _check(load().pat_debug_set(int(what), int(value)))
 
 
 def pat_project_static_max_kernels() -> int:

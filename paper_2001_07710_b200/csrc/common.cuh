@@ -110,6 +110,19 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 #endif
 
 int set_error(int code, const char* fmt, ...);
+
+// Per-device facts and one-time set-up of a kernel family (function attributes and SM counts belong to a device, and
+// a thread may switch devices between calls): each family keeps a thread-local table and asks for the current device's
+// entry.  Returns nullptr when the device cannot be queried.
+constexpr int kMaxDevices = 64;
+struct DeviceSlot { int sms = 0; bool ready = false; };
+inline DeviceSlot* device_slot(DeviceSlot (&table)[kMaxDevices]) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceSlot& d = table[dev];
+  if (d.sms == 0 && cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+  return &d;
+}
 int check_library(const uint16_t* masks, int K);
 int check_cuda(cudaError_t e, const char* what);
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }

@@ -11,12 +11,15 @@ bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int st
 size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                  const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
+int conv_f16_img_debug(int what, long long value);
 size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                  const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
 }
 
 using namespace pat;
+
+extern "C" int pat_debug_set(int what, long long value) { return conv_f16_img_debug(what, value); }
 
 static int check_conv_args(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep, int dtype,
                            const void* x, const void* y, int N, int H, int W, int stride) {

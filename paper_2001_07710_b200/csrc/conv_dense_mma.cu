@@ -143,12 +143,10 @@ int conv_dense_c3_mma(const float* w, const void* x, void* y, int N, int H, int 
   a.N = N; a.H = H; a.W = W;
   a.tiles_x = (W + TW - 1) / TW; a.tiles_y = (H + TH - 1) / TH;
   a.n_tiles = (long long)N * a.tiles_x * a.tiles_y;
-  static thread_local int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
-    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
-  }
+  static thread_local DeviceSlot slots[kMaxDevices];
+  DeviceSlot* dv = device_slot(slots);
+  if (!dv) return set_error(PAT_ERR_CUDA, "pat_conv3x3_dense: cannot query the current device");
+  const int sm_count = dv->sms;
   const long long want = (long long)sm_count * 8;         // eight resident blocks of four warps per SM
   const unsigned grid = (unsigned)(a.n_tiles < want ? a.n_tiles : want);
   k_conv_dense_c3_mma<<<grid, NTHREADS, 0, st>>>(a);

@@ -549,18 +549,17 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
     if (cr != CUDA_SUCCESS) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cuTensorMapEncodeTiled failed (%d)", (int)cr);
   }
 
-  static thread_local int sm_count = 0;
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
-    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
+  static thread_local DeviceSlot slots[kMaxDevices];
+  DeviceSlot* dv = device_slot(slots);
+  if (!dv) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot query the current device");
+  const int sm_count = dv->sms;
+  if (!dv->ready) {
     if (int rc = check_cuda(cudaFuncSetAttribute(k_conv_f16_s1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
     cudaFuncAttributes fa;
     if (int rc = check_cuda(cudaFuncGetAttributes(&fa, k_conv_f16_s1), "query kernel attributes")) return rc;
     if (fa.numRegs < LAUNCH_REGS)
       return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
-    attr_set = true;
+    dv->ready = true;
   }
   const int grid = (int)std::min<long long>(items, sm_count);
   k_conv_f16_s1<<<grid, NTHREADS, SMEM_BYTES, st>>>(tm, p);

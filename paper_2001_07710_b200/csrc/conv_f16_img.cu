@@ -75,6 +75,8 @@ struct Params {
   // k_reduce_parts adds them up in a fixed order.  parts == 1: no cutting.
   int n_whole, n_split, parts;
   float* partials;
+  unsigned long long wait_ns;   // limit of every wait of the convolution kernel
+  int test_skip;           // test hook: the producer never issues the copies of this stage number (-1: none)
   uint16_t masks[256];     // the library (checked against the blob header)
 };
 
@@ -228,7 +230,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
     set_warp_registers<OTHER_REGS>();
     if (warp == W_PRODUCER) {
       // ========================================================================= producer warp
-      int pslot = 0;
+      int pslot = 0, stage_no = 0;
       uint32_t epar = 1u;                  // parity to wait for on slot_empty of the current slot
       uint32_t armed = 0u, armed_par = 0u; // slots with a copy that may still be in flight, and the phase it completes
       bool alive = true;
@@ -242,14 +244,17 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         uint32_t o0 = __ldg(bo + c0);
         for (int cb = c0; cb < c1 && alive; ++cb) {
           const uint32_t o1 = __ldg(bo + cb + 1);
-          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag, p.wait_ns)) { alive = false; break; }
           if (lane == 0) {
             const uint32_t dbytes = (o1 - o0) * 16u;
             const uint32_t dst = slot0 + (uint32_t)pslot * SLOT;
             mbar_arrive_expect_tx(slot_full(pslot), (uint32_t)IMG_BYTES + dbytes);
-            bulk_load(dst + IMG_BYTES, p.dblk + (size_t)o0 * 16, dbytes, slot_full(pslot));
-            bulk_load(dst, img + (size_t)cb * IMG_BYTES, (uint32_t)IMG_BYTES, slot_full(pslot));
+            if (stage_no != p.test_skip) {
+              bulk_load(dst + IMG_BYTES, p.dblk + (size_t)o0 * 16, dbytes, slot_full(pslot));
+              bulk_load(dst, img + (size_t)cb * IMG_BYTES, (uint32_t)IMG_BYTES, slot_full(pslot));
+            }
           }
+          ++stage_no;
           armed |= 1u << pslot;
           armed_par = (armed_par & ~(1u << pslot)) | ((epar ^ 1u) << pslot);
           o0 = o1;
@@ -257,7 +262,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         }
         // output stages: hand the next two slots to the consumers as they become free (a piece has none)
         for (int o = 0; o < TR4 / 2 && alive && !piece; ++o) {
-          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<kFillSleepNs>(slot_empty(pslot), epar, abort_flag, p.wait_ns)) { alive = false; break; }
           if (lane == 0) mbar_arrive(slot_full(pslot));
           armed &= ~(1u << pslot);
           if (++pslot == NS) { pslot = 0; epar ^= 1u; }
@@ -270,7 +275,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           if (!((armed >> s) & 1u)) continue;
           for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
             if (mbar_try_wait(slot_full(s), (armed_par >> s) & 1u)) break;
-            if (global_ns() - t0 > kWaitNs) break;
+            if (global_ns() - t0 > p.wait_ns) break;
           }
         }
         atomicExch(p.status, PAT_ERR_TIMEOUT);
@@ -314,7 +319,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       // the warp holds, then (flag kOpSwap) the other filter's; the last one carries kOpEnd and the place of the
       // warp's list in the next stage's block.  The next operation and the first two window rows of the current
       // one are loaded before the pattern's code runs.
-      if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+      if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag, p.wait_ns)) { alive = false; break; }
       uint32_t sl = slot0 + (uint32_t)pslot * SLOT;
       uint32_t pl0 = sl + offA;
       const uint32_t hw = lds32(sl + IMG_BYTES + (uint32_t)warp * 4u);
@@ -346,7 +351,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           if (lane == 0) mbar_arrive(slot_empty(pslot));
           if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
           if (++cb == c1) break;
-          if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag)) { alive = false; break; }
+          if (!mbar_wait<0>(slot_full(pslot), fpar, abort_flag, p.wait_ns)) { alive = false; break; }
           sl = slot0 + (uint32_t)pslot * SLOT;
           pl0 = sl + offA;
           e = sl + IMG_BYTES + kBlockHeaderBytes + (cm >> kOpNextShift) * 16u;
@@ -382,8 +387,8 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       const uint32_t cposB = ((uint32_t)__ldg(p.xfilt + g_out * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 2u;
       const int s0 = pslot, s1 = (pslot + 1 == NS) ? 0 : pslot + 1;
       const uint32_t par1 = (pslot + 1 == NS) ? (fpar ^ 1u) : fpar;
-      if (!mbar_wait<0>(slot_full(s0), fpar, abort_flag)) { alive = false; break; }
-      if (!mbar_wait<0>(slot_full(s1), par1, abort_flag)) { alive = false; break; }
+      if (!mbar_wait<0>(slot_full(s0), fpar, abort_flag, p.wait_ns)) { alive = false; break; }
+      if (!mbar_wait<0>(slot_full(s1), par1, abort_flag, p.wait_ns)) { alive = false; break; }
       const uint32_t ob0 = slot0 + (uint32_t)s0 * SLOT, ob1 = slot0 + (uint32_t)s1 * SLOT;
       {
         // tiles 16-31 sit one word further on: lanes l and l + 16 would otherwise store to the same banks
@@ -404,7 +409,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(out_ready(0));
-      if (!mbar_wait<0>(out_ready(0), (uint32_t)(it_idx & 1), abort_flag)) { alive = false; break; }
+      if (!mbar_wait<0>(out_ready(0), (uint32_t)(it_idx & 1), abort_flag, p.wait_ns)) { alive = false; break; }
       {
         const Region it = decode_region(p, item / p.NG);
         const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
@@ -456,6 +461,16 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
   if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
+// The blob was packed with the parameters of this call (every thread reads the same header: a uniform decision).
+__device__ __forceinline__ bool blob_matches(const Params& p) {
+  const BlobHeader* bh = p.hdr;
+  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
+            bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep &&
+            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * kChanTile + kBlockWarps;
+  for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
+  return ok;
+}
+
 // NCODES / GENERIC: the pattern codes the kernel carries code for (see one_kernel4); the host picks the smallest
 // set that covers the library.
 template <int NCODES, bool GENERIC>
@@ -464,12 +479,10 @@ k_conv_f16_img(const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   // refuse a blob packed with other parameters (uniform decision: every thread reads the same header)
   const BlobHeader* bh = p.hdr;
-  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
-            bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep &&
-            bh->max_block_entries >= 0 && bh->max_block_entries <= FG * kChanTile + kBlockWarps;
-  for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
+  const bool ok = blob_matches(p);
   if (!ok) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
   // everything below reads the stage images or writes the output: the stage-image grid must be complete
@@ -488,8 +501,9 @@ constexpr int MAX_PIECES = 256;            // pieces in flight (the workspace ho
 constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
 constexpr int RP_THREADS = 1024, MAX_PARTS = 8, RP_XH = TC / 2;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
-  __shared__ __align__(16) unsigned char stage[OUT_ROW];
   asm volatile("griddepcontrol.wait;" ::: "memory");   // launched as a programmatic dependent of the convolution kernel
+  if (!blob_matches(p)) return;                          // the convolution kernel refused the blob and wrote no partial sums
+  __shared__ __align__(16) unsigned char stage[OUT_ROW];
   // block = (cut item, row of the thread tiles, left or right half of the tile columns)
   const int xh = (int)blockIdx.x & 1, y = ((int)blockIdx.x >> 1) % TR4, li = (int)blockIdx.x / (2 * TR4);
   const int item = p.n_whole + li;
@@ -562,6 +576,16 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
 
 }  // namespace img16
 
+// test hooks of the bounded waits (see pat_debug_set)
+static unsigned long long g_wait_ns = fast16::kWaitNs;
+static int g_test_skip = -1;
+int conv_f16_img_debug(int what, long long value) {
+  if (what == 0) g_wait_ns = value > 0 ? (unsigned long long)value : fast16::kWaitNs;
+  else if (what == 1) g_test_skip = value < 0 ? -1 : (int)value;
+  else return set_error(PAT_ERR_INVALID_ARG, "pat_debug_set: unknown switch %d", what);
+  return PAT_OK;
+}
+
 // True when the stage-image kernels cover this layer.
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
@@ -580,7 +604,7 @@ size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
   using namespace img16;
   if (!conv_f16_img_supported(F, C, dtype, N, H, W, stride)) return 0;
   Params p;
-  fill_geometry(p, F, C, N, H, W);
+  if (!fill_geometry(p, F, C, N, H, W)) return 0;
   return align256((size_t)p.n_regions * p.nct * IMG_BYTES) + MAX_PIECES * PIECE_FLOATS * sizeof(float);
 }
 
@@ -601,6 +625,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.status = status_word();
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
+  p.wait_ns = g_wait_ns; p.test_skip = g_test_skip;
   p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
@@ -613,12 +638,11 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   using KernelFn = void (*)(const Params);
   static const KernelFn kernels[3] = {k_conv_f16_img<6, false>, k_conv_f16_img<kNumCodes, false>, k_conv_f16_img<kNumCodes, true>};
 
-  static thread_local int sm_count = 0;
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
-    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
+  static thread_local DeviceSlot slots[kMaxDevices];
+  DeviceSlot* dv = device_slot(slots);
+  if (!dv) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot query the current device");
+  const int sm_count = dv->sms;
+  if (!dv->ready) {
     if (int rc = check_cuda(cudaFuncSetAttribute(k_stage_images, cudaFuncAttributeMaxDynamicSharedMemorySize, SI_SMEM), "set shared memory size")) return rc;
     for (KernelFn fn : kernels) {
       if (int rc = check_cuda(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
@@ -627,7 +651,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
       if (fa.numRegs < LAUNCH_REGS)
         return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
     }
-    attr_set = true;
+    dv->ready = true;
   }
   int grid = std::min(p.n_items, sm_count);
   // fewer work items than half the SMs (small batches): every item is cut along the input channels, so that up to

@@ -502,17 +502,25 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
   if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
-template <int NCODES, bool GENERIC>
-__global__ void __launch_bounds__(NTHREADS, 1)
-k_conv_f32_img(const Params p) {
-  extern __shared__ __align__(1024) unsigned char smem[];
+// The blob was packed with the parameters of this call (every thread reads the same header: a uniform decision).
+__device__ __forceinline__ bool blob_matches(const Params& p) {
   const BlobHeader* bh = p.hdr;
   bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
             bh->K == p.K && bh->dtype == PAT_F32 && bh->n_keep == p.n_keep &&
             bh->max_block_entries >= 0 && bh->max_block_entries <= FG * CBI + kBlockWarps;
   for (int j = 0; ok && j < p.K; ++j) ok = bh->masks[j] == p.masks[j];
-  if (!ok) {
+  return ok;
+}
+
+template <int NCODES, bool GENERIC>
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_conv_f32_img(const Params p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  // refuse a blob packed with other parameters (uniform decision: every thread reads the same header)
+  const BlobHeader* bh = p.hdr;
+  if (!blob_matches(p)) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(p.status, PAT_ERR_BLOB);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     return;
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -528,6 +536,7 @@ constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
 constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!blob_matches(p)) return;                          // the convolution kernel refused the blob and wrote no partial sums
   const int v = (int)blockIdx.x % (TR4 * TC), li = (int)blockIdx.x / (TR4 * TC);
   const int item = p.n_whole + li;
   const int g = item % p.NG;
@@ -620,12 +629,11 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   using KernelFn = void (*)(const Params);
   static const KernelFn kernels[3] = {k_conv_f32_img<6, false>, k_conv_f32_img<kNumCodes, false>, k_conv_f32_img<kNumCodes, true>};
 
-  static thread_local int sm_count = 0;
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    if (int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice")) return rc;
-    if (int rc = check_cuda(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev), "query SM count")) return rc;
+  static thread_local DeviceSlot slots[kMaxDevices];
+  DeviceSlot* dv = device_slot(slots);
+  if (!dv) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot query the current device");
+  const int sm_count = dv->sms;
+  if (!dv->ready) {
     if (int rc = check_cuda(cudaFuncSetAttribute(k_stage_images_f32, cudaFuncAttributeMaxDynamicSharedMemorySize, SI_SMEM), "set shared memory size")) return rc;
     for (KernelFn fn : kernels) {
       if (int rc = check_cuda(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES), "set shared memory size")) return rc;
@@ -634,7 +642,7 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
       if (fa.numRegs < LAUNCH_REGS)
         return set_error(PAT_ERR_CUDA, "pat_conv3x3: kernel was compiled with %d registers per thread, the register split needs %d", fa.numRegs, LAUNCH_REGS);
     }
-    attr_set = true;
+    dv->ready = true;
   }
   int grid = std::min(p.n_items, sm_count);
   // fewer work items than half the SMs (small batches): every item is cut along the input channels, so that up to

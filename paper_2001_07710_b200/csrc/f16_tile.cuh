@@ -50,13 +50,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: gives up after kWaitNs of wall time (or kSpinLimit polls), raises the block-wide abort flag
+// Bounded wait: gives up after limit_ns of wall time (or kSpinLimit polls), raises the block-wide abort flag
 // and returns false; also returns false as soon as another thread of the block has given up.
 // SLEEP_NS > 0: sleep between polls.  The fill and store warps wait that way: a polling warp takes issue
 // slots from the four consumer warps of its SM partition, and those warps have slack (they work ahead by up
 // to three ring slots).  Consumers poll without sleeping: they rarely wait, and must restart at once.
 template <int SLEEP_NS>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns = kWaitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
@@ -64,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 31u) == 31u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitNs) break;
+      if (global_ns() - t0 > limit_ns) break;
     }
   }
   *abort_flag = 1;

@@ -191,6 +191,9 @@ template <typename T, bool TABLE>
 __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ wm, const uint8_t* __restrict__ pid,
                                                       int C, int K, int nct, MaskTable lib, BlobPtrs bp) {
   pdl_wait();
+  // k_pack_ptrs refused the inputs (pattern_id keeps another number of kernels than n_keep): the positions computed
+  // below would leave the sections sized by n_keep, so nothing is written
+  if (bp.hdr->magic != kBlobMagic) return;
   extern __shared__ __align__(16) uint8_t sm_raw[];
   int* tile_pat = reinterpret_cast<int*>(sm_raw);                          // [nct][K] (TABLE only)
   int* tile_start = tile_pat + (TABLE ? nct * K : 0);                      // [nct + 1] kept kernels before tile t
@@ -285,6 +288,7 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
 // Launched with one warp per block (lane = consumer warp, lanes 16-31 idle apart from the shuffles).
 __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
   pdl_wait();
+  if (bp.hdr->magic != kBlobMagic) return;   // refused by k_pack_ptrs, see k_pack_scatter
   const int blk = blockIdx.x, lane = threadIdx.x;
   const int g = blk / nct, cb = blk % nct;
   const bool active = lane < kBlockWarps;
@@ -354,6 +358,7 @@ __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable
 // Offsets (header words, "next list", dboff) count 16-byte units as in fp16 blobs, so an operation is two units.
 __global__ void __launch_bounds__(32) k_pack_blocks_f32(int nct, int nblk, MaskTable lib, BlobPtrs bp) {
   pdl_wait();
+  if (bp.hdr->magic != kBlobMagic) return;   // refused by k_pack_ptrs, see k_pack_scatter
   const int blk = blockIdx.x, lane = threadIdx.x;
   const int nst = 2 * nct;                                   // stages of 8 channels
   const int g = blk / nst, st8 = blk % nst;
@@ -491,28 +496,30 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const MaskTable lib = make_table(masks, K);
   const BlobPtrs bp = blob_ptrs(blob, L, F, K);
-  launch_dependent(k_pack_count, dim3(F), dim3(256), K * sizeof(int), st, pattern_id, C, K, bp, status);
-  launch_dependent(k_pack_rank, dim3(F), dim3(128), 0, st, F, K, bp);
-  launch_dependent(k_pack_ptrs, dim3(1), dim3(1024), 0, st, F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status);
-  {
-    const size_t table = sizeof(int) * (size_t)L.nct * K;
-    const bool use_table = table <= 24 * 1024;
-    const size_t smem = (use_table ? table : 0) + sizeof(int) * ((size_t)L.nct + 1) + (size_t)C;
-    if (smem > 48 * 1024) return set_error(PAT_ERR_SHAPE, "pat_pack: C=%d too large for the packing kernel", C);
-    if (dtype == PAT_F16) {
-      if (use_table) launch_dependent(k_pack_scatter<__half, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
-      else launch_dependent(k_pack_scatter<__half, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
-    } else {
-      if (use_table) launch_dependent(k_pack_scatter<float, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
-      else launch_dependent(k_pack_scatter<float, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp);
-    }
+  // every check that can refuse the call comes before the first launch
+  const size_t table = sizeof(int) * (size_t)L.nct * K;
+  const bool use_table = table <= 24 * 1024;
+  const size_t smem = (use_table ? table : 0) + sizeof(int) * ((size_t)L.nct + 1) + (size_t)C;
+  if (smem > 48 * 1024) return set_error(PAT_ERR_SHAPE, "pat_pack: C=%d too large for the packing kernel", C);
+  cudaError_t le = cudaSuccess;                   // first launch error, if any
+  auto note = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
+  note(launch_dependent(k_pack_count, dim3(F), dim3(256), K * sizeof(int), st, pattern_id, C, K, bp, status));
+  note(launch_dependent(k_pack_rank, dim3(F), dim3(128), 0, st, F, K, bp));
+  note(launch_dependent(k_pack_ptrs, dim3(1), dim3(1024), 0, st, F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status));
+  if (dtype == PAT_F16) {
+    if (use_table) note(launch_dependent(k_pack_scatter<__half, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));
+    else note(launch_dependent(k_pack_scatter<__half, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));
+  } else {
+    if (use_table) note(launch_dependent(k_pack_scatter<float, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));
+    else note(launch_dependent(k_pack_scatter<float, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));
   }
   count_launches(4);
   if (L.nblk > 0) {
-    if (dtype == PAT_F16) launch_dependent(k_pack_blocks, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
-    else launch_dependent(k_pack_blocks_f32, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp);
+    if (dtype == PAT_F16) note(launch_dependent(k_pack_blocks, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp));
+    else note(launch_dependent(k_pack_blocks_f32, dim3(L.nblk), dim3(32), 0, st, L.nct, L.nblk, lib, bp));
     count_launches(1);
   }
+  if (le != cudaSuccess) return check_cuda(le, "pat_pack launch");
   return check_cuda(cudaGetLastError(), "pat_pack launch");
 }
 

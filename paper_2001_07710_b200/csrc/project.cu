@@ -292,13 +292,16 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   if (mode < 0) {
     if (int rc = check_cuda(cudaMemsetAsync(ws.hist, 0, 4 * kHistWords, st), "pat_project memset")) return rc;
   }
-  launch_dependent(k_select_pattern, dim3(nb256), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0);
+  cudaError_t le = cudaSuccess;                   // first launch error, if any
+  auto note = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
+  note(launch_dependent(k_select_pattern, dim3(nb256), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0));
   if (mode < 0) {
-    for (int pass = 1; pass < kPasses; ++pass) launch_dependent(k_sel_hist, dim3(nb256), dim3(256), 0, st, ws.key, FC, pass, ws.st, ws.hist);
-    launch_dependent(k_tie_count, dim3(nblk), dim3(kSelBlock), 0, st, ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord);
+    for (int pass = 1; pass < kPasses; ++pass) note(launch_dependent(k_sel_hist, dim3(nb256), dim3(256), 0, st, ws.key, FC, pass, ws.st, ws.hist));
+    note(launch_dependent(k_tie_count, dim3(nblk), dim3(kSelBlock), 0, st, ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord));
   }
-  launch_dependent(k_finalize, dim3(nblk), dim3(kSelBlock), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode);
+  note(launch_dependent(k_finalize, dim3(nblk), dim3(kSelBlock), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode));
   count_launches(mode < 0 ? 6 : 2);
+  if (le != cudaSuccess) return check_cuda(le, "pat_project launch");
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
 

@@ -1,9 +1,12 @@
 """Full-size parity on the five evaluation configurations, in the launch configuration bench.py times.
 
 Projection and packing are compared bit for bit with the oracle on every layer.  The convolution output of the
-full batch is compared on sampled coordinates (all corners and edges of the first and last image plus seeded random
-points), each computed by the oracle's direct float64 definition; every output element is also checked to have
-been written (finite) and the status word to be clean.
+full batch is compared element by element on whole images - the first, the middle and the last of the batch - for
+every layer whose single image costs the oracle's direct float64 definition at most WHOLE_IMAGE_MACS multiply-adds
+(test id "...-whole"; all layers of the five configurations do), and on sampled coordinates of all images (all
+corners and edges of the first and last image plus seeded random points); a layer above that cost would be
+compared on the samples only (id "...-sampled").  Every output element is also checked to have been written
+(finite) and the status word to be clean.
 """
 import numpy as np
 import pytest
@@ -17,6 +20,11 @@ from helpers import check_close, read_blob
 pytestmark = pytest.mark.gpu
 
 N_RANDOM = 3000
+WHOLE_IMAGE_MACS = 2.5e9      # dense 9 * C * F * Ho * Wo of one image: about a second of the oracle on 16 cores
+
+
+def _whole(L) -> bool:
+    return 9.0 * L.C * L.F * L.Ho * L.Wo <= WHOLE_IMAGE_MACS
 
 
 def _sample_coords(rng, N, Ho, Wo, F):
@@ -62,11 +70,16 @@ def _check_layer(cfg, L):
     ref = oracle.conv3x3_at(wst, xs, coords, L.stride)
     out = y[coords[:, 0], coords[:, 1], coords[:, 2], coords[:, 3]].float().cpu().numpy()
     check_close(out, ref, dtype)
+    if _whole(L):
+        for n in sorted({0, cfg.N // 2, cfg.N - 1}):
+            ref_img = oracle.conv3x3(wst, xs[n:n + 1], L.stride)
+            check_close(y[n:n + 1].float().cpu().numpy(), ref_img, dtype)
 
 
 def _layers(cfg_no):
     cfg = workloads.configs()[cfg_no]
-    return [pytest.param(cfg_no, i, id=f"cfg{cfg_no}-{L.name}") for i, L in enumerate(cfg.layers)]
+    return [pytest.param(cfg_no, i, id=f"cfg{cfg_no}-{L.name}-{'whole' if _whole(L) else 'sampled'}")
+            for i, L in enumerate(cfg.layers)]
 
 
 @pytest.mark.parametrize("cfg_no,layer_idx", _layers(0) + _layers(1) + _layers(2) + _layers(3) + _layers(4))

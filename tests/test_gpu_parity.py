@@ -371,3 +371,90 @@ def test_dense_conv_matches_oracle(N, H, W, C, F, stride, dtype):
     ref = oracle.conv3x3(stored_weights(w, dtype), x, stride)
     y = pc.pat_conv3x3_dense(torch.from_numpy(w).cuda(), dtype, torch.from_numpy(x).cuda(), stride)
     check_close(y.float().cpu().numpy(), ref, dtype)
+
+
+# ------------------------------------------------------------------ refused inputs and failed waits
+def test_pack_refuses_wrong_n_keep_and_writes_nothing_outside_the_blob():
+    """pattern_id keeps more kernels than the n_keep given to pat_pack: the blob is refused (status PAT_ERR_BLOB,
+    magic cleared) and no kernel writes past the sections sized by n_keep: the blob sits inside a buffer of
+    canary bytes that must stay untouched."""
+    F, C, K = 64, 64, 8
+    masks = oracle.library(K)
+    w = torch.from_numpy(_weights(11, F, C)).cuda()
+    pid, wm = pc.pat_project(w, masks, F * C // 2)                   # 2048 kernels kept
+    for dtype in ("f32", "f16"):
+        n_wrong = F * C // 8                                         # pack is told 512
+        size = pc.pat_pack_size(F, C, K, n_wrong, dtype)
+        pad = 1 << 20
+        buf = torch.full((size + 2 * pad,), 0xC5, dtype=torch.uint8, device="cuda")
+        blob = buf[pad:pad + size]
+        assert blob.data_ptr() % 256 == 0
+        pc.pat_pack(wm, pid, masks, n_wrong, dtype, blob=blob)
+        with pytest.raises(pc.PatError) as e:
+            pc.pat_query_status()
+        assert e.value.code == 6
+        assert bool((buf[:pad] == 0xC5).all()) and bool((buf[pad + size:] == 0xC5).all())
+        assert int(blob[:4].view(torch.int32)[0]) == 0               # the header's magic: the blob cannot be used
+    assert pc.pat_query_status() == 0
+
+
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+def test_blob_mismatch_on_the_workspace_path_writes_nothing(dtype):
+    """A blob packed with another library, on a shape the workspace kernels cover with cut items (one small image:
+    the reduce kernel would run): the status word says PAT_ERR_BLOB and y is untouched; the same holds for a header
+    whose magic or version word was overwritten."""
+    N, H, W, C, F, K = 1, 28, 28, 64, 32, 8
+    masks = oracle.library(K)
+    n_keep = F * C // 4
+    _, _, blob = gpu_project_pack(_weights(12, F, C), masks, n_keep, dtype)
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    x = torch.zeros((N, H, W, C), dtype=tdt, device="cuda")
+    assert pc.pat_conv3x3_workspace(F, C, dtype, N, H, W, 1) > 0
+    other = oracle.library(12)[4:12]
+
+    def refused(blob_, masks_):
+        y = torch.full((N, H, W, F), 7.0, dtype=tdt, device="cuda")
+        pc.pat_conv3x3(blob_, F, C, masks_, n_keep, dtype, x, 1, y=y)
+        with pytest.raises(pc.PatError) as e:
+            pc.pat_query_status()
+        assert e.value.code == 6
+        assert float(y.min()) == 7.0 and float(y.max()) == 7.0
+
+    refused(blob, other)
+    for word in (0, 1):                                              # magic, version
+        bad = blob.clone()
+        bad[4 * word:4 * word + 4] = 0x5A
+        refused(bad, masks)
+    assert pc.pat_query_status() == 0
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, x, 1)        # the intact blob still runs
+    assert pc.pat_query_status() == 0 and not y.any()
+
+
+def test_bounded_wait_runs_out_and_is_reported():
+    """The copies of one pipeline stage are never issued (test hook) and the wait limit is 1 ms: the kernel must
+    end by itself, report PAT_ERR_TIMEOUT once, and leave the device usable: the next, normal call matches the
+    oracle."""
+    N, H, W, C, F, K = 4, 56, 56, 64, 64, 8
+    rng = np.random.default_rng(31)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), "f16")
+    masks = oracle.library(K)
+    n_keep = F * C // 8
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    _, _, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    xt = torch.from_numpy(x).cuda()
+    assert pc.pat_conv3x3_workspace(F, C, "f16", N, H, W, 1) > 0
+    try:
+        pc.pat_debug_set(0, 1_000_000)       # 1 ms
+        pc.pat_debug_set(1, 1)               # second stage of every thread block
+        pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1)
+        with pytest.raises(pc.PatError) as e:
+            pc.pat_query_status()
+        assert e.value.code == 9
+    finally:
+        pc.pat_debug_set(1, -1)
+        pc.pat_debug_set(0, 0)
+    assert pc.pat_query_status() == 0        # the word was cleared
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1)
+    assert pc.pat_query_status() == 0
+    check_close(y.float().cpu().numpy(), oracle.conv3x3(stored_weights(wm_o, "f16"), x, 1), "f16")

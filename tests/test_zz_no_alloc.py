@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2001_07710_b200 as pc
 from paper_2001_07710_b200 import workloads
 
@@ -16,19 +17,33 @@ pytestmark = pytest.mark.gpu
 
 
 def _run_both(seed, F, C, K, n_keep):
-    w = torch.from_numpy(workloads.make_weights(np.random.default_rng(seed), F, C)).cuda()
+    w_np = workloads.make_weights(np.random.default_rng(seed), F, C)
+    w = torch.from_numpy(w_np).cuda()
     masks = pc.pat_library_builtin(K)
     # reference: the ordinary entry point with a caller-provided workspace
     pid_ref, wm_ref = pc.pat_project(w, masks, n_keep)
+    torch.cuda.synchronize()
     # outputs are preallocated here, before the call: the call itself must allocate nothing
     pid = torch.full((F, C), 0x5A, dtype=torch.uint8, device="cuda")
     wm = torch.full((F, C, 3, 3), float("nan"), dtype=torch.float32, device="cuda")
+    # a first call on this device looks up the scratch array's address (and loads the module); the calls that are
+    # measured come after it
+    pc.pat_project_static(w, masks, n_keep, pid, wm)
+    pid.fill_(0x5A)
+    wm.fill_(float("nan"))
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
+    before = torch.cuda.memory_allocated()          # torch's allocator ...
+    torch.cuda.reset_peak_memory_stats()            # ... and its high-water mark from here on
+    free_before = torch.cuda.mem_get_info()[0]      # the driver's view (cudaMemGetInfo): sees any cudaMalloc
     pc.pat_project_static(w, masks, n_keep, pid, wm)
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.max_memory_allocated() == before and torch.cuda.memory_allocated() == before
+    assert torch.cuda.mem_get_info()[0] == free_before
     assert pc.pat_query_status() == 0
+    # against the oracle (brute force over the library, sort for connectivity): bit for bit
+    pid_o, wm_o, _ = oracle.project(w_np, masks, n_keep)
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    assert np.array_equal(wm.cpu().numpy().view(np.uint32), wm_o.view(np.uint32))
     # integer and bit-pattern work: the tolerance of the projection tests is exact equality
     assert torch.equal(pid, pid_ref)
     assert torch.equal(wm.view(torch.int32), wm_ref.view(torch.int32))
