@@ -368,7 +368,9 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       int cb = c0;
 #pragma unroll 1
       for (;;) {
-        const uint32_t cm = m0, coff = off;
+        // all lanes hold the same descriptor word; the warp-wide reduction makes that known to the compiler, so that
+        // the branches of this visit are uniform branches without reconvergence bookkeeping (see conv_f16_img.cu)
+        const uint32_t cm = __reduce_or_sync(0xFFFFFFFFu, m0), coff = off;
         float w[4] = {__uint_as_float(w0), __uint_as_float(w1), __uint_as_float(w2), __uint_as_float(w3)};
         float r0[16];                      // the first window row of this kernel (window rows 0-3 share the lane's swizzle)
         lds_row_f32(r0, pl0 + coff, swb);
