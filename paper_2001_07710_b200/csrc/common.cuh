@@ -9,7 +9,7 @@
 namespace pat {
 
 constexpr uint32_t kBlobMagic = 0x50415443u;  // "PATC"
-constexpr uint32_t kBlobVersion = 3u;
+constexpr uint32_t kBlobVersion = 4u;
 constexpr int kChanTile = 16;                 // granularity (input channels) of the execution section
 constexpr int kExecGroup = 32;                // filters per execution group (aligned groups of original filters)
 constexpr int kMaxK = 255;
@@ -108,6 +108,27 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
+
+// Division of 0 <= n < 2^32 by a number known on the host (Granlund and Montgomery's multiply-and-shift): three
+// instructions instead of the twenty-odd of a division by a run-time value.
+struct FastDiv {
+  uint32_t d, m, sh1, sh2;
+  void set(int div) {
+    d = (uint32_t)div;
+    uint32_t l = 0;
+    while ((1ull << l) < (unsigned long long)d) ++l;                       // ceil(log2 d)
+    m = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+    sh1 = l < 1 ? l : 1;
+    sh2 = l > 0 ? l - 1 : 0;
+  }
+#ifdef __CUDACC__
+  __device__ __forceinline__ int div(int n) const {
+    const uint32_t t = __umulhi(m, (uint32_t)n);
+    return (int)((t + (((uint32_t)n - t) >> sh1)) >> sh2);
+  }
+  __device__ __forceinline__ int mod(int n) const { return n - div(n) * (int)d; }
+#endif
+};
 
 int set_error(int code, const char* fmt, ...);
 

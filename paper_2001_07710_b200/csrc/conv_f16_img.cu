@@ -75,6 +75,7 @@ struct Params {
   // k_reduce_parts adds them up in a fixed order.  parts == 1: no cutting.
   int n_whole, n_split, parts;
   float* partials;
+  FastDiv d_CG, d_TY, d_NG;     // divisions by CG, TY, NG
   unsigned long long wait_ns;   // limit of every wait of the convolution kernel
   int test_skip;           // test hook: the producer never issues the copies of this stage number (-1: none)
   uint16_t masks[256];     // the library (checked against the blob header)
@@ -92,10 +93,11 @@ struct Region {
 
 __device__ __forceinline__ Region decode_region(const Params& p, int reg) {
   Region r;
-  r.cg = reg % p.CG;
-  const int gt0 = (reg / p.CG) * LY;
-  r.ig0 = gt0 / p.TY;
-  r.ta0 = gt0 % p.TY;
+  const int rb = p.d_CG.div(reg);
+  r.cg = reg - rb * p.CG;
+  const int gt0 = rb * LY;
+  r.ig0 = p.d_TY.div(gt0);
+  r.ta0 = gt0 - r.ig0 * p.TY;
   r.n0 = min(LY, p.TY - r.ta0);
   r.band1 = (r.n0 < LY) && (r.ig0 + 1 < p.NIG);
   r.nrows = r.band1 ? MAXROWS : TR4 * r.n0 + 2;
@@ -236,7 +238,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       bool alive = true;
       for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
         const int item = item_of(it_idx);
-        const int g = item % p.NG, reg = item / p.NG;
+        const int reg = p.d_NG.div(item), g = item - reg * p.NG;
         const char* img = p.images + (size_t)reg * nct * IMG_BYTES;
         const uint32_t* bo = p.dboff + (size_t)g * nct;
         int c0, c1;
@@ -303,7 +305,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
     for (int it_idx = 0; it_idx < n_my_items && alive; ++it_idx) {
       uint32_t offA;                     // the lane's address of logical chunk 0 of window row 0, relative to a channel plane
       {                                  // (logical chunk 1 sits at offA ^ 16)
-        const Region it = decode_region(p, item_of(it_idx) / p.NG);
+        const Region it = decode_region(p, p.d_NG.div(item_of(it_idx)));
         const int ly = lane >> 2, lx = lane & 3;
         const int b = (ly < it.n0) ? 0 : 1;                  // band of this lane's tile row
         offA = (uint32_t)((TR4 * ly + 2 * b) * ROWB + lx * SEGB + ((ly & 1) << 4));
@@ -329,6 +331,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       uint32_t m0, w01, w23, off;
       lds128(e, m0, w01, w23, off);
       int cb = c0;
+      uint32_t where = 0u;               // output channels of the warp's two filters (read from the last stage's block)
 #pragma unroll 1
       for (;;) {
         const uint32_t a0 = pl0 + off;
@@ -352,6 +355,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
         one_kernel4<NCODES, GENERIC>(acc, pl0, cm, c01, c23, coff, r0, r1);
       stage_end:
         if (cm & kOpEnd) {
+          if (cb + 1 == c1) where = lds32(sl + IMG_BYTES + (uint32_t)(kBlockWarps + warp) * 4u);
           __syncwarp();
           if (lane == 0) mbar_arrive(slot_empty(pslot));
           if (++pslot == NS) { pslot = 0; fpar ^= 1u; }
@@ -386,10 +390,9 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       // results: fp32 -> fp16 (round to nearest even) into the two output stages (tile rows 0-1 and 2-3), then,
       // once all 16 warps have written, every warp copies two thread tiles to global memory
       const int item = item_of(it_idx);
-      const int g_out = item % p.NG;
+      const int g_out = p.d_NG.mod(item);
       // byte offsets of filters 0 / 1 inside the group of 32 output channels
-      const uint32_t cposA = ((uint32_t)__ldg(p.xfilt + g_out * FG + warp) & (uint32_t)(FG - 1)) * 2u;
-      const uint32_t cposB = ((uint32_t)__ldg(p.xfilt + g_out * FG + FG - 1 - warp) & (uint32_t)(FG - 1)) * 2u;
+      const uint32_t cposA = (where & 0xFFu) * 2u, cposB = ((where >> 8) & 0xFFu) * 2u;
       const int s0 = pslot, s1 = (pslot + 1 == NS) ? 0 : pslot + 1;
       const uint32_t par1 = (pslot + 1 == NS) ? (fpar ^ 1u) : fpar;
       if (!mbar_wait<0>(slot_full(s0), fpar, abort_flag, p.wait_ns)) { alive = false; break; }
@@ -416,7 +419,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
       if (lane == 0) mbar_arrive(out_ready(0));
       if (!mbar_wait<0>(out_ready(0), (uint32_t)(it_idx & 1), abort_flag, p.wait_ns)) { alive = false; break; }
       {
-        const Region it = decode_region(p, item / p.NG);
+        const Region it = decode_region(p, p.d_NG.div(item));
         const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
         // 14 pixels x 4 chunks of 8 channels per tile row: consecutive lanes take consecutive chunks, so every pixel
         // is written as one 64-byte run; all loads of a tile are issued before its stores
@@ -512,8 +515,8 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   // block = (cut item, row of the thread tiles, left or right half of the tile columns)
   const int xh = (int)blockIdx.x & 1, y = ((int)blockIdx.x >> 1) % TR4, li = (int)blockIdx.x / (2 * TR4);
   const int item = p.n_whole + li;
-  const int g = item % p.NG;
-  const Region it = decode_region(p, item / p.NG);
+  const int g = p.d_NG.mod(item);
+  const Region it = decode_region(p, p.d_NG.div(item));
   const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS;
   constexpr int PER_THREAD = FG * RP_XH * 32 / RP_THREADS;   // 7
   static_assert(FG * RP_XH * 32 % RP_THREADS == 0, "elements per thread");
@@ -576,6 +579,7 @@ static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
   p.n_regions = (int)regions;
   p.n_items = (int)items;
   p.n_whole = p.n_items; p.n_split = 0; p.parts = 1; p.partials = nullptr;
+  p.d_CG.set(p.CG); p.d_TY.set(p.TY); p.d_NG.set(p.NG);
   return true;
 }
 

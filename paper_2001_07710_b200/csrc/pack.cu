@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(256) k_pack_scatter(const float* __restrict__ 
 // whatever the previous stage left), first the kernels of that filter, then - only if the other filter has kernels
 // in this tile - a swap and the other filter's kernels.
 //   header   32 words; word w < 16: first operation of warp w (bits 0-15) | filter whose tile is in registers when
-//            the stage begins (bit 31).  Words 16-31 unused.
+//            the stage begins (bit 31).  Word 16 + w: the output channels (inside the group of 32) of warp w's filters.
 //   lists    16 bytes per operation, warp after warp, every list one slot longer than the warp's kernels:
 //            {channel inside the tile | pattern_word(mask) | flags, taps 0-1 (fp16 x2), taps 2-3 (fp16 x2),
 //             byte offset of the kernel's window in a stage image: channel plane + window row shift}
@@ -325,7 +325,13 @@ __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable
     atomicMax(&bp.hdr->max_block_entries, tot);
   }
   char* base = bp.dblk + (size_t)off16 * 16;
-  reinterpret_cast<uint32_t*>(base)[lane] = active ? ((uint32_t)start | ((uint32_t)cur << 31)) : 0u;
+  // words 16-31: for consumer warp lane - 16, where the results of its two filters go inside the group's 32 output
+  // channels (original filter index modulo 32, filter A in bits 0-7, filter B in bits 8-15)
+  const int wo = lane - kBlockWarps;
+  const uint32_t where = active ? 0u
+      : ((uint32_t)bp.xfilt[g * kExecGroup + wo] & (uint32_t)(kExecGroup - 1)) |
+        (((uint32_t)bp.xfilt[g * kExecGroup + kExecGroup - 1 - wo] & (uint32_t)(kExecGroup - 1)) << 8);
+  reinterpret_cast<uint32_t*>(base)[lane] = active ? ((uint32_t)start | ((uint32_t)cur << 31)) : where;
   if (!active) return;
   uint4* ent = reinterpret_cast<uint4*>(base + kBlockHeaderBytes) + start;
   const uint2* tw4 = static_cast<const uint2*>(bp.tw4);
