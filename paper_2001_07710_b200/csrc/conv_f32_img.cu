@@ -150,12 +150,22 @@ __device__ __forceinline__ void lds_row_f32(float (&h)[16], uint32_t a, uint32_t
 // The code of one pattern on a 4 x 14 tile (see pattern_body4 in f16_tile.cuh): a0 = address of logical chunk 0 of
 // window row `sh`, swb = the lane's chunk swizzle (bits 4-5) for window rows 0-3; from window row 4 on the rows
 // belong to the next tile row's group, whose parity bit is the other one.
-template <uint32_t MASK>
+// S2 (stride 2): only the results at even rows and columns of the tile are wanted (tiles start at even image
+// coordinates), so the multiply-adds of the other three quarters and the window rows only they read are left out.
+__host__ __device__ constexpr bool row_used(uint32_t mask, int j, bool s2) {
+  for (int t = 0; t < 4; ++t) {
+    const int y = j - nth_bit(mask, t) / 3;
+    if (y >= 0 && y < TR4 && (!s2 || (y & 1) == 0)) return true;
+  }
+  return false;
+}
+template <uint32_t MASK, bool S2>
 __device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a0, uint32_t sh, uint32_t swb, const float (&w)[4],
                                                const float (&r0)[16]) {
   constexpr int NR = last_tap_row(MASK) + TR4;
 #pragma unroll
   for (int j = 0; j < NR; ++j) {
+    if (!row_used(MASK, j, S2)) continue;
     uint32_t x = swb;
     if (j >= 4) x ^= 32u;
     else if (j == 3) x ^= sh << 5;
@@ -170,15 +180,15 @@ __device__ __forceinline__ void pattern_body4f(float (&acc)[TR4][TC], uint32_t a
     for (int t = 0; t < 4; ++t) {
       const int b = nth_bit(MASK, t);
       const int y = j - b / 3, c = b % 3;
-      if (y >= 0 && y < TR4) {
+      if (y >= 0 && y < TR4 && (!S2 || (y & 1) == 0)) {
 #pragma unroll
-        for (int xx = 0; xx < TC; ++xx) acc[y][xx] = fmaf(h[xx + c], w[t], acc[y][xx]);
+        for (int xx = 0; xx < TC; xx += (S2 ? 2 : 1)) acc[y][xx] = fmaf(h[xx + c], w[t], acc[y][xx]);
       }
     }
   }
 }
 
-template <int NCODES, bool GENERIC>
+template <int NCODES, bool GENERIC, bool S2>
 __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t plane, uint32_t swb, uint32_t meta, uint32_t off,
                                              float (&w)[4], const float (&r0)[16]) {
   static_assert(NCODES == 6 || NCODES == kNumCodes, "code sets with compiled dispatch trees");
@@ -193,12 +203,12 @@ __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t pla
 #define PAT_TAP4F(B)                                                                         \
   if (meta & (16u << (B))) {                                                                 \
     _Pragma("unroll")                                                                        \
-    for (int y = 0; y < TR4; ++y) {                                                          \
+    for (int y = 0; y < TR4; y += (S2 ? 2 : 1)) {                                            \
       float h[16];                                                                           \
       const int jr = y + (B) / 3;                                                            \
       lds_row_f32(h, base + jr * ROWF, jr >= 4 ? (swb ^ 32u) : swb);                         \
       _Pragma("unroll")                                                                      \
-      for (int xx = 0; xx < TC; ++xx) acc[y][xx] = fmaf(h[xx + (B) % 3], w[0], acc[y][xx]);  \
+      for (int xx = 0; xx < TC; xx += (S2 ? 2 : 1)) acc[y][xx] = fmaf(h[xx + (B) % 3], w[0], acc[y][xx]);  \
     }                                                                                        \
     w[0] = w[1]; w[1] = w[2]; w[2] = w[3];                                                   \
   }
@@ -206,26 +216,26 @@ __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t pla
 #undef PAT_TAP4F
       }
     } else if constexpr (NCODES > 8) {
-      if (code & 1u) pattern_body4f<code_mask(9)>(acc, a0, sh, swb, w, r0);
-      else pattern_body4f<code_mask(8)>(acc, a0, sh, swb, w, r0);
+      if (code & 1u) pattern_body4f<code_mask(9), S2>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(8), S2>(acc, a0, sh, swb, w, r0);
     }
   } else if (code & 4u) {
     if (NCODES > 6 && (code & 2u)) {
       if constexpr (NCODES > 6) {
-        if (code & 1u) pattern_body4f<code_mask(7)>(acc, a0, sh, swb, w, r0);
-        else pattern_body4f<code_mask(6)>(acc, a0, sh, swb, w, r0);
+        if (code & 1u) pattern_body4f<code_mask(7), S2>(acc, a0, sh, swb, w, r0);
+        else pattern_body4f<code_mask(6), S2>(acc, a0, sh, swb, w, r0);
       }
     } else {
-      if (code & 1u) pattern_body4f<code_mask(5)>(acc, a0, sh, swb, w, r0);
-      else pattern_body4f<code_mask(4)>(acc, a0, sh, swb, w, r0);
+      if (code & 1u) pattern_body4f<code_mask(5), S2>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(4), S2>(acc, a0, sh, swb, w, r0);
     }
   } else {
     if (code & 2u) {
-      if (code & 1u) pattern_body4f<code_mask(3)>(acc, a0, sh, swb, w, r0);
-      else pattern_body4f<code_mask(2)>(acc, a0, sh, swb, w, r0);
+      if (code & 1u) pattern_body4f<code_mask(3), S2>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(2), S2>(acc, a0, sh, swb, w, r0);
     } else {
-      if (code & 1u) pattern_body4f<code_mask(1)>(acc, a0, sh, swb, w, r0);
-      else pattern_body4f<code_mask(0)>(acc, a0, sh, swb, w, r0);
+      if (code & 1u) pattern_body4f<code_mask(1), S2>(acc, a0, sh, swb, w, r0);
+      else pattern_body4f<code_mask(0), S2>(acc, a0, sh, swb, w, r0);
     }
   }
 }
@@ -234,7 +244,7 @@ __device__ __forceinline__ void one_kernel4f(float (&acc)[TR4][TC], uint32_t pla
 // Ring protocol as in conv_f16_img.cu: per work item nst stages of 8 channels, then two output stages whose slots
 // the consumers use as staging for the results - here twice (tile rows 0-1, then 2-3), with a block-wide barrier
 // after writing and after copying out the first pair of rows.
-template <bool SPARSE, int NCODES, bool GENERIC>
+template <bool SPARSE, int NCODES, bool GENERIC, bool S2>
 __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
   constexpr int NS = SPARSE ? 3 : 2;
   constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
@@ -383,7 +393,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           cur ^= 1u;
           fetch(cur, acc);
         }
-        one_kernel4f<NCODES, GENERIC>(acc, pl0, swb, cm, coff, w, r0);
+        one_kernel4f<NCODES, GENERIC, S2>(acc, pl0, swb, cm, coff, w, r0);
       stage_end:
         if (cm & kOpEnd) {
           __syncwarp();
@@ -514,7 +524,8 @@ __device__ __forceinline__ bool blob_matches(const Params& p) {
   return ok;
 }
 
-template <int NCODES, bool GENERIC>
+// S2: the stride-2 variant (a quarter of the multiply-adds, see pattern_body4f)
+template <int NCODES, bool GENERIC, bool S2>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f32_img(const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -526,8 +537,8 @@ k_conv_f32_img(const Params p) {
     return;
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC>(p, smem);
-  else conv_body<false, NCODES, GENERIC>(p, smem);
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC, S2>(p, smem);
+  else conv_body<false, NCODES, GENERIC, S2>(p, smem);
 }
 
 // ------------------------------------------------------------------------------------------ cut items
@@ -629,7 +640,9 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     variant = std::max(variant, code == kGenericCode ? 2 : (code >= 6 ? 1 : 0));
   }
   using KernelFn = void (*)(const Params);
-  static const KernelFn kernels[3] = {k_conv_f32_img<6, false>, k_conv_f32_img<kNumCodes, false>, k_conv_f32_img<kNumCodes, true>};
+  // [stride - 1][code set]
+  static const KernelFn kernels[6] = {k_conv_f32_img<6, false, false>, k_conv_f32_img<kNumCodes, false, false>, k_conv_f32_img<kNumCodes, true, false>,
+                                      k_conv_f32_img<6, false, true>, k_conv_f32_img<kNumCodes, false, true>, k_conv_f32_img<kNumCodes, true, true>};
 
   static thread_local DeviceSlot slots[kMaxDevices];
   DeviceSlot* dv = device_slot(slots);
@@ -675,7 +688,7 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   cudaLaunchConfig_t cfg = {};
   cfg.stream = st; cfg.attrs = &pdl; cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM_BYTES;
-  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant], p), "pat_conv3x3 launch")) return rc;
+  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[3 * p.sub + variant], p), "pat_conv3x3 launch")) return rc;
   count_launches(2);
   if (p.parts > 1) {
     cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * TC)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
