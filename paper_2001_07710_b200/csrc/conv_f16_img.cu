@@ -479,6 +479,16 @@ __device__ __forceinline__ bool blob_matches(const Params& p) {
   return ok;
 }
 
+// The same decision taken by a whole thread block at once (all loads in flight together, the masks spread over the
+// threads): one memory round trip at the start of a short kernel instead of a chain of them.
+__device__ __forceinline__ bool blob_matches_block(const Params& p) {
+  const BlobHeader* bh = p.hdr;
+  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
+            bh->K == p.K && bh->dtype == PAT_F16 && bh->n_keep == p.n_keep;
+  for (int j = threadIdx.x; j < p.K; j += blockDim.x) ok = ok && bh->masks[j] == p.masks[j];
+  return __syncthreads_and(ok) != 0;
+}
+
 // NCODES / GENERIC: the pattern codes the kernel carries code for (see one_kernel4); the host picks the smallest
 // set that covers the library.
 template <int NCODES, bool GENERIC>
@@ -510,7 +520,7 @@ constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
 constexpr int RP_THREADS = 1024, MAX_PARTS = 8, RP_XH = TC / 2;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");   // launched as a programmatic dependent of the convolution kernel
-  if (!blob_matches(p)) return;                          // the convolution kernel refused the blob and wrote no partial sums
+  if (!blob_matches_block(p)) return;                    // the convolution kernel refused the blob and wrote no partial sums
   __shared__ __align__(16) unsigned char stage[OUT_ROW];
   // block = (cut item, row of the thread tiles, left or right half of the tile columns)
   const int xh = (int)blockIdx.x & 1, y = ((int)blockIdx.x >> 1) % TR4, li = (int)blockIdx.x / (2 * TR4);

@@ -524,6 +524,16 @@ __device__ __forceinline__ bool blob_matches(const Params& p) {
   return ok;
 }
 
+// The same decision taken by a whole thread block at once (all loads in flight together, the masks spread over the
+// threads): one memory round trip at the start of a short kernel instead of a chain of them.
+__device__ __forceinline__ bool blob_matches_block(const Params& p) {
+  const BlobHeader* bh = p.hdr;
+  bool ok = bh->magic == kBlobMagic && bh->version == kBlobVersion && bh->F == p.F && bh->C == p.C &&
+            bh->K == p.K && bh->dtype == PAT_F32 && bh->n_keep == p.n_keep;
+  for (int j = threadIdx.x; j < p.K; j += blockDim.x) ok = ok && bh->masks[j] == p.masks[j];
+  return __syncthreads_and(ok) != 0;
+}
+
 // S2: the stride-2 variant (a quarter of the multiply-adds, see pattern_body4f)
 template <int NCODES, bool GENERIC, bool S2>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -549,7 +559,7 @@ constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
 constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (!blob_matches(p)) return;                          // the convolution kernel refused the blob and wrote no partial sums
+  if (!blob_matches_block(p)) return;                    // the convolution kernel refused the blob and wrote no partial sums
   const int v = (int)blockIdx.x % (TR4 * TC), li = (int)blockIdx.x / (TR4 * TC);
   const int item = p.n_whole + li;
   const int g = item % p.NG;
