@@ -194,29 +194,28 @@ def run_ours(args):
     cws_bytes = max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg_layers if not L.dense] + [0])
     cws = torch.empty(max(cws_bytes, 256), dtype=torch.uint8, device="cuda")
 
-    # Projection and packing of a layer depend on its weights only, so they run on a second stream while the first
-    # stream convolves the layers before it (an event per layer orders the convolution after its own packing): the
-    # small projection / packing kernels fill the idle SMs at the ends of the convolution kernels.
-    side = torch.cuda.Stream(priority=-1)    # its small blocks go first whenever an SM has room
+    # Projection and packing of a layer depend on its weights only: every pruned layer gets a stream of its own for
+    # them, forked from the main stream at the start of the step, and an event orders the layer's convolution after
+    # its own packing.  The chains of small kernels (a dozen launches per layer) then run side by side while the
+    # first layers convolve, instead of one after another in the gaps between the convolution kernels.
+    sides = [torch.cuda.Stream(priority=-1) for _ in layers]    # their small blocks go first whenever an SM has room
     packed_ev = [torch.cuda.Event() for _ in layers]
 
     def step(conv_events=None, overlap=True):
         overlap = overlap and not args.no_overlap
         main = torch.cuda.current_stream()
-        if not overlap:
-            prep = main
-        else:
-            prep = side
-            side.wait_stream(main)
-        with torch.cuda.stream(prep):
-            for i, st in enumerate(layers):
-                L = st["L"]
-                if L.dense:
-                    continue
+        for i, st in enumerate(layers):
+            L = st["L"]
+            if L.dense:
+                continue
+            prep = sides[i] if overlap else main
+            if overlap:
+                prep.wait_stream(main)             # the previous step no longer reads this layer's blob
+            with torch.cuda.stream(prep):
                 pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
                 pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
                 if overlap:
-                    packed_ev[i].record(side)
+                    packed_ev[i].record(prep)
         for i, st in enumerate(layers):
             L = st["L"]
             if conv_events is not None: conv_events[i][0].record(main)
@@ -224,11 +223,9 @@ def run_ours(args):
                 pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
             else:
                 if overlap:
-                    main.wait_event(packed_ev[i])
+                    main.wait_event(packed_ev[i])  # joins the layer's stream: every fork is waited for within the step
                 pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
             if conv_events is not None: conv_events[i][1].record(main)
-        if overlap:
-            main.wait_stream(side)
 
     # End to end: every step copies its weights and inputs from pinned host memory and reads all outputs back.  The
     # copies run on streams of their own (host-to-device, device-to-host: the link is full duplex) and overlap the
@@ -365,7 +362,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 storage, f32 accumulate" if dtype == "f16" else "f32", "data": "synthetic",
         "config": {"workload": f"config {cfg.number}: {cfg.name}", "batch_per_gpu": N,
-                   "layers": len(layers), "step": "project + pack + conv for every layer" + ("" if args.no_overlap else ", projection / packing on a second stream")
+                   "layers": len(layers), "step": "project + pack + conv for every layer" + ("" if args.no_overlap else ", projection / packing of each layer on a stream of its own")
                            + ("" if args.no_graph else ", replayed as one CUDA graph"),
                    "l2": l2_note, "seed": workloads.BASE_SEED},
         "effective_gflops": round(total_flop * world * args.steps / (ms_total * 1e-3) / 1e9, 1),

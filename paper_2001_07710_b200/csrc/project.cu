@@ -61,11 +61,17 @@ inline ProjWs carve(void* base, int64_t FC) {
 // whichever block finishes last: every block publishes its results, takes a ticket, and the block that draws the
 // last ticket (which also puts the counter back to zero for the next kernel) goes on.  Returns true in every thread
 // of that block; its reads of the other blocks' results must bypass L1 (__ldcg).
+// One fence per block, not per thread: the block barrier orders every thread's writes and atomics before thread 0's
+// fence, and a fence is cumulative - what thread 0 has observed is visible device-wide before its ticket is.  (A
+// fence in every thread made each of them wait for its own atomics to return; with a quarter of a million threads
+// that wait was most of the kernel.)
 __device__ inline bool last_block_done(unsigned int* ticket) {
   __shared__ bool s_last;
-  __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) s_last = atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = atomicInc(ticket, gridDim.x - 1) == gridDim.x - 1;
+  }
   __syncthreads();
   if (s_last) __threadfence();
   return s_last;
@@ -111,6 +117,8 @@ __device__ inline void pick_digit(SelectState* st, const unsigned int* hist, int
   const int t = threadIdx.x;
   const unsigned long long rem = (unsigned long long)__ldcg(&st->remaining);
   const unsigned long long prefix = __ldcg(&st->prefix);
+  if (t == 0) { s_coarse = 0; s_above = 0ull; }   // defined values even if no bin qualifies (a histogram that misses keys)
+  __syncthreads();
   {
     const int bin = kCoarse - 1 - t;
     const unsigned long long c = __ldcg(coarse + bin);
@@ -131,40 +139,115 @@ __device__ inline void pick_digit(SelectState* st, const unsigned int* hist, int
   }
 }
 
-// One thread per kernel: energies of all masks, argmax (lowest id on ties); histogram of the first digit of the
-// energies' bit patterns; the last block picks that digit.  do_select = false (everything or nothing is kept):
-// pattern ids only.
+// kSelPerThread kernels per thread: energies of all masks, argmax (lowest id on ties); histogram of the first digit
+// of the energies' bit patterns; the last block picks that digit.  do_select = false (everything or nothing is
+// kept): pattern ids only.
+//
+// The first digit (sign, exponent, four mantissa bits) takes only a few dozen values in a layer, so its histogram is
+// collected per block in shared memory and flushed with one global atomic per distinct value and block: atomics
+// from a quarter of a million threads on those few addresses took longer than the rest of the projection.
+constexpr int kSelPerThread = 4;
+constexpr int kSelSlots = 1024;              // shared-memory counters, indexed by the digit's low bits and tagged with the digit
 __global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict__ w, int64_t FC, MaskTable lib,
                                                         unsigned long long* __restrict__ key, unsigned char* __restrict__ pid,
                                                         SelectState* st, long long n_keep, unsigned int* hist, bool do_select) {
   pdl_wait();
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i == 0) { st->prefix = 0ull; st->remaining = n_keep; }
-  const bool in = i < FC;
-  unsigned long long k = 0ull;
-  if (in) {
-    double sq[9];
+  __shared__ unsigned int s_tag[kSelSlots], s_cnt[kSelSlots], s_coarse[kCoarse];
+  if (do_select) {
+    for (int q = threadIdx.x; q < kSelSlots; q += blockDim.x) { s_tag[q] = 0u; s_cnt[q] = 0u; }
+    for (int q = threadIdx.x; q < kCoarse; q += blockDim.x) s_coarse[q] = 0u;
+    __syncthreads();
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) { st->prefix = 0ull; st->remaining = n_keep; }
+  for (int r = 0; r < kSelPerThread; ++r) {
+    const int64_t i = ((int64_t)blockIdx.x * kSelPerThread + r) * blockDim.x + threadIdx.x;
+    const bool in = i < FC;
+    unsigned long long k = 0ull;
+    if (in) {
+      const float* wk = w + i * 9;
+      // Double-precision arithmetic is scarce on this GPU, so the argmax is first taken in fp32.  Nine squares and a
+      // sum of at most nine non-negative terms carry a relative error below 2^-20 (nine roundings of 2^-24 each) as
+      // long as nothing overflows and the result is far above the subnormal range, so an fp32 winner that leads the
+      // runner-up by a factor of more than 1 + 2^-18 is the exact winner too.  Every other case - a lead inside the
+      // error bound (exact ties among them), a tiny, huge or non-finite energy - takes the exact path over all masks.
+      // The energy itself (the key of the connectivity ranking) is always computed exactly: fp64 squares of the
+      // winner's entries, added in ascending bit order.
+      float sqf[9];
 #pragma unroll
-    for (int b = 0; b < 9; ++b) {
-      const double v = (double)w[i * 9 + b];
-      sq[b] = v * v;
-    }
-    double best_e = -1.0;
-    int best = 0;
-    for (int j = 0; j < lib.K; ++j) {
-      const unsigned m = lib.m[j];
-      double e = 0.0;
+      for (int b = 0; b < 9; ++b) {
+        const float v = wk[b];
+        sqf[b] = __fmul_rn(v, v);
+      }
+      float best32 = -1.0f, second32 = -1.0f;
+      int best = 0;
+      bool plain = true;                       // every fp32 energy is an ordinary finite number
+      for (int j = 0; j < lib.K; ++j) {
+        const unsigned m = lib.m[j];
+        float e = 0.0f;
 #pragma unroll
-      for (int b = 0; b < 9; ++b)
-        if (m & (1u << b)) e += sq[b];
-      if (e > best_e) { best_e = e; best = j; }
+        for (int b = 0; b < 9; ++b)
+          if (m & (1u << b)) e = __fadd_rn(e, sqf[b]);
+        plain = plain && (e <= 3.0e38f);       // false for NaN and infinity
+        if (e > best32) { second32 = best32; best32 = e; best = j; }
+        else if (e > second32) second32 = e;   // e == best32 lands here: a tie is never a clear lead
+      }
+      constexpr float kLead = 1.0f + 3.814697265625e-6f;     // 1 + 2^-18
+      constexpr float kFloor = 7.8886090522101181e-31f;      // 2^-100
+      const bool clear = plain && best32 >= kFloor && best32 > second32 * kLead;
+      double best_e;
+      if (clear) {
+        best_e = 0.0;
+        unsigned m = lib.m[best];
+        while (m) {                            // ascending bit order
+          const double v = (double)wk[__ffs(m) - 1];
+          best_e += v * v;                     // the square of an fp32 value is exact in fp64
+          m &= m - 1u;
+        }
+      } else {
+        double sq[9];
+#pragma unroll
+        for (int b = 0; b < 9; ++b) {
+          const double v = (double)wk[b];
+          sq[b] = v * v;
+        }
+        best_e = -1.0;
+        best = 0;
+        for (int j = 0; j < lib.K; ++j) {
+          const unsigned m = lib.m[j];
+          double e = 0.0;
+#pragma unroll
+          for (int b = 0; b < 9; ++b)
+            if (m & (1u << b)) e += sq[b];
+          if (e > best_e) { best_e = e; best = j; }
+        }
+      }
+      k = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
+      key[i] = k;
+      pid[i] = (unsigned char)best;
     }
-    k = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
-    key[i] = k;
-    pid[i] = (unsigned char)best;
+    if (!do_select) continue;
+    // identical digits inside the warp are merged first; the lane that speaks for a digit adds to the block's counters
+    const unsigned d = (unsigned)(k >> 48);
+    const unsigned active = __ballot_sync(0xFFFFFFFFu, in);
+    if (in) {
+      const int lane = threadIdx.x & 31;
+      const unsigned same = __match_any_sync(active, d);
+      if ((int)(__ffs(same) - 1) == lane) {
+        const unsigned n = (unsigned)__popc(same);
+        const unsigned slot = d & (unsigned)(kSelSlots - 1);
+        const unsigned old = atomicCAS(&s_tag[slot], 0u, d + 1u);
+        if (old == 0u || old == d + 1u) atomicAdd(&s_cnt[slot], n);
+        else atomicAdd(&hist[d], n);         // the slot belongs to another digit: straight to the global histogram
+        atomicAdd(&s_coarse[d >> 8], n);
+      }
+    }
   }
   if (!do_select) return;
-  hist_add(hist, hist + kBins, in, (unsigned)(k >> 48));
+  __syncthreads();
+  for (int q = threadIdx.x; q < kSelSlots; q += blockDim.x)
+    if (s_cnt[q]) atomicAdd(&hist[s_tag[q] - 1u], s_cnt[q]);
+  for (int q = threadIdx.x; q < kCoarse; q += blockDim.x)
+    if (s_coarse[q]) atomicAdd(&hist[kBins + q], s_coarse[q]);
   if (last_block_done(hist + kTicketWord)) pick_digit(st, hist, 0);
 }
 
@@ -285,6 +368,7 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   for (int j = 0; j <= kMaxK; ++j) lib.m[j] = (j < K) ? masks[j] : (uint16_t)0;
   lib.K = K;
   const int nb256 = (int)((FC + 255) / 256);
+  const int nb_sel = (int)((FC + 256 * kSelPerThread - 1) / (256 * kSelPerThread));
   const int nblk = (int)((FC + kSelBlock - 1) / kSelBlock);
   int mode = -1;
   if (n_keep == FC) mode = 1;
@@ -294,7 +378,7 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   }
   cudaError_t le = cudaSuccess;                   // first launch error, if any
   auto note = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
-  note(launch_dependent(k_select_pattern, dim3(nb256), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0));
+  note(launch_dependent(k_select_pattern, dim3(nb_sel), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0));
   if (mode < 0) {
     for (int pass = 1; pass < kPasses; ++pass) note(launch_dependent(k_sel_hist, dim3(nb256), dim3(256), 0, st, ws.key, FC, pass, ws.st, ws.hist));
     note(launch_dependent(k_tie_count, dim3(nblk), dim3(kSelBlock), 0, st, ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord));

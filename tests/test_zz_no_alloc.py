@@ -5,6 +5,8 @@ plug-ins inside another allocator, loops that must not trigger an allocation's d
 The file is named so that pytest collects it last: a run that stops at the first failure has then already
 run every other test.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -31,13 +33,14 @@ def _run_both(seed, F, C, K, n_keep):
     pc.pat_project_static(w, masks, n_keep, pid, wm)
     pid.fill_(0x5A)
     wm.fill_(float("nan"))
+    gc.collect()                                    # tensors that earlier tests left in reference cycles go now, not inside the window
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()          # torch's allocator ...
     torch.cuda.reset_peak_memory_stats()            # ... and its high-water mark from here on
     free_before = torch.cuda.mem_get_info()[0]      # the driver's view (cudaMemGetInfo): sees any cudaMalloc
     pc.pat_project_static(w, masks, n_keep, pid, wm)
     torch.cuda.synchronize()
-    assert torch.cuda.max_memory_allocated() == before and torch.cuda.memory_allocated() == before
+    assert torch.cuda.max_memory_allocated() == before and torch.cuda.memory_allocated() <= before
     assert torch.cuda.mem_get_info()[0] == free_before
     assert pc.pat_query_status() == 0
     # against the oracle (brute force over the library, sort for connectivity): bit for bit
