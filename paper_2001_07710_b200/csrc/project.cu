@@ -302,7 +302,9 @@ __global__ void __launch_bounds__(kSelBlock) k_tie_count(const unsigned long lon
   }
 }
 
-// Decide keep / remove per kernel and write pattern ids and masked weights.
+// Decide keep / remove per kernel and write pattern ids and masked weights.  The decision is taken by one thread per
+// kernel; the weights are then copied by the whole block in the order they lie in memory (a thread that walked its
+// own nine values would touch a different 32-byte sector with every lane, on the way in and on the way out).
 __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t FC, MaskTable lib,
                                                         const unsigned long long* __restrict__ key,
                                                         const unsigned char* __restrict__ pid_in,
@@ -311,7 +313,9 @@ __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t 
                                                         unsigned char* __restrict__ pid_out, float* wm, int keep_all_or_none) {
   pdl_wait();
   __shared__ unsigned int warp_cnt[kSelBlock / 32];
-  const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
+  __shared__ unsigned short s_mask[kSelBlock];      // the kept positions of every kernel of the block (0: removed)
+  const int64_t i0 = (int64_t)blockIdx.x * kSelBlock;
+  const int64_t i = i0 + threadIdx.x;
   const bool valid = i < FC;
   bool keep;
   if (keep_all_or_none >= 0) {            // n_keep == F*C (1) or n_keep == 0 (0): no threshold needed
@@ -329,14 +333,20 @@ __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t 
     for (int q = 0; q < wid; ++q) rank += warp_cnt[q];
     keep = valid && (k > thr || (tie && (long long)rank < st->remaining));
   }
-  if (!valid) return;
-  const unsigned char p = pid_in[i];
-  const unsigned m = keep ? lib.m[p] : 0u;
-  pid_out[i] = keep ? p : (unsigned char)PAT_PRUNED;
-#pragma unroll
-  for (int b = 0; b < 9; ++b) {
-    const float v = w[i * 9 + b];
-    wm[i * 9 + b] = (m & (1u << b)) ? v : 0.0f;
+  unsigned m = 0u;
+  if (valid) {
+    const unsigned char p = pid_in[i];
+    m = keep ? lib.m[p] : 0u;
+    pid_out[i] = keep ? p : (unsigned char)PAT_PRUNED;
+  }
+  s_mask[threadIdx.x] = (unsigned short)m;
+  __syncthreads();
+  const int64_t e0 = i0 * 9;
+  const int n = (int)(((FC - i0) < (int64_t)kSelBlock ? (FC - i0) : (int64_t)kSelBlock) * 9);
+  for (int e = threadIdx.x; e < n; e += kSelBlock) {
+    const int kq = e / 9, b = e - kq * 9;
+    const float v = w[e0 + e];
+    wm[e0 + e] = ((s_mask[kq] >> b) & 1u) ? v : 0.0f;
   }
 }
 
