@@ -5,10 +5,11 @@
 // Connectivity pruning ranks kernels by their L2 norm (Section 6.1) and keeps the n_keep strongest of the layer.
 //
 // Exactness: squares of fp32 values are exact in fp64 and are added in ascending bit order, so the energies
-// are the same bits on any IEEE machine.  The n_keep-th largest energy is found with a 4-pass, 16-bit radix
-// select over the (monotone) bit pattern of the non-negative doubles; ties at the threshold are resolved by
-// index with a block scan.  Six launches per layer: the step after each histogram (and after the tie counts)
-// that needs all blocks' results is done by the block that finishes last.
+// are the same bits on any IEEE machine.  The n_keep-th largest energy is found with a radix select over the
+// (monotone) bit pattern of the non-negative doubles: two 16-bit digits by histograms over the whole layer (the
+// second one also lists the keys that share the first digit with the threshold), the remaining 32 bits and the
+// index that separates kept from removed ties by one thread block over that list.  Three launches per layer: the
+// steps that need all blocks' results are done by the block that finishes last.
 #include "common.cuh"
 
 namespace pat {
@@ -18,21 +19,24 @@ constexpr int kSelBlock = 1024;
 constexpr int kBins = 65536;
 
 struct SelectState {
-  unsigned long long prefix;   // bits of the threshold key decided so far
+  unsigned long long prefix;   // bits of the threshold key decided so far; in the end the threshold itself
   long long remaining;         // how many keys with this prefix (and below-decided digits) are still to be kept
+  unsigned int cut;            // kernels whose key equals the threshold are kept up to this index
+  unsigned int pad;
 };
 
 // workspace layout
 constexpr int kCoarse = 256;                 // coarse histogram: the upper 8 bits of a 16-bit digit
-constexpr int kPasses = 4;                   // 64-bit keys, 16 bits per pass
-constexpr size_t kHistWords = (size_t)kPasses * (kBins + kCoarse) + 4;   // one fine + one coarse histogram per pass, then the block tickets
+constexpr int kPasses = 2;                   // digits found with histograms over the whole layer (16 bits each)
+constexpr size_t kHistWords = (size_t)kPasses * (kBins + kCoarse) + 4;   // one fine + one coarse histogram per pass, then two control words
 constexpr size_t kTicketWord = (size_t)kPasses * (kBins + kCoarse);     // hist[kTicketWord]: blocks of the running kernel that are done
+constexpr size_t kListWord = kTicketWord + 1;                             // hist[kListWord]: length of the candidate list
 
 struct ProjWs {
   unsigned long long* key;     // [FC] energy bit patterns
   unsigned char* pid;          // [FC] best pattern per kernel
   unsigned int* hist;          // [kPasses][65536 fine | 256 coarse]; zeroed by every call
-  unsigned int* blk;           // [nblk + 1] tie counts per block, then exclusive offsets
+  unsigned int* cand;          // [FC] indices of the keys that share the first digit with the threshold (any order)
   SelectState* st;
   size_t bytes;
 };
@@ -40,7 +44,7 @@ struct ProjWs {
 constexpr size_t ws_align(size_t x) { return (x + 255) & ~size_t(255); }
 constexpr size_t ws_bytes(int64_t FC) {
   return ws_align(8 * (size_t)FC) + ws_align((size_t)FC) + ws_align(4 * kHistWords) +
-         ws_align(4 * ((size_t)((FC + kSelBlock - 1) / kSelBlock) + 1)) + ws_align(sizeof(SelectState));
+         ws_align(4 * (size_t)FC) + ws_align(sizeof(SelectState));
 }
 
 inline ProjWs carve(void* base, int64_t FC) {
@@ -50,14 +54,14 @@ inline ProjWs carve(void* base, int64_t FC) {
   w.key = reinterpret_cast<unsigned long long*>(p + o); o += ws_align(8 * (size_t)FC);
   w.pid = reinterpret_cast<unsigned char*>(p + o);      o += ws_align((size_t)FC);
   w.hist = reinterpret_cast<unsigned int*>(p + o);      o += ws_align(4 * kHistWords);
-  w.blk = reinterpret_cast<unsigned int*>(p + o);       o += ws_align(4 * ((size_t)((FC + kSelBlock - 1) / kSelBlock) + 1));
+  w.cand = reinterpret_cast<unsigned int*>(p + o);      o += ws_align(4 * (size_t)FC);
   w.st = reinterpret_cast<SelectState*>(p + o);         o += ws_align(sizeof(SelectState));
   w.bytes = o;
   return w;
 }
 
 // The selection kernels end with a step that needs the work of all their blocks (choosing the digit from the
-// complete histogram, scanning the per-block tie counts).  Instead of a launch of its own that step is done by
+// complete histogram, finishing the selection on the candidate list).  Instead of a launch of its own that step is done by
 // whichever block finishes last: every block publishes its results, takes a ticket, and the block that draws the
 // last ticket (which also puts the counter back to zero for the next kernel) goes on.  Returns true in every thread
 // of that block; its reads of the other blocks' results must bypass L1 (__ldcg).
@@ -90,7 +94,7 @@ __device__ inline void hist_add(unsigned int* fine, unsigned int* coarse, bool i
   }
 }
 
-// Inclusive scan over the 256 threads of a block, thread 0 first.
+// Inclusive scan over the threads of a block (any size up to 1024; warp_tot: 32 words), thread 0 first.
 __device__ inline unsigned long long block_scan_256(unsigned long long v, unsigned long long* warp_tot) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 #pragma unroll
@@ -106,33 +110,34 @@ __device__ inline unsigned long long block_scan_256(unsigned long long v, unsign
   return v + add;
 }
 
-// One block of 256 threads: find the digit d with  count(digit > d) < remaining <= count(digit >= d), first in
+// One block of 256 threads or more: find the digit d with  count(digit > d) < remaining <= count(digit >= d), first in
 // the coarse histogram, then among the 256 fine bins of the coarse bin found.  Thread 0 owns the highest bin.
 __device__ inline void pick_digit(SelectState* st, const unsigned int* hist, int pass) {
-  __shared__ unsigned long long warp_tot[8];
+  __shared__ unsigned long long warp_tot[32];
   __shared__ int s_coarse;
   __shared__ unsigned long long s_above;
   const unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
   const unsigned int* coarse = fine + kBins;
   const int t = threadIdx.x;
+  const bool owner = t < kCoarse;            // threads beyond the first 256 only take part in the scans
   const unsigned long long rem = (unsigned long long)__ldcg(&st->remaining);
   const unsigned long long prefix = __ldcg(&st->prefix);
   if (t == 0) { s_coarse = 0; s_above = 0ull; }   // defined values even if no bin qualifies (a histogram that misses keys)
   __syncthreads();
   {
     const int bin = kCoarse - 1 - t;
-    const unsigned long long c = __ldcg(coarse + bin);
+    const unsigned long long c = owner ? __ldcg(coarse + bin) : 0ull;
     const unsigned long long incl = block_scan_256(c, warp_tot);
-    if (rem > incl - c && rem <= incl) { s_coarse = bin; s_above = incl - c; }
+    if (owner && rem > incl - c && rem <= incl) { s_coarse = bin; s_above = incl - c; }
   }
   __syncthreads();
   const int cb = s_coarse;
   const unsigned long long above = s_above;
   {
     const int bin = cb * 256 + (255 - t);
-    const unsigned long long c = __ldcg(fine + bin);
+    const unsigned long long c = owner ? __ldcg(fine + bin) : 0ull;
     const unsigned long long incl = above + block_scan_256(c, warp_tot);
-    if (rem > incl - c && rem <= incl) {
+    if (owner && rem > incl - c && rem <= incl) {
       st->prefix = (prefix << 16) | (unsigned long long)bin;
       st->remaining = (long long)(rem - (incl - c));
     }
@@ -251,55 +256,116 @@ __global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict_
   if (last_block_done(hist + kTicketWord)) pick_digit(st, hist, 0);
 }
 
-// Histogram of the current 16-bit digit over the keys that match the decided prefix; the last block picks the digit.
-__global__ void __launch_bounds__(256) k_sel_hist(const unsigned long long* __restrict__ key, int64_t FC, int pass,
-                                                  SelectState* st, unsigned int* hist) {
+// Among 256 counters (one per thread of the first 256; the others pass 0), the bin where the running count - taken
+// from the highest bin down (DESCENDING) or from the lowest bin up - first reaches `rem`.  Returns the bin and sets
+// `before` to the count of the bins passed on the way.  All threads of the block call it; `cnt` is this thread's bin
+// (thread t owns bin 255 - t when descending, bin t otherwise).
+template <bool DESCENDING>
+__device__ inline int pick_bin_256(unsigned long long cnt, unsigned long long rem, unsigned long long* warp_tot,
+                                   unsigned long long& before) {
+  __shared__ int s_bin;
+  __shared__ unsigned long long s_before;
+  if (threadIdx.x == 0) { s_bin = 0; s_before = 0ull; }
+  __syncthreads();
+  const unsigned long long incl = block_scan_256(cnt, warp_tot);
+  if (threadIdx.x < 256 && rem > incl - cnt && rem <= incl) { s_bin = DESCENDING ? 255 - (int)threadIdx.x : (int)threadIdx.x; s_before = incl - cnt; }
+  __syncthreads();
+  before = s_before;
+  const int bin = s_bin;
+  __syncthreads();                           // the shared results may be overwritten by the next call
+  return bin;
+}
+
+// Second digit and everything after it.  All blocks: histogram of the second 16-bit digit over the keys whose first
+// digit is the threshold's, and a list of those keys' indices (any order).  The last block picks the second digit
+// and then works alone: it gathers from the list the keys that agree with the threshold in both digits (a handful
+// for ordinary weights; they stay in shared memory - if there are more than fit, the passes below walk the list
+// itself), finds the remaining 32 bits of the threshold in four 8-bit passes with a histogram in shared memory and
+// then, among the keys equal to the threshold, the index below which `remaining` of them lie (four more passes,
+// over the index bits).  Kernels whose key equals the threshold are kept in index order.
+constexpr int kRestThreads = 1024;
+constexpr int kShortList = 2048;
+static_assert(kRestThreads == kSelBlock, "launched with one block per kSelBlock kernels");
+__global__ void __launch_bounds__(kRestThreads) k_select_rest(const unsigned long long* __restrict__ key, int64_t FC,
+                                                              SelectState* st, unsigned int* hist, unsigned int* cand) {
   pdl_wait();
+  __shared__ unsigned long long warp_tot[32];
+  __shared__ unsigned int s_hist[256];
+  __shared__ unsigned long long s_key[kShortList];
+  __shared__ unsigned int s_idx[kShortList];
+  __shared__ unsigned int s_n;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int shift = 48 - 16 * pass;
   bool in = i < FC;
   unsigned d = 0;
   if (in) {
     const unsigned long long k = key[i];
-    in = (k >> (shift + 16)) == st->prefix;
-    d = (unsigned)((k >> shift) & 0xFFFFull);
+    in = (k >> 48) == st->prefix;
+    d = (unsigned)((k >> 32) & 0xFFFFull);
   }
-  unsigned int* fine = hist + (size_t)pass * (kBins + kCoarse);
+  unsigned int* fine = hist + (size_t)(kBins + kCoarse);
   hist_add(fine, fine + kBins, in, d);
-  if (last_block_done(hist + kTicketWord)) pick_digit(st, hist, pass);
-}
-
-// Ties at the threshold: count per block of 1024 consecutive kernels; the last block turns the counts into
-// exclusive offsets (sequential over chunks of 1024 blocks).
-__global__ void __launch_bounds__(kSelBlock) k_tie_count(const unsigned long long* __restrict__ key, int64_t FC,
-                                                         const SelectState* __restrict__ st, unsigned int* blk, int nblk,
-                                                         unsigned int* ticket) {
-  pdl_wait();
-  __shared__ unsigned int part[kSelBlock];
-  __shared__ unsigned int carry;
-  const int64_t i = (int64_t)blockIdx.x * kSelBlock + threadIdx.x;
-  const int tie = (i < FC && key[i] == st->prefix) ? 1 : 0;
-  const int n = __syncthreads_count(tie);
-  if (threadIdx.x == 0) blk[blockIdx.x] = (unsigned)n;
-  if (!last_block_done(ticket)) return;
-  if (threadIdx.x == 0) carry = 0u;
-  __syncthreads();
-  for (int base = 0; base < nblk; base += kSelBlock) {
-    const int q = base + threadIdx.x;
-    const unsigned int v = (q < nblk) ? __ldcg(blk + q) : 0u;
-    part[threadIdx.x] = v;
-    __syncthreads();
-    for (int off = 1; off < kSelBlock; off <<= 1) {
-      unsigned int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0u;
-      __syncthreads();
-      part[threadIdx.x] += a;
-      __syncthreads();
-    }
-    if (q < nblk) blk[q] = carry + part[threadIdx.x] - v;
-    __syncthreads();
-    if (threadIdx.x == kSelBlock - 1) carry += part[kSelBlock - 1];
-    __syncthreads();
+  {
+    const unsigned active = __ballot_sync(0xFFFFFFFFu, in);
+    const int lane = threadIdx.x & 31;
+    unsigned base = 0u;
+    if (active && lane == (int)(__ffs(active) - 1)) base = atomicAdd(&hist[kListWord], (unsigned)__popc(active));
+    if (active) base = __shfl_sync(0xFFFFFFFFu, base, __ffs(active) - 1);
+    if (in) cand[base + __popc(active & ((1u << lane) - 1u))] = (unsigned)i;
   }
+  if (!last_block_done(hist + kTicketWord)) return;
+  pick_digit(st, hist, 1);
+  const int t = threadIdx.x;
+  if (t == 0) s_n = 0u;
+  __syncthreads();
+  unsigned long long prefix = __ldcg(&st->prefix);             // 32 bits decided
+  unsigned long long rem = (unsigned long long)__ldcg(&st->remaining);
+  const unsigned n = __ldcg(&hist[kListWord]);
+  for (unsigned j = t; j < n; j += kRestThreads) {
+    const unsigned idx = __ldcg(cand + j);
+    const unsigned long long k = key[idx];
+    if ((k >> 32) == prefix) {
+      const unsigned pos = atomicAdd(&s_n, 1u);
+      if (pos < (unsigned)kShortList) { s_key[pos] = k; s_idx[pos] = idx; }
+    }
+  }
+  __syncthreads();
+  const bool fits = s_n <= (unsigned)kShortList;
+  const unsigned m = fits ? s_n : n;
+  auto entry = [&](unsigned j, unsigned long long& k, unsigned& idx) {
+    if (fits) { k = s_key[j]; idx = s_idx[j]; }
+    else { idx = __ldcg(cand + j); k = key[idx]; }
+  };
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (t < 256) s_hist[t] = 0u;
+    __syncthreads();
+    for (unsigned j = t; j < m; j += kRestThreads) {
+      unsigned long long k; unsigned idx;
+      entry(j, k, idx);
+      if ((k >> (shift + 8)) == prefix) atomicAdd(&s_hist[(unsigned)(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    unsigned long long above;
+    const int bin = pick_bin_256<true>(t < 256 ? s_hist[255 - t] : 0u, rem, warp_tot, above);
+    prefix = (prefix << 8) | (unsigned long long)bin;
+    rem -= above;
+  }
+  // prefix is the threshold now and rem (>= 1) the number of keys equal to it that are kept: the rem lowest indices
+  unsigned long long ipre = 0ull;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (t < 256) s_hist[t] = 0u;
+    __syncthreads();
+    for (unsigned j = t; j < m; j += kRestThreads) {
+      unsigned long long k; unsigned idx;
+      entry(j, k, idx);
+      if (k == prefix && ((unsigned long long)idx >> (shift + 8)) == ipre) atomicAdd(&s_hist[(idx >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    unsigned long long below;
+    const int bin = pick_bin_256<false>(t < 256 ? s_hist[t] : 0u, rem, warp_tot, below);
+    ipre = (ipre << 8) | (unsigned long long)bin;
+    rem -= below;
+  }
+  if (t == 0) { st->prefix = prefix; st->cut = (unsigned int)ipre; }
 }
 
 // Decide keep / remove per kernel and write pattern ids and masked weights.  The decision is taken by one thread per
@@ -309,10 +375,8 @@ __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t 
                                                         const unsigned long long* __restrict__ key,
                                                         const unsigned char* __restrict__ pid_in,
                                                         const SelectState* __restrict__ st,
-                                                        const unsigned int* __restrict__ blk,
                                                         unsigned char* __restrict__ pid_out, float* wm, int keep_all_or_none) {
   pdl_wait();
-  __shared__ unsigned int warp_cnt[kSelBlock / 32];
   __shared__ unsigned short s_mask[kSelBlock];      // the kept positions of every kernel of the block (0: removed)
   const int64_t i0 = (int64_t)blockIdx.x * kSelBlock;
   const int64_t i = i0 + threadIdx.x;
@@ -323,15 +387,7 @@ __global__ void __launch_bounds__(kSelBlock) k_finalize(const float* w, int64_t 
   } else {
     const unsigned long long thr = st->prefix;
     const unsigned long long k = valid ? key[i] : 0ull;
-    const bool tie = valid && k == thr;
-    // rank of this tie among all ties in index order
-    const unsigned ballot = __ballot_sync(0xFFFFFFFFu, tie);
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    if (lane == 0) warp_cnt[wid] = __popc(ballot);
-    __syncthreads();
-    unsigned rank = blk[blockIdx.x] + __popc(ballot & ((1u << lane) - 1u));
-    for (int q = 0; q < wid; ++q) rank += warp_cnt[q];
-    keep = valid && (k > thr || (tie && (long long)rank < st->remaining));
+    keep = valid && (k > thr || (k == thr && (unsigned int)i <= st->cut));   // ties: lowest indices first
   }
   unsigned m = 0u;
   if (valid) {
@@ -377,7 +433,6 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   MaskTable lib;
   for (int j = 0; j <= kMaxK; ++j) lib.m[j] = (j < K) ? masks[j] : (uint16_t)0;
   lib.K = K;
-  const int nb256 = (int)((FC + 255) / 256);
   const int nb_sel = (int)((FC + 256 * kSelPerThread - 1) / (256 * kSelPerThread));
   const int nblk = (int)((FC + kSelBlock - 1) / kSelBlock);
   int mode = -1;
@@ -390,11 +445,10 @@ extern "C" int pat_project(const float* w, int F, int C, const uint16_t* masks, 
   auto note = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
   note(launch_dependent(k_select_pattern, dim3(nb_sel), dim3(256), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, (long long)n_keep, ws.hist, mode < 0));
   if (mode < 0) {
-    for (int pass = 1; pass < kPasses; ++pass) note(launch_dependent(k_sel_hist, dim3(nb256), dim3(256), 0, st, ws.key, FC, pass, ws.st, ws.hist));
-    note(launch_dependent(k_tie_count, dim3(nblk), dim3(kSelBlock), 0, st, ws.key, FC, ws.st, ws.blk, nblk, ws.hist + kTicketWord));
+    note(launch_dependent(k_select_rest, dim3(nblk), dim3(kRestThreads), 0, st, ws.key, FC, ws.st, ws.hist, ws.cand));
   }
-  note(launch_dependent(k_finalize, dim3(nblk), dim3(kSelBlock), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, ws.blk, pattern_id, w_masked, mode));
-  count_launches(mode < 0 ? 6 : 2);
+  note(launch_dependent(k_finalize, dim3(nblk), dim3(kSelBlock), 0, st, w, FC, lib, ws.key, ws.pid, ws.st, pattern_id, w_masked, mode));
+  count_launches(mode < 0 ? 3 : 2);
   if (le != cudaSuccess) return check_cuda(le, "pat_project launch");
   return check_cuda(cudaGetLastError(), "pat_project launch");
 }
