@@ -111,56 +111,59 @@ __global__ void __launch_bounds__(128) k_pack_rank(int F, int K, BlobPtrs bp) {
   }
 }
 
-// One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
-__global__ void __launch_bounds__(1024) k_pack_ptrs(int F, int C, int K, long long n_keep, int dtype, MaskTable lib,
-                                                    unsigned long long total_bytes, BlobPtrs bp, int* status) {
-  pdl_wait();
-  __shared__ int part[1024];
-  __shared__ int carry;
-  if (threadIdx.x == 0) carry = 0;
+// Inclusive scan over the threads of a block (up to 1024; warp_tot: 32 words), thread 0 first: shuffles inside a
+// warp, the warp totals through shared memory.
+__device__ inline int block_scan_int(int v, int* warp_tot) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int u = __shfl_up_sync(0xFFFFFFFFu, v, off);
+    if (lane >= off) v += u;
+  }
+  if (lane == 31) warp_tot[wid] = v;
   __syncthreads();
-  for (int base = 0; base < F; base += 1024) {
+  int add = 0;
+  for (int q = 0; q < wid; ++q) add += warp_tot[q];
+  __syncthreads();
+  return v + add;
+}
+
+// One block: fptr = exclusive scan of kept counts in the new order; pattern segment pointers; header.
+constexpr int kPtrsThreads = 512;
+__global__ void __launch_bounds__(kPtrsThreads) k_pack_ptrs(int F, int C, int K, long long n_keep, int dtype, MaskTable lib,
+                                                            unsigned long long total_bytes, BlobPtrs bp, int* status) {
+  pdl_wait();
+  __shared__ int warp_tot[32];
+  __shared__ int s_total;
+  int carry = 0;                           // kept kernels of the filters in earlier chunks (the same in every thread)
+  for (int base = 0; base < F; base += kPtrsThreads) {
     const int q = base + threadIdx.x;
     const int v = (q < F) ? bp.cnt[bp.perm[q]] : 0;
-    part[threadIdx.x] = v;
-    __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-      const int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0;
-      __syncthreads();
-      part[threadIdx.x] += a;
-      __syncthreads();
-    }
+    const int incl = block_scan_int(v, warp_tot);
     if (q < F) {
-      const int start = carry + part[threadIdx.x] - v;
+      const int start = carry + incl - v;
       bp.fptr[q] = start;
       const int32_t* h = bp.hist + (size_t)bp.perm[q] * K;
       int pos = start;
       for (int j = 0; j < K; ++j) { bp.pptr[(size_t)q * (K + 1) + j] = pos; pos += h[j]; }
       bp.pptr[(size_t)q * (K + 1) + K] = pos;
     }
+    if (threadIdx.x == kPtrsThreads - 1) s_total = incl;
     __syncthreads();
-    if (threadIdx.x == 1023) carry += part[1023];
+    carry += s_total;
     __syncthreads();
   }
-  // same scan in execution order
   const int total = carry;
-  __syncthreads();
-  if (threadIdx.x == 0) carry = 0;
-  __syncthreads();
-  for (int base = 0; base < F; base += 1024) {
+  // same scan in execution order
+  carry = 0;
+  for (int base = 0; base < F; base += kPtrsThreads) {
     const int e = base + threadIdx.x;
     const int v = (e < F) ? bp.cnt[bp.xfilt[e]] : 0;
-    part[threadIdx.x] = v;
+    const int incl = block_scan_int(v, warp_tot);
+    if (e < F) bp.xbase[e] = carry + incl - v;
+    if (threadIdx.x == kPtrsThreads - 1) s_total = incl;
     __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-      const int a = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0;
-      __syncthreads();
-      part[threadIdx.x] += a;
-      __syncthreads();
-    }
-    if (e < F) bp.xbase[e] = carry + part[threadIdx.x] - v;
-    __syncthreads();
-    if (threadIdx.x == 1023) carry += part[1023];
+    carry += s_total;
     __syncthreads();
   }
   if (threadIdx.x == 0) {
@@ -297,9 +300,15 @@ __global__ void __launch_bounds__(32) k_pack_blocks(int nct, int nblk, MaskTable
   const int32_t* rowB = bp.tptr + (size_t)(g * kExecGroup + kExecGroup - 1 - w) * (nct + 1);
   // which tile the warp holds when this stage begins
   int cur = 0;
-  for (int t = 0; t < cb; ++t) {
-    const int nother = cur ? rowA[t + 1] - rowA[t] : rowB[t + 1] - rowB[t];
-    if (nother > 0) cur ^= 1;
+  {
+    // both rows are read whatever `cur` is: the loads do not wait for the decision of the tile before
+    int pa = rowA[0], pb = rowB[0];
+    for (int t = 0; t < cb; ++t) {
+      const int na = rowA[t + 1], nb = rowB[t + 1];
+      const int nother = cur ? na - pa : nb - pb;
+      if (nother > 0) cur ^= 1;
+      pa = na; pb = nb;
+    }
   }
   const int aA = rowA[cb], nA = rowA[cb + 1] - aA, aB = rowB[cb], nB = rowB[cb + 1] - aB;
   const int cap = active ? nA + nB + 1 : 0;                       // list slots of this warp in this block
@@ -511,7 +520,7 @@ extern "C" int pat_pack(const float* w_masked, const uint8_t* pattern_id, int F,
   auto note = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
   note(launch_dependent(k_pack_count, dim3(F), dim3(256), K * sizeof(int), st, pattern_id, C, K, bp, status));
   note(launch_dependent(k_pack_rank, dim3(F), dim3(128), 0, st, F, K, bp));
-  note(launch_dependent(k_pack_ptrs, dim3(1), dim3(1024), 0, st, F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status));
+  note(launch_dependent(k_pack_ptrs, dim3(1), dim3(kPtrsThreads), 0, st, F, C, K, (long long)n_keep, dtype, lib, (unsigned long long)L.total, bp, status));
   if (dtype == PAT_F16) {
     if (use_table) note(launch_dependent(k_pack_scatter<__half, true>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));
     else note(launch_dependent(k_pack_scatter<__half, false>, dim3(F), dim3(256), smem, st, w_masked, pattern_id, C, K, L.nct, lib, bp));

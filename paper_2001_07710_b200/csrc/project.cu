@@ -15,7 +15,7 @@
 namespace pat {
 namespace {
 
-constexpr int kSelBlock = 1024;
+constexpr int kSelBlock = 256;
 constexpr int kBins = 65536;
 
 struct SelectState {
@@ -283,7 +283,7 @@ __device__ inline int pick_bin_256(unsigned long long cnt, unsigned long long re
 // itself), finds the remaining 32 bits of the threshold in four 8-bit passes with a histogram in shared memory and
 // then, among the keys equal to the threshold, the index below which `remaining` of them lie (four more passes,
 // over the index bits).  Kernels whose key equals the threshold are kept in index order.
-constexpr int kRestThreads = 1024;
+constexpr int kRestThreads = 256;
 constexpr int kShortList = 2048;
 static_assert(kRestThreads == kSelBlock, "launched with one block per kSelBlock kernels");
 __global__ void __launch_bounds__(kRestThreads) k_select_rest(const unsigned long long* __restrict__ key, int64_t FC,
