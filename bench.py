@@ -414,30 +414,68 @@ def quick_config(pc, torch, cfg_no: int, peaks, steps: int = 10):
     cws = torch.empty(max([pc.pat_conv3x3_workspace(L.F, L.C, dtype, N, L.H, L.W, L.stride) for L in cfg.layers if not L.dense] + [256]),
                       dtype=torch.uint8, device="cuda")
     main = torch.cuda.current_stream()
+    sides = [torch.cuda.Stream(priority=-1) for _ in layers]
+    packed_ev = [torch.cuda.Event() for _ in layers]
 
     def step(ev=None):
+        # ev given: one stream, events around every convolution; otherwise projection / packing of every layer on a
+        # stream of its own, as in the main run
+        cur = torch.cuda.current_stream()
         for i, st in enumerate(layers):
             L = st["L"]
-            if not L.dense:
+            if L.dense:
+                continue
+            prep = cur if ev is not None else sides[i]
+            if ev is None:
+                prep.wait_stream(cur)
+            with torch.cuda.stream(prep):
                 pc.pat_project(st["w"], masks[L.K], L.n_keep, st["pid"], st["wm"], st["ws"])
                 pc.pat_pack(st["wm"], st["pid"], masks[L.K], L.n_keep, dtype, st["blob"])
-            if ev is not None: ev[i][0].record(main)
+                if ev is None:
+                    packed_ev[i].record(prep)
+        for i, st in enumerate(layers):
+            L = st["L"]
+            if ev is not None: ev[i][0].record(cur)
             if L.dense:
                 pc.pat_conv3x3_dense(st["w"], dtype, st["x"], L.stride, y=st["y"])
             else:
+                if ev is None:
+                    cur.wait_event(packed_ev[i])
                 pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], L.stride, y=st["y"], workspace=cws)
-            if ev is not None: ev[i][1].record(main)
+            if ev is not None: ev[i][1].record(cur)
 
     for _ in range(3):
         step()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(main)
-    for _ in range(steps):
-        step()
-    e1.record(main)
-    torch.cuda.synchronize()
-    ms_step = e0.elapsed_time(e1) / steps
+    gstream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(gstream):
+        with torch.cuda.graph(graph, stream=gstream):
+            step()
+        graph.replay()
+        gstream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(gstream)
+        for _ in range(steps):
+            graph.replay()
+        e1.record(gstream)
+        gstream.synchronize()
+        ms_step = e0.elapsed_time(e1) / steps
+        touched = sum((st["x"].numel() + st["y"].numel()) * elem for st in layers)
+        ms_cold = None
+        if touched <= 4 * 126e6:
+            # working set inside L2: also a cold figure, every step after a buffer larger than L2 has been written
+            flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for a, b in pairs:
+                flush.fill_(1)
+                a.record(gstream)
+                graph.replay()
+                b.record(gstream)
+            gstream.synchronize()
+            ms_cold = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+            del flush
+    del graph
     ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(3)]
     for k in range(3):
         step(ev[k])
@@ -453,13 +491,17 @@ def quick_config(pc, torch, cfg_no: int, peaks, steps: int = 10):
         roof_s += roof_us
         if not L.dense:
             fracs.append(roof_us / (ms * 1e3)); flop_s += flop; ms_s += ms
-    touched = sum((st["x"].numel() + st["y"].numel()) * elem for st in layers)
     res = {"workload": f"config {cfg.number}: {cfg.name}", "batch": N, "dtype": dtype, "steps": steps,
            "images_per_s": round(N / (ms_step * 1e-3), 1), "ms_per_step": round(ms_step, 4),
            "conv_ms_per_step": round(sum(conv_ms), 4),
            "sparse_conv_tflops": round(flop_s / (ms_s * 1e-3) / 1e12, 3),
            "roof_frac": round(roof_s / (sum(conv_ms) * 1e3), 4), "min_layer_frac": round(min(fracs), 4),
+           "timing": "step: CUDA-graph replays, projection / packing of each layer on a stream of its own; convolution times: plain launches on one stream",
            "l2": "inputs and outputs larger than L2" if touched > 4 * 126e6 else "warm L2 (working set %.0f MB, no flush between steps)" % (touched / 1e6)}
+    if ms_cold is not None:
+        res["ms_per_step_cold"] = round(ms_cold, 4)
+        res["images_per_s_cold"] = round(N / (ms_cold * 1e-3), 1)
+        res["cold"] = "a 512 MB buffer is written before every step (L2 flushed)"
     del layers, cws
     torch.cuda.empty_cache()
     return res

@@ -278,11 +278,11 @@ __device__ inline int pick_bin_256(unsigned long long cnt, unsigned long long re
 
 // Second digit and everything after it.  All blocks: histogram of the second 16-bit digit over the keys whose first
 // digit is the threshold's, and a list of those keys' indices (any order).  The last block picks the second digit
-// and then works alone: it gathers from the list the keys that agree with the threshold in both digits (a handful
-// for ordinary weights; they stay in shared memory - if there are more than fit, the passes below walk the list
-// itself), finds the remaining 32 bits of the threshold in four 8-bit passes with a histogram in shared memory and
-// then, among the keys equal to the threshold, the index below which `remaining` of them lie (four more passes,
-// over the index bits).  Kernels whose key equals the threshold are kept in index order.
+// and then works alone: it gathers from the list the keys that agree with the threshold in both digits - a handful
+// for ordinary weights, which are ranked directly in shared memory.  If there are more than fit there (weights with
+// few distinct values), it finds the remaining 32 bits of the threshold in four 8-bit passes over the list with a
+// histogram in shared memory and then, among the keys equal to the threshold, the index below which `remaining` of
+// them lie (four more passes, over the index bits).  Kernels whose key equals the threshold are kept in index order.
 constexpr int kRestThreads = 256;
 constexpr int kShortList = 2048;
 static_assert(kRestThreads == kSelBlock, "launched with one block per kSelBlock kernels");
@@ -331,9 +331,26 @@ __global__ void __launch_bounds__(kRestThreads) k_select_rest(const unsigned lon
   __syncthreads();
   const bool fits = s_n <= (unsigned)kShortList;
   const unsigned m = fits ? s_n : n;
+  if (fits) {
+    // The kept kernels of the short list are its first `rem` in the order (key descending, index ascending): the
+    // entry with rem - 1 others before it carries the threshold and the last kept index.  A handful of entries: every
+    // thread ranks its own against all others.
+    for (unsigned j = t; j < m; j += kRestThreads) {
+      const unsigned long long kj = s_key[j];
+      const unsigned ij = s_idx[j];
+      unsigned long long before = 0ull;
+      for (unsigned q = 0; q < m; ++q) {
+        const unsigned long long kq = s_key[q];
+        before += (kq > kj || (kq == kj && s_idx[q] < ij)) ? 1ull : 0ull;
+      }
+      if (before + 1ull == rem) { st->prefix = kj; st->cut = ij; }
+    }
+    return;
+  }
+  // more entries than the short list holds (weights with few distinct values): digit by digit over the list itself
   auto entry = [&](unsigned j, unsigned long long& k, unsigned& idx) {
-    if (fits) { k = s_key[j]; idx = s_idx[j]; }
-    else { idx = __ldcg(cand + j); k = key[idx]; }
+    idx = __ldcg(cand + j);
+    k = key[idx];
   };
   for (int shift = 24; shift >= 0; shift -= 8) {
     if (t < 256) s_hist[t] = 0u;

@@ -59,6 +59,22 @@ def test_project_ties_and_extremes(n_keep):
     assert int((pid.cpu().numpy() != 255).sum()) == n_keep
 
 
+@pytest.mark.parametrize("n_keep", [1, 2500, 2731, 5000, 8191])
+def test_project_ties_beyond_the_short_list(n_keep):
+    """Three distinct kernels over 8192 positions: every threshold has thousands of equal keys, more than the
+    selection kernel ranks in shared memory, so its digit-by-digit passes over the candidate list run."""
+    rng = np.random.default_rng(11)
+    F, C = 64, 128
+    base = rng.standard_normal((3, 3, 3)).astype(np.float32)
+    w = base[rng.integers(0, 3, size=(F, C))]
+    masks = oracle.library(8)
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    pid, wm = pc.pat_project(torch.from_numpy(w).cuda(), masks, n_keep)
+    assert np.array_equal(pid.cpu().numpy(), pid_o)
+    assert np.array_equal(wm.cpu().numpy().view(np.uint32), wm_o.view(np.uint32))
+    assert int((pid.cpu().numpy() != 255).sum()) == n_keep
+
+
 # ------------------------------------------------------------------ pack: bit exact, round trip
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
 @pytest.mark.parametrize("F,C,K,num,den", [(8, 8, 8, 3, 10), (64, 64, 8, 3, 10), (37, 53, 12, 1, 8), (256, 256, 4, 1, 2),
