@@ -305,12 +305,19 @@ __global__ void __launch_bounds__(kRestThreads) k_select_rest(const unsigned lon
   unsigned int* fine = hist + (size_t)(kBins + kCoarse);
   hist_add(fine, fine + kBins, in, d);
   {
+    // a place in the list: one atomic per block (the warps' counts are added up in shared memory first)
+    __shared__ unsigned int s_wcount[kRestThreads / 32], s_base;
     const unsigned active = __ballot_sync(0xFFFFFFFFu, in);
-    const int lane = threadIdx.x & 31;
-    unsigned base = 0u;
-    if (active && lane == (int)(__ffs(active) - 1)) base = atomicAdd(&hist[kListWord], (unsigned)__popc(active));
-    if (active) base = __shfl_sync(0xFFFFFFFFu, base, __ffs(active) - 1);
-    if (in) cand[base + __popc(active & ((1u << lane) - 1u))] = (unsigned)i;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) s_wcount[wid] = (unsigned)__popc(active);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned tot = 0u;
+      for (int q = 0; q < kRestThreads / 32; ++q) { const unsigned c = s_wcount[q]; s_wcount[q] = tot; tot += c; }
+      s_base = tot ? atomicAdd(&hist[kListWord], tot) : 0u;
+    }
+    __syncthreads();
+    if (in) cand[s_base + s_wcount[wid] + __popc(active & ((1u << lane) - 1u))] = (unsigned)i;
   }
   if (!last_block_done(hist + kTicketWord)) return;
   pick_digit(st, hist, 1);
