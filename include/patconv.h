@@ -91,7 +91,7 @@ int pat_project(const float *w, int F, int C, const uint16_t *masks, int K, int6
  * Who needs it: code that is not allowed to allocate device memory where it runs - a server that gave its
  * whole device budget to a memory pool at start-up, a plug-in living inside another framework's allocator,
  * a real-time loop that cannot accept the device-wide synchronisation an allocation may cause.
- * The scratch space is a fixed array inside the library image (about 3.4 MB on every GPU that loads the
+ * The scratch space is a fixed array inside the library image (about 3.9 MB on every GPU that loads the
  * library, held until the process exits), sized for layers of up to pat_project_static_max_kernels() =
  * 262144 kernels (F * C; a 512 x 512 layer).  Larger layers are refused with PAT_ERR_WORKSPACE and nothing
  * is launched; use pat_project for them.  Arguments and results are those of pat_project.

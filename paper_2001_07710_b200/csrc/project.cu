@@ -488,7 +488,7 @@ namespace pat {
 namespace {
 
 constexpr int64_t kStaticMaxKernels = 262144;   // F * C limit of pat_project_static (a 512 x 512 layer)
-constexpr size_t kStaticScratchBytes = ws_bytes(kStaticMaxKernels);   // about 3.4 MB
+constexpr size_t kStaticScratchBytes = ws_bytes(kStaticMaxKernels);   // about 3.9 MB
 
 // Every GPU that loads the library holds this array until the process ends.
 static __device__ __align__(256) unsigned char g_project_scratch[kStaticScratchBytes];
