@@ -44,6 +44,9 @@ def lib():
                                   C.c_int, C.c_void_p]
         L.orc_conv3x3_at.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                      C.c_int, C.c_void_p, C.c_int64, C.c_void_p]
+        L.orc_simplex_project.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_argmax_binarize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_extract_library.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -142,3 +145,39 @@ def conv3x3_at(wm: np.ndarray, x: np.ndarray, coords: np.ndarray, stride: int = 
     if rc != 0:
         raise ValueError(f"orc_conv3x3_at failed ({rc})")
     return out
+
+
+def simplex_project(d: np.ndarray):
+    """Projection of every row of d [n,K] (fp32) onto the probability simplex.  Returns (u f32 [n,K], nu f64 [n])."""
+    d = np.ascontiguousarray(d, dtype=np.float32)
+    n, K = d.shape
+    u = np.empty_like(d)
+    nu = np.empty(n, dtype=np.float64)
+    rc = lib().orc_simplex_project(_p(d), n, K, _p(u), _p(nu))
+    if rc != 0:
+        raise ValueError(f"orc_simplex_project failed ({rc})")
+    return u, nu
+
+
+def argmax_binarize(z: np.ndarray):
+    """Index of the largest entry of every row of z [n,K] (lowest index on ties) and the one-hot rows."""
+    z = np.ascontiguousarray(z, dtype=np.float32)
+    n, K = z.shape
+    idx = np.empty(n, dtype=np.uint8)
+    onehot = np.empty_like(z)
+    rc = lib().orc_argmax_binarize(_p(z), n, K, _p(idx), _p(onehot))
+    if rc != 0:
+        raise ValueError(f"orc_argmax_binarize failed ({rc})")
+    return idx, onehot
+
+
+def extract_library(w: np.ndarray, masks: np.ndarray, K_out: int):
+    """One reduction step of the library extraction on kernels w [n,3,3].  Returns (masks_out u16 [K_out], counts i64 [K_in])."""
+    w = np.ascontiguousarray(w, dtype=np.float32).reshape(-1, 9)
+    masks = np.ascontiguousarray(masks, dtype=np.uint16)
+    out = np.empty(K_out, dtype=np.uint16)
+    counts = np.empty(len(masks), dtype=np.int64)
+    rc = lib().orc_extract_library(_p(w), len(w), _p(masks), len(masks), int(K_out), _p(out), _p(counts))
+    if rc != 0:
+        raise ValueError(f"orc_extract_library failed ({rc})")
+    return out, counts

@@ -21,6 +21,13 @@
  *   orc_conv3x3          pinned: library float64 conv2d, delta / identity / all-ones closed forms,
  *                        an independent sparse-gather evaluation, stride-2 subsampling, linearity.
  *   orc_f32_to_f16       pinned: library round-to-nearest-even conversion, exhaustive round trip.
+ *   orc_simplex_project  pinned: bisection on the defining equation, optimality conditions, closed forms
+ *                        (vector already on the simplex, constant vector, one dominant entry, K = 1, 2).
+ *   orc_argmax_binarize  pinned: library argmax, distance to every one-hot vector; the tie rule is a
+ *                        convention: "parity unpinned".
+ *   orc_extract_library  pinned: for the full 126-mask library the assignment is "the four largest |w|"
+ *                        (independent numpy), planted pattern frequencies are recovered; the tie rule and
+ *                        the order of the survivors are conventions: "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -283,4 +290,97 @@ int orc_conv3x3_at(const double *wm, int F, int C, const void *x, int xdt, int N
     for (int64_t i = 0; i < n_points; ++i)
         out[i] = conv_point(wm, x, xdt, H, W, C, coords[4 * i], coords[4 * i + 1], coords[4 * i + 2], coords[4 * i + 3], stride);
     return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Proximal step of the pattern-selection ADMM (Section 5.1): for a vector d of K reals,
+ *     u = [d - nu 1]_+   with nu the root of   1^T [d - nu 1]_+ = 1,
+ * the Euclidean projection of d onto the probability simplex.  g(nu) = sum_j max(d_j - nu, 0) is
+ * continuous, piecewise linear and strictly decreasing wherever it is positive, so the root is
+ * unique; between two consecutive sorted entries g is linear, so the root is found exactly: with
+ * d sorted descending, d_(1) >= d_(2) >= ..., the root lies in the piece where the first r entries
+ * are above nu, nu = (d_(1) + ... + d_(r) - 1) / r, and r is the largest count for which the
+ * r-th entry is still above that value.  Inputs are fp32, all arithmetic is float64, the result
+ * is rounded once to fp32.  n vectors, row-major [n][K].
+ * ---------------------------------------------------------------------------------------- */
+static int cmp_desc_double(const void *a, const void *b) {
+    const double x = *(const double *)a, y = *(const double *)b;
+    return (x < y) - (x > y);
+}
+
+int orc_simplex_project(const float *d, int64_t n, int K, float *u, double *nu_out) {
+    if (K < 1 || n < 0) return 1;
+    double *s = (double *)malloc(sizeof(double) * (size_t)K);
+    if (!s) return 2;
+    for (int64_t i = 0; i < n; ++i) {
+        const float *di = d + i * K;
+        for (int j = 0; j < K; ++j) s[j] = (double)di[j];
+        qsort(s, (size_t)K, sizeof(double), cmp_desc_double);
+        double run = 0.0, nu = 0.0;
+        for (int r = 1; r <= K; ++r) {
+            run += s[r - 1];
+            const double cand = (run - 1.0) / (double)r;
+            if (s[r - 1] > cand) nu = cand;      /* the r largest entries are all above cand */
+            else break;                          /* and once one is not, no longer prefix is */
+        }
+        for (int j = 0; j < K; ++j) {
+            const double v = (double)di[j] - nu;
+            u[i * K + j] = (float)(v > 0.0 ? v : 0.0);
+        }
+        if (nu_out) nu_out[i] = nu;
+    }
+    free(s);
+    return 0;
+}
+
+/* Binarisation (Section 5.1): the closest one-hot vector to z is the one with its 1 at
+ * argmax_j z_j.  The paper does not say which of several equal maxima wins: the lowest index. */
+int orc_argmax_binarize(const float *z, int64_t n, int K, uint8_t *index_out, float *onehot_out) {
+    if (K < 1 || K > 256 || n < 0) return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        int best = 0;
+        for (int j = 1; j < K; ++j)
+            if (z[i * K + j] > z[i * K + best]) best = j;
+        index_out[i] = (uint8_t)best;
+        if (onehot_out)
+            for (int j = 0; j < K; ++j) onehot_out[i * K + j] = (j == best) ? 1.0f : 0.0f;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * One reduction step of the library extraction (Algorithm 1, Section 5.2), without the training
+ * loop around it: "calculate the pattern distribution of the current library" = every kernel is
+ * given the mask of the library that keeps most of its energy (the argmax of Section 5.1, as in
+ * orc_project: float64 sums in ascending bit order, lowest id on ties) and the kernels per mask
+ * are counted; "remove the patterns with fewest occurrences" = the K_out most frequent masks
+ * stay.  Readings where the paper is silent: among masks of equal count the lower id stays; the
+ * surviving masks keep their order in the library.  w: n kernels [n][3][3] (the kernels of all
+ * layers that share a library, one after another).  counts_out[K_in]; masks_out[K_out].
+ * The paper's schedule is 126 -> 12 -> 8 / 4 (Section 5.2, Section 7.1): call it once per step.
+ * ---------------------------------------------------------------------------------------- */
+int orc_extract_library(const float *w, int64_t n, const uint16_t *masks_in, int K_in, int K_out,
+                        uint16_t *masks_out, int64_t *counts_out) {
+    if (K_in < 1 || K_out < 1 || K_out > K_in || n < 0) return 1;
+    for (int j = 0; j < K_in; ++j) counts_out[j] = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int best = 0;
+        double best_e = -1.0;
+        for (int j = 0; j < K_in; ++j) {
+            double e = 0.0;
+            for (int b = 0; b < 9; ++b)
+                if (masks_in[j] & (1 << b)) e += (double)w[i * 9 + b] * (double)w[i * 9 + b];
+            if (e > best_e) { best_e = e; best = j; }
+        }
+        counts_out[best] += 1;
+    }
+    /* a mask stays if fewer than K_out masks come before it in (count descending, id ascending) */
+    int m = 0;
+    for (int j = 0; j < K_in; ++j) {
+        int before = 0;
+        for (int q = 0; q < K_in; ++q)
+            if (counts_out[q] > counts_out[j] || (counts_out[q] == counts_out[j] && q < j)) ++before;
+        if (before < K_out) masks_out[m++] = masks_in[j];
+    }
+    return m == K_out ? 0 : 2;
 }
