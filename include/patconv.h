@@ -202,6 +202,42 @@ uint64_t pat_launch_count(void);
  * The paper has no counterpart (it reports end-to-end latencies, Section 7.2). */
 int pat_measure_fma_peak(int kind, void *scratch, size_t scratch_bytes, double *tflops_out, void *stream);
 
+/* ---- Primitives of the pattern-selection ADMM and of the library extraction (training side; the loop around them,
+ * the loss and the data are not part of this library).  All pointers are device pointers unless marked host. ---- */
+
+/* Proximal step of Section 5.1: for each of n vectors d of K reals, u = [d - nu 1]_+ where nu is the root of
+ * 1^T [d - nu 1]_+ = 1, i.e. the Euclidean projection of d onto the probability simplex.
+ *   d   dev in  [n][K] fp32, row-major, 4-byte aligned, finite values
+ *   u   dev out [n][K] fp32 (may be d itself); every entry >= 0, every row sums to 1 up to fp32 rounding
+ * Arithmetic in fp64, one rounding to fp32.  1 <= K <= 256; n = 0 is accepted and does nothing.  Asynchronous on
+ * `stream`; allocates nothing.
+ * Errors: PAT_ERR_INVALID_ARG (null), PAT_ERR_SHAPE (K or n out of range), PAT_ERR_ALIGN, PAT_ERR_CUDA. */
+int pat_simplex_project(const float *d, int64_t n, int K, float *u, void *stream);
+
+/* Binarisation of Section 5.1: the one-hot vector closest to z has its 1 at argmax_j z_j; among equal maxima the
+ * lowest index wins (the paper does not say).
+ *   z           dev in  [n][K] fp32, finite values
+ *   index_out   dev out [n] u8: the argmax
+ *   onehot_out  dev out [n][K] fp32 or NULL: the binary vector itself
+ * 1 <= K <= 256.  Asynchronous on `stream`.  Errors as above. */
+int pat_argmax_binarize(const float *z, int64_t n, int K, uint8_t *index_out, float *onehot_out, void *stream);
+
+/* One reduction step of the library extraction (Algorithm 1, Section 5.2: "calculate the pattern distribution of the
+ * current library; remove the patterns with fewest occurrences"), without the training loop: every kernel is given
+ * the mask of the library that keeps most of its energy (as in pat_project), the kernels per mask are counted and
+ * the K_out most frequent masks stay.  Among masks of equal count the lower id stays; the survivors keep the order
+ * they have in masks_in (both are this library's readings, the paper is silent).  The paper's schedule is
+ * 126 -> 12 -> 8 or 4 (Section 5.2, Section 7.1): one call per step, the masks_out of one call (copied to the host)
+ * being the masks_in of the next.
+ *   w           dev in  [n][3][3] fp32: the kernels of all layers that share the library, one after another
+ *   masks_in    HOST in [K_in] 9-bit masks with exactly four bits, distinct; 1 <= K_in <= 255
+ *   masks_out   dev out [K_out] u16, 1 <= K_out <= K_in
+ *   counts_out  dev out [K_in] u64, 8-byte aligned: kernels per mask of masks_in
+ * Asynchronous on `stream` (a memset and two kernels); allocates nothing.
+ * Errors: PAT_ERR_INVALID_ARG, PAT_ERR_LIBRARY, PAT_ERR_SHAPE, PAT_ERR_ALIGN, PAT_ERR_CUDA. */
+int pat_extract_library(const float *w, int64_t n, const uint16_t *masks_in, int K_in, int K_out,
+                        uint16_t *masks_out, uint64_t *counts_out, void *stream);
+
 /* Test hooks of the convolution kernels' bounded waits (host-side, process-wide, not thread safe).  The paper has
  * no counterpart.
  *   what = 0  limit of every device-side wait in nanoseconds (value <= 0: back to the default of 2 s);

@@ -24,7 +24,8 @@ TORCH_DTYPE = {PAT_F32: torch.float32, PAT_F16: torch.float16}
 EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project_workspace", "pat_project",
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
            "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels",
-           "pat_conv3x3_workspace", "pat_conv3x3_ws", "pat_debug_set", "pat_measure_fma_peak"]
+           "pat_conv3x3_workspace", "pat_conv3x3_ws", "pat_debug_set", "pat_measure_fma_peak",
+           "pat_simplex_project", "pat_argmax_binarize", "pat_extract_library"]
 
 
 class PatError(RuntimeError):
@@ -64,6 +65,9 @@ def load() -> C.CDLL:
     L.pat_project_static_max_kernels.argtypes = []; L.pat_project_static_max_kernels.restype = i64
     L.pat_debug_set.argtypes = [i32, C.c_longlong]
     L.pat_measure_fma_peak.argtypes = [i32, vp, sz, vp, vp]
+    L.pat_simplex_project.argtypes = [vp, i64, i32, vp, vp]
+    L.pat_argmax_binarize.argtypes = [vp, i64, i32, vp, vp, vp]
+    L.pat_extract_library.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp]
     _lib = L
     return L
 
@@ -199,6 +203,42 @@ def pat_measure_fma_peak(kind: int = 1, stream=None) -> float:
     out = C.c_double(0.0)
     _check(load().pat_measure_fma_peak(int(kind), _ptr(scratch), scratch.numel(), C.byref(out), _stream(stream)))
     return float(out.value)
+
+
+def pat_simplex_project(d: torch.Tensor, u: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """d: cuda fp32 [n,K].  Returns u [n,K]: every row projected onto the probability simplex."""
+    n, K = int(d.shape[0]), int(d.shape[1])
+    if u is None:
+        u = torch.empty_like(d)
+    _check(load().pat_simplex_project(_ptr(d), n, K, _ptr(u), _stream(stream)))
+    return u
+
+
+def pat_argmax_binarize(z: torch.Tensor, index: Optional[torch.Tensor] = None, onehot: Optional[torch.Tensor] = None,
+                        want_onehot: bool = True, stream=None):
+    """z: cuda fp32 [n,K].  Returns (index u8 [n], onehot fp32 [n,K] or None)."""
+    n, K = int(z.shape[0]), int(z.shape[1])
+    if index is None:
+        index = torch.empty(n, dtype=torch.uint8, device=z.device)
+    if onehot is None and want_onehot:
+        onehot = torch.empty_like(z)
+    _check(load().pat_argmax_binarize(_ptr(z), n, K, _ptr(index), _ptr(onehot), _stream(stream)))
+    return index, onehot
+
+
+def pat_extract_library(w: torch.Tensor, masks, K_out: int, masks_out: Optional[torch.Tensor] = None,
+                        counts: Optional[torch.Tensor] = None, stream=None):
+    """w: cuda fp32 [n,3,3] (any leading shape).  Returns (masks_out int16-typed u16 bits [K_out], counts int64 [K_in]),
+    both on the device."""
+    m = _masks(masks)
+    n = int(w.numel() // 9)
+    if masks_out is None:
+        masks_out = torch.empty(int(K_out), dtype=torch.int16, device=w.device)
+    if counts is None:
+        counts = torch.empty(len(m), dtype=torch.int64, device=w.device)
+    _check(load().pat_extract_library(_ptr(w), n, m.ctypes.data, len(m), int(K_out), _ptr(masks_out), _ptr(counts),
+                                      _stream(stream)))
+    return masks_out, counts
 
 
 def pat_debug_set(what: int, value: int) -> None:

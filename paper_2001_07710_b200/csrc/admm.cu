@@ -1,0 +1,208 @@
+// Primitives of the pattern-selection ADMM (Section 5.1) and of the library extraction (Algorithm 1, Section 5.2),
+// batched over all kernels of a layer (or of a network): the training loop around them is not part of this library.
+//
+//   pat_simplex_project   u = [d - nu 1]_+ with nu the root of 1^T [d - nu 1]_+ = 1 (the proximal step's closed form)
+//   pat_argmax_binarize   the one-hot vector closest to z: 1 at argmax_j z_j
+//   pat_extract_library   "calculate the pattern distribution, remove the patterns with fewest occurrences"
+//
+// The first two stream n x K floats in and out once (8 and 4 - 8 bytes per element): one warp per vector, lanes
+// strided over its entries so that every load and store is a full line.
+#include "common.cuh"
+#include "select.cuh"
+
+namespace pat {
+namespace {
+
+constexpr int kVecMaxK = 256;              // entries per vector: eight per lane
+constexpr int kVecPerLane = kVecMaxK / 32;
+constexpr int kVecWarps = 8;               // vectors per block
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  return v;                                // the same bits in every lane: a butterfly adds the same pairs everywhere
+}
+
+// The root is found without sorting: start with every entry above nu, take nu = (sum of those entries - 1) / their
+// number, drop the entries that are not above it, repeat.  nu only grows, an entry once dropped stays dropped, and
+// when nothing is dropped any more the entries left are exactly those above nu: the piece of the piecewise linear
+// equation that holds its root.  At most K rounds, a handful for ordinary data.  All arithmetic in fp64 (the inputs
+// are fp32, so the sums are exact to about 1e-16 relative), one rounding to fp32 at the end.
+__global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float* __restrict__ d, long long n, int K,
+                                                                     float* __restrict__ u) {
+  const int lane = threadIdx.x & 31;
+  const long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+  if (i >= n) return;                      // whole warps leave together
+  const float* di = d + i * K;
+  double v[kVecPerLane];
+  unsigned above = 0u;                     // bit q: entry lane + 32 q exists and is still above nu
+#pragma unroll
+  for (int q = 0; q < kVecPerLane; ++q) {
+    const int j = lane + 32 * q;
+    v[q] = 0.0;
+    if (j < K) { v[q] = (double)di[j]; above |= 1u << q; }
+  }
+  double nu = 0.0;
+  for (int round = 0; round < K; ++round) {
+    double s = 0.0;
+#pragma unroll
+    for (int q = 0; q < kVecPerLane; ++q) s += ((above >> q) & 1u) ? v[q] : 0.0;
+    s = warp_sum(s);
+    int cnt = __popc(above);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, off);
+    nu = (s - 1.0) / (double)cnt;          // cnt >= 1: nu <= (largest entry) - 1 / cnt, so the largest entry always stays
+    unsigned keep = 0u;
+#pragma unroll
+    for (int q = 0; q < kVecPerLane; ++q) keep |= (((above >> q) & 1u) && v[q] > nu) ? (1u << q) : 0u;
+    const bool changed = keep != above;
+    above = keep;
+    if (!__any_sync(0xFFFFFFFFu, changed)) break;
+  }
+  float* ui = u + i * K;
+#pragma unroll
+  for (int q = 0; q < kVecPerLane; ++q) {
+    const int j = lane + 32 * q;
+    if (j < K) {
+      const double r = v[q] - nu;
+      ui[j] = (float)(r > 0.0 ? r : 0.0);
+    }
+  }
+}
+
+// Largest entry of every vector, the lowest index among equal ones; optionally the one-hot vector itself.
+__global__ void __launch_bounds__(32 * kVecWarps) k_argmax_binarize(const float* __restrict__ z, long long n, int K,
+                                                                     unsigned char* __restrict__ index_out,
+                                                                     float* __restrict__ onehot_out) {
+  const int lane = threadIdx.x & 31;
+  const long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+  if (i >= n) return;
+  const float* zi = z + i * K;
+  float best = 0.0f;
+  int bj = 0x7FFFFFFF;                     // no entry yet
+#pragma unroll
+  for (int q = 0; q < kVecPerLane; ++q) {
+    const int j = lane + 32 * q;
+    if (j < K) {
+      const float x = zi[j];
+      if (bj == 0x7FFFFFFF || x > best) { best = x; bj = j; }     // ascending j inside a lane: the first maximum stays
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+    const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
+    if (oj != 0x7FFFFFFF && (bj == 0x7FFFFFFF || ob > best || (ob == best && oj < bj))) { best = ob; bj = oj; }
+  }
+  if (lane == 0) index_out[i] = (unsigned char)bj;
+  if (onehot_out) {
+    float* oi = onehot_out + i * K;
+#pragma unroll
+    for (int q = 0; q < kVecPerLane; ++q) {
+      const int j = lane + 32 * q;
+      if (j < K) oi[j] = (j == bj) ? 1.0f : 0.0f;
+    }
+  }
+}
+
+// Pattern distribution: every kernel is given the mask that keeps most of its energy (as in pat_project) and the
+// kernels per mask are counted, per block in shared memory first.
+constexpr int kAssignPerThread = 4;
+__global__ void __launch_bounds__(256) k_assign_count(const float* __restrict__ w, long long n, MaskTable lib,
+                                                      unsigned long long* __restrict__ counts) {
+  __shared__ unsigned int s_cnt[kMaxK + 1];
+  for (int q = threadIdx.x; q <= kMaxK; q += blockDim.x) s_cnt[q] = 0u;
+  __syncthreads();
+  for (int r = 0; r < kAssignPerThread; ++r) {
+    const long long i = ((long long)blockIdx.x * kAssignPerThread + r) * blockDim.x + threadIdx.x;
+    if (i < n) {
+      double e;
+      atomicAdd(&s_cnt[best_mask(w + i * 9, lib, e)], 1u);
+    }
+  }
+  __syncthreads();
+  for (int q = threadIdx.x; q < lib.K; q += blockDim.x)
+    if (s_cnt[q]) atomicAdd(&counts[q], (unsigned long long)s_cnt[q]);
+}
+
+// The K_out most frequent masks stay (equal counts: the lower id), in the order they have in the library.  One block:
+// thread j ranks mask j among all masks, the survivors are written in id order.
+__global__ void __launch_bounds__(256) k_pick_survivors(MaskTable lib, const unsigned long long* __restrict__ counts,
+                                                        int K_out, unsigned short* __restrict__ masks_out) {
+  pdl_wait();
+  __shared__ unsigned long long s_c[kMaxK + 1];
+  __shared__ int s_warp[8];
+  const int j = threadIdx.x;
+  s_c[j] = (j < lib.K) ? counts[j] : 0ull;
+  __syncthreads();
+  bool stays = false;
+  if (j < lib.K) {
+    int before = 0;
+    const unsigned long long cj = s_c[j];
+    for (int q = 0; q < lib.K; ++q) before += (s_c[q] > cj || (s_c[q] == cj && q < j)) ? 1 : 0;
+    stays = before < K_out;
+  }
+  const unsigned ballot = __ballot_sync(0xFFFFFFFFu, stays);
+  const int lane = j & 31, wid = j >> 5;
+  if (lane == 0) s_warp[wid] = __popc(ballot);
+  __syncthreads();
+  int pos = __popc(ballot & ((1u << lane) - 1u));
+  for (int q = 0; q < wid; ++q) pos += s_warp[q];
+  if (stays) masks_out[pos] = lib.m[j];
+}
+
+}  // namespace
+}  // namespace pat
+
+using namespace pat;
+
+extern "C" int pat_simplex_project(const float* d, int64_t n, int K, float* u, void* stream) {
+  if (n == 0 && K >= 1 && K <= kVecMaxK) return PAT_OK;      // nothing to do (an empty batch may come with null pointers)
+  if (!d || !u) return set_error(PAT_ERR_INVALID_ARG, "pat_simplex_project: null pointer");
+  if (K < 1 || K > kVecMaxK) return set_error(PAT_ERR_SHAPE, "pat_simplex_project: K=%d outside 1..%d", K, kVecMaxK);
+  if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_simplex_project: n=%lld out of range", (long long)n);
+  if (!aligned(d, 4) || !aligned(u, 4)) return set_error(PAT_ERR_ALIGN, "pat_simplex_project: buffers must be 4-byte aligned");
+  if (n == 0) return PAT_OK;
+  const unsigned grid = (unsigned)((n + kVecWarps - 1) / kVecWarps);
+  k_simplex_project<<<grid, 32 * kVecWarps, 0, reinterpret_cast<cudaStream_t>(stream)>>>(d, (long long)n, K, u);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "pat_simplex_project launch");
+}
+
+extern "C" int pat_argmax_binarize(const float* z, int64_t n, int K, uint8_t* index_out, float* onehot_out, void* stream) {
+  if (n == 0 && K >= 1 && K <= kVecMaxK) return PAT_OK;
+  if (!z || !index_out) return set_error(PAT_ERR_INVALID_ARG, "pat_argmax_binarize: null pointer");
+  if (K < 1 || K > kVecMaxK) return set_error(PAT_ERR_SHAPE, "pat_argmax_binarize: K=%d outside 1..%d", K, kVecMaxK);
+  if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_argmax_binarize: n=%lld out of range", (long long)n);
+  if (!aligned(z, 4) || (onehot_out && !aligned(onehot_out, 4))) return set_error(PAT_ERR_ALIGN, "pat_argmax_binarize: buffers must be 4-byte aligned");
+  if (n == 0) return PAT_OK;
+  const unsigned grid = (unsigned)((n + kVecWarps - 1) / kVecWarps);
+  k_argmax_binarize<<<grid, 32 * kVecWarps, 0, reinterpret_cast<cudaStream_t>(stream)>>>(z, (long long)n, K, index_out, onehot_out);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "pat_argmax_binarize launch");
+}
+
+extern "C" int pat_extract_library(const float* w, int64_t n, const uint16_t* masks_in, int K_in, int K_out,
+                                   uint16_t* masks_out, uint64_t* counts_out, void* stream) {
+  if (!w || !masks_out || !counts_out) return set_error(PAT_ERR_INVALID_ARG, "pat_extract_library: null pointer");
+  if (int rc = check_library(masks_in, K_in)) return rc;
+  if (K_out < 1 || K_out > K_in) return set_error(PAT_ERR_INVALID_ARG, "pat_extract_library: K_out=%d outside 1..%d", K_out, K_in);
+  if (n < 0 || n > 0x7FFFFFFFll * 256) return set_error(PAT_ERR_SHAPE, "pat_extract_library: n=%lld out of range", (long long)n);
+  if (!aligned(w, 4) || !aligned(counts_out, 8) || !aligned(masks_out, 2)) return set_error(PAT_ERR_ALIGN, "pat_extract_library: misaligned buffer");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  MaskTable lib;
+  for (int j = 0; j <= kMaxK; ++j) lib.m[j] = (j < K_in) ? masks_in[j] : (uint16_t)0;
+  lib.K = K_in;
+  if (int rc = check_cuda(cudaMemsetAsync(counts_out, 0, sizeof(uint64_t) * (size_t)K_in, st), "pat_extract_library memset")) return rc;
+  if (n > 0) {
+    const unsigned grid = (unsigned)((n + 256 * kAssignPerThread - 1) / (256 * kAssignPerThread));
+    k_assign_count<<<grid, 256, 0, st>>>(w, (long long)n, lib, reinterpret_cast<unsigned long long*>(counts_out));
+    count_launches(1);
+  }
+  cudaError_t le = launch_dependent(k_pick_survivors, dim3(1), dim3(256), 0, st, lib,
+                                    reinterpret_cast<const unsigned long long*>(counts_out), K_out,
+                                    reinterpret_cast<unsigned short*>(masks_out));
+  count_launches(1);
+  if (le != cudaSuccess) return check_cuda(le, "pat_extract_library launch");
+  return check_cuda(cudaGetLastError(), "pat_extract_library launch");
+}

@@ -11,6 +11,7 @@
 // index that separates kept from removed ties by one thread block over that list.  Three launches per layer: the
 // steps that need all blocks' results are done by the block that finishes last.
 #include "common.cuh"
+#include "select.cuh"
 
 namespace pat {
 namespace {
@@ -169,63 +170,8 @@ __global__ void __launch_bounds__(256) k_select_pattern(const float* __restrict_
     const bool in = i < FC;
     unsigned long long k = 0ull;
     if (in) {
-      const float* wk = w + i * 9;
-      // Double-precision arithmetic is scarce on this GPU, so the argmax is first taken in fp32.  Nine squares and a
-      // sum of at most nine non-negative terms carry a relative error below 2^-20 (nine roundings of 2^-24 each) as
-      // long as nothing overflows and the result is far above the subnormal range, so an fp32 winner that leads the
-      // runner-up by a factor of more than 1 + 2^-18 is the exact winner too.  Every other case - a lead inside the
-      // error bound (exact ties among them), a tiny, huge or non-finite energy - takes the exact path over all masks.
-      // The energy itself (the key of the connectivity ranking) is always computed exactly: fp64 squares of the
-      // winner's entries, added in ascending bit order.
-      float sqf[9];
-#pragma unroll
-      for (int b = 0; b < 9; ++b) {
-        const float v = wk[b];
-        sqf[b] = __fmul_rn(v, v);
-      }
-      float best32 = -1.0f, second32 = -1.0f;
-      int best = 0;
-      bool plain = true;                       // every fp32 energy is an ordinary finite number
-      for (int j = 0; j < lib.K; ++j) {
-        const unsigned m = lib.m[j];
-        float e = 0.0f;
-#pragma unroll
-        for (int b = 0; b < 9; ++b)
-          if (m & (1u << b)) e = __fadd_rn(e, sqf[b]);
-        plain = plain && (e <= 3.0e38f);       // false for NaN and infinity
-        if (e > best32) { second32 = best32; best32 = e; best = j; }
-        else if (e > second32) second32 = e;   // e == best32 lands here: a tie is never a clear lead
-      }
-      constexpr float kLead = 1.0f + 3.814697265625e-6f;     // 1 + 2^-18
-      constexpr float kFloor = 7.8886090522101181e-31f;      // 2^-100
-      const bool clear = plain && best32 >= kFloor && best32 > second32 * kLead;
       double best_e;
-      if (clear) {
-        best_e = 0.0;
-        unsigned m = lib.m[best];
-        while (m) {                            // ascending bit order
-          const double v = (double)wk[__ffs(m) - 1];
-          best_e += v * v;                     // the square of an fp32 value is exact in fp64
-          m &= m - 1u;
-        }
-      } else {
-        double sq[9];
-#pragma unroll
-        for (int b = 0; b < 9; ++b) {
-          const double v = (double)wk[b];
-          sq[b] = v * v;
-        }
-        best_e = -1.0;
-        best = 0;
-        for (int j = 0; j < lib.K; ++j) {
-          const unsigned m = lib.m[j];
-          double e = 0.0;
-#pragma unroll
-          for (int b = 0; b < 9; ++b)
-            if (m & (1u << b)) e += sq[b];
-          if (e > best_e) { best_e = e; best = j; }
-        }
-      }
+      const int best = best_mask(w + i * 9, lib, best_e);
       k = (unsigned long long)__double_as_longlong(best_e);   // e >= +0: bit pattern is monotone
       key[i] = k;
       pid[i] = (unsigned char)best;
