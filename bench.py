@@ -384,12 +384,72 @@ def run_ours(args):
     if world == 1 and not args.no_other_configs and args.batch is None and args.layers is None:
         # the other four configurations: short measurements of their own, after the main timed region
         out["other_configs"] = {str(c): quick_config(pc, torch, c, peaks) for c in range(5) if c != cfg.number}
+    if world == 1 and not args.no_other_configs and args.batch is None and args.layers is None:
+        out["admm_primitives"] = admm_primitives(pc, torch, peaks, with_cpu=not args.no_cpu)
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_seconds)
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def admm_primitives(pc, torch, peaks, with_cpu: bool, reps: int = 10):
+    """The training-side primitives on the kernels of a 512 x 512 layer with the full library of 126 masks (the
+    start of the library extraction): simplex projection and binarisation of 262 144 vectors of 126 entries (132 MB
+    in, 132 MB out: larger than L2), and one reduction step 126 -> 12 of the library.  CUDA events, after three
+    warm-up calls; the oracle is timed beside them on a bounded sample."""
+    import itertools
+    n, K = 512 * 512, 126
+    rng = np.random.default_rng(20200107)
+    d_np = (rng.standard_normal((n, K)) * 0.3 + 1.0 / K).astype(np.float32)
+    w_np = workloads.make_weights(rng, 512, 512)
+    masks = np.array([sum(1 << b for b in c) for c in itertools.combinations(range(9), 4)], dtype=np.uint16)
+    d = torch.from_numpy(d_np).cuda()
+    u = torch.empty_like(d)
+    idx = torch.empty(n, dtype=torch.uint8, device="cuda")
+    w = torch.from_numpy(w_np).cuda()
+    mout = torch.empty(12, dtype=torch.int16, device="cuda")
+    counts = torch.empty(K, dtype=torch.int64, device="cuda")
+    st = torch.cuda.current_stream()
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(reps):
+            fn()
+        e1.record(st)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e-3
+
+    hbm = peaks["hbm_gbs"]
+    t_sp = timed(lambda: pc.pat_simplex_project(d, u))
+    t_am = timed(lambda: pc.pat_argmax_binarize(u, idx, want_onehot=False))
+    t_ex = timed(lambda: pc.pat_extract_library(w, masks, 12, mout, counts))
+    res = {"workload": "262144 vectors / kernels (a 512 x 512 layer), library of 126 masks; inputs and outputs larger than L2",
+           "simplex_project": {"ms": round(t_sp * 1e3, 4), "GB/s": round(8.0 * n * K / t_sp / 1e9, 1),
+                               "roofline": {"bound": "hbm", "peak": hbm, "frac": round(8.0 * n * K / t_sp / 1e9 / hbm, 4)},
+                               "bytes": "read once + written once, 8 per entry"},
+           "argmax_binarize": {"ms": round(t_am * 1e3, 4), "GB/s": round((4.0 * n * K + n) / t_am / 1e9, 1),
+                               "roofline": {"bound": "hbm", "peak": hbm, "frac": round((4.0 * n * K + n) / t_am / 1e9 / hbm, 4)},
+                               "bytes": "read once, one index byte per vector"},
+           "extract_library_126_to_12": {"ms": round(t_ex * 1e3, 4), "kernels_per_s": round(n / t_ex, 0),
+                                         "note": "a memset and two launches; 126 mask energies per kernel (fp32, exact fp64 fallback): arithmetic, not memory"}}
+    if with_cpu:
+        import oracle
+        m = 8192                                      # a bounded sample of the same vectors / kernels
+        t0 = time.perf_counter(); oracle.simplex_project(d_np[:m]); t1 = time.perf_counter()
+        oracle.argmax_binarize(d_np[:m]); t2 = time.perf_counter()
+        oracle.extract_library(w_np.reshape(-1, 3, 3)[:m], masks, 12); t3 = time.perf_counter()
+        res["cpu_oracle"] = {"sample": f"{m} vectors / kernels, one thread", "simplex_project_vectors_per_s": round(m / (t1 - t0), 0),
+                             "argmax_binarize_vectors_per_s": round(m / (t2 - t1), 0), "extract_library_kernels_per_s": round(m / (t3 - t2), 0),
+                             "gpu_simplex_project_vectors_per_s": round(n / t_sp, 0)}
+    del d, u, w
+    torch.cuda.empty_cache()
+    return res
 
 
 def quick_config(pc, torch, cfg_no: int, peaks, steps: int = 10):
@@ -608,6 +668,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="override the batch size (profiling small cases)")
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling one layer)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--admm-only", action="store_true", help="only the training-side primitives (simplex projection, binarisation, library extraction): prints their JSON object")
     ap.add_argument("--no-overlap", action="store_true", help="projection / packing on the same stream as the convolutions")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
@@ -636,6 +697,12 @@ def main():
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
         print(json.dumps({"fma_rn_f32_tflops": round(pc.pat_measure_fma_peak(0), 2), "fma_rn_f32_f16_tflops": round(pc.pat_measure_fma_peak(1), 2),
                           "derived_tflops": round(FMA_PEAK_TFLOPS, 2)}))
+        return
+    if args.admm_only:
+        import torch
+        import paper_2001_07710_b200 as pc
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        print(json.dumps(admm_primitives(pc, torch, measured_peaks()[0], with_cpu=not args.no_cpu)))
         return
     run_ours(args)
 

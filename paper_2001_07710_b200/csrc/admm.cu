@@ -23,50 +23,82 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;                                // the same bits in every lane: a butterfly adds the same pairs everywhere
 }
 
-// The root is found without sorting: start with every entry above nu, take nu = (sum of those entries - 1) / their
-// number, drop the entries that are not above it, repeat.  nu only grows, an entry once dropped stays dropped, and
-// when nothing is dropped any more the entries left are exactly those above nu: the piece of the piecewise linear
-// equation that holds its root.  At most K rounds, a handful for ordinary data.  All arithmetic in fp64 (the inputs
-// are fp32, so the sums are exact to about 1e-16 relative), one rounding to fp32 at the end.
-__global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float* __restrict__ d, long long n, int K,
-                                                                     float* __restrict__ u) {
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  return v;
+}
+__device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }   // one instruction for integers
+
+// The root is found without sorting.  g(nu) = sum_j max(d_j - nu, 0) is convex, piecewise linear and decreasing, and
+// Newton's step for g(nu) = 1 from a point nu is nu' = (sum of the entries above nu - 1) / (their number): from any
+// start whose set of entries above it is not empty the steps reach the root in finitely many rounds (after the first
+// step they approach it from below and never pass it), and at the root the set no longer changes.  Most rounds run
+// in fp32, starting with all entries (then every step only drops entries, and the largest one always stays): they
+// find the set of entries above the root up to rounding.  The last rounds repeat the step in fp64 from that set
+// until it is stable - usually one or two - so the result is the exact piece of the equation: the sums are exact to
+// about 1e-16 relative (the inputs are fp32), and there is one rounding to fp32 at the end.
+// Q = entries per lane (K <= 32 Q).  u may be d.
+template <int Q>
+__global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float* d, long long n, int K, float* u) {
   const int lane = threadIdx.x & 31;
-  const long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+  const long long stride = (long long)gridDim.x * kVecWarps;
+  long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
   if (i >= n) return;                      // whole warps leave together
-  const float* di = d + i * K;
-  double v[kVecPerLane];
-  unsigned above = 0u;                     // bit q: entry lane + 32 q exists and is still above nu
+  unsigned exists = 0u;                    // bit q: entry lane + 32 q exists
 #pragma unroll
-  for (int q = 0; q < kVecPerLane; ++q) {
-    const int j = lane + 32 * q;
-    v[q] = 0.0;
-    if (j < K) { v[q] = (double)di[j]; above |= 1u << q; }
-  }
-  double nu = 0.0;
-  for (int round = 0; round < K; ++round) {
-    double s = 0.0;
+  for (int q = 0; q < Q; ++q) exists |= (lane + 32 * q < K) ? (1u << q) : 0u;
+  // a warp walks over its vectors with the next one's loads already in flight (the grid is a few blocks per SM)
+  float nxt[Q];
 #pragma unroll
-    for (int q = 0; q < kVecPerLane; ++q) s += ((above >> q) & 1u) ? v[q] : 0.0;
-    s = warp_sum(s);
-    int cnt = __popc(above);
+  for (int q = 0; q < Q; ++q) nxt[q] = ((exists >> q) & 1u) ? __ldcs(d + i * K + lane + 32 * q) : 0.0f;
+  for (; i < n; i += stride) {
+    float x[Q];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, off);
-    nu = (s - 1.0) / (double)cnt;          // cnt >= 1: nu <= (largest entry) - 1 / cnt, so the largest entry always stays
-    unsigned keep = 0u;
+    for (int q = 0; q < Q; ++q) x[q] = nxt[q];
+    if (i + stride < n) {
 #pragma unroll
-    for (int q = 0; q < kVecPerLane; ++q) keep |= (((above >> q) & 1u) && v[q] > nu) ? (1u << q) : 0u;
-    const bool changed = keep != above;
-    above = keep;
-    if (!__any_sync(0xFFFFFFFFu, changed)) break;
-  }
-  float* ui = u + i * K;
-#pragma unroll
-  for (int q = 0; q < kVecPerLane; ++q) {
-    const int j = lane + 32 * q;
-    if (j < K) {
-      const double r = v[q] - nu;
-      ui[j] = (float)(r > 0.0 ? r : 0.0);
+      for (int q = 0; q < Q; ++q)
+        if ((exists >> q) & 1u) nxt[q] = __ldcs(d + (i + stride) * K + lane + 32 * q);
     }
+    unsigned above = exists;               // bit q: entry q of this lane is above nu
+    for (int round = 0; round < K; ++round) {          // fp32 rounds
+      float s = 0.0f;
+#pragma unroll
+      for (int q = 0; q < Q; ++q) s += ((above >> q) & 1u) ? x[q] : 0.0f;
+      s = warp_sum(s);
+      const int cnt = warp_sum(__popc(above));
+      const float nu32 = (s - 1.0f) / (float)cnt;
+      unsigned keep = 0u;
+#pragma unroll
+      for (int q = 0; q < Q; ++q) keep |= (((above >> q) & 1u) && x[q] > nu32) ? (1u << q) : 0u;
+      if (!__any_sync(0xFFFFFFFFu, keep != 0u)) break;   // rounding only: keep the last set that was not empty
+      const bool changed = keep != above;
+      above = keep;
+      if (!__any_sync(0xFFFFFFFFu, changed)) break;
+    }
+    double nu = 0.0;
+    for (int round = 0; round < K + 2; ++round) {       // fp64 rounds from the set found
+      double s = 0.0;
+#pragma unroll
+      for (int q = 0; q < Q; ++q) s += ((above >> q) & 1u) ? (double)x[q] : 0.0;
+      s = warp_sum(s);
+      const int cnt = warp_sum(__popc(above));          // >= 1, see above
+      nu = (s - 1.0) / (double)cnt;
+      unsigned now = 0u;
+#pragma unroll
+      for (int q = 0; q < Q; ++q) now |= (((exists >> q) & 1u) && (double)x[q] > nu) ? (1u << q) : 0u;
+      const bool changed = now != above;
+      if (!__any_sync(0xFFFFFFFFu, changed) || !__any_sync(0xFFFFFFFFu, now != 0u)) break;   // empty: entries too large for 1 to count
+      above = now;
+    }
+    float* ui = u + i * K;
+#pragma unroll
+    for (int q = 0; q < Q; ++q)
+      if ((exists >> q) & 1u) {
+        const double r = (double)x[q] - nu;
+        __stcs(ui + lane + 32 * q, (float)(r > 0.0 ? r : 0.0));
+      }
   }
 }
 
@@ -75,32 +107,47 @@ __global__ void __launch_bounds__(32 * kVecWarps) k_argmax_binarize(const float*
                                                                      unsigned char* __restrict__ index_out,
                                                                      float* __restrict__ onehot_out) {
   const int lane = threadIdx.x & 31;
-  const long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+  const long long stride = (long long)gridDim.x * kVecWarps;
+  long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
   if (i >= n) return;
-  const float* zi = z + i * K;
-  float best = 0.0f;
-  int bj = 0x7FFFFFFF;                     // no entry yet
+  float nxt[kVecPerLane];
 #pragma unroll
   for (int q = 0; q < kVecPerLane; ++q) {
     const int j = lane + 32 * q;
-    if (j < K) {
-      const float x = zi[j];
-      if (bj == 0x7FFFFFFF || x > best) { best = x; bj = j; }     // ascending j inside a lane: the first maximum stays
-    }
+    nxt[q] = (j < K) ? __ldcs(z + i * K + j) : 0.0f;
   }
+  for (; i < n; i += stride) {
+    float x[kVecPerLane];
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
-    const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
-    if (oj != 0x7FFFFFFF && (bj == 0x7FFFFFFF || ob > best || (ob == best && oj < bj))) { best = ob; bj = oj; }
-  }
-  if (lane == 0) index_out[i] = (unsigned char)bj;
-  if (onehot_out) {
-    float* oi = onehot_out + i * K;
+    for (int q = 0; q < kVecPerLane; ++q) x[q] = nxt[q];
+    if (i + stride < n) {
+#pragma unroll
+      for (int q = 0; q < kVecPerLane; ++q) {
+        const int j = lane + 32 * q;
+        if (j < K) nxt[q] = __ldcs(z + (i + stride) * K + j);
+      }
+    }
+    float best = 0.0f;
+    int bj = 0x7FFFFFFF;                   // no entry yet
 #pragma unroll
     for (int q = 0; q < kVecPerLane; ++q) {
       const int j = lane + 32 * q;
-      if (j < K) oi[j] = (j == bj) ? 1.0f : 0.0f;
+      if (j < K && (bj == 0x7FFFFFFF || x[q] > best)) { best = x[q]; bj = j; }   // ascending j inside a lane: the first maximum stays
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+      const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
+      if (oj != 0x7FFFFFFF && (bj == 0x7FFFFFFF || ob > best || (ob == best && oj < bj))) { best = ob; bj = oj; }
+    }
+    if (lane == 0) index_out[i] = (unsigned char)bj;
+    if (onehot_out) {
+      float* oi = onehot_out + i * K;
+#pragma unroll
+      for (int q = 0; q < kVecPerLane; ++q) {
+        const int j = lane + 32 * q;
+        if (j < K) __stcs(oi + j, (j == bj) ? 1.0f : 0.0f);
+      }
     }
   }
 }
@@ -151,6 +198,15 @@ __global__ void __launch_bounds__(256) k_pick_survivors(MaskTable lib, const uns
   if (stays) masks_out[pos] = lib.m[j];
 }
 
+// Blocks of the vector kernels: enough for eight resident blocks per SM, each warp then walks over its vectors.
+unsigned vec_grid(int64_t n) {
+  static thread_local DeviceSlot slots[kMaxDevices];
+  DeviceSlot* dv = device_slot(slots);
+  const long long want = (long long)(dv ? dv->sms : 148) * 8;
+  const long long need = (n + kVecWarps - 1) / kVecWarps;
+  return (unsigned)(need < want ? need : want);
+}
+
 }  // namespace
 }  // namespace pat
 
@@ -163,8 +219,12 @@ extern "C" int pat_simplex_project(const float* d, int64_t n, int K, float* u, v
   if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_simplex_project: n=%lld out of range", (long long)n);
   if (!aligned(d, 4) || !aligned(u, 4)) return set_error(PAT_ERR_ALIGN, "pat_simplex_project: buffers must be 4-byte aligned");
   if (n == 0) return PAT_OK;
-  const unsigned grid = (unsigned)((n + kVecWarps - 1) / kVecWarps);
-  k_simplex_project<<<grid, 32 * kVecWarps, 0, reinterpret_cast<cudaStream_t>(stream)>>>(d, (long long)n, K, u);
+  const unsigned grid = vec_grid(n);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (K <= 32) k_simplex_project<1><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else if (K <= 64) k_simplex_project<2><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else if (K <= 128) k_simplex_project<4><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else k_simplex_project<8><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_simplex_project launch");
 }
@@ -176,7 +236,7 @@ extern "C" int pat_argmax_binarize(const float* z, int64_t n, int K, uint8_t* in
   if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_argmax_binarize: n=%lld out of range", (long long)n);
   if (!aligned(z, 4) || (onehot_out && !aligned(onehot_out, 4))) return set_error(PAT_ERR_ALIGN, "pat_argmax_binarize: buffers must be 4-byte aligned");
   if (n == 0) return PAT_OK;
-  const unsigned grid = (unsigned)((n + kVecWarps - 1) / kVecWarps);
+  const unsigned grid = vec_grid(n);
   k_argmax_binarize<<<grid, 32 * kVecWarps, 0, reinterpret_cast<cudaStream_t>(stream)>>>(z, (long long)n, K, index_out, onehot_out);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_argmax_binarize launch");
