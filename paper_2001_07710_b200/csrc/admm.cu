@@ -23,12 +23,13 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;                                // the same bits in every lane: a butterfly adds the same pairs everywhere
 }
 
-__device__ __forceinline__ float warp_sum(float v) {
+// Sums over the L lanes that share a vector (L a power of two, groups aligned): the same bits in every lane of a group.
+template <int L, typename T>
+__device__ __forceinline__ T group_sum(T v) {
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+  for (int off = L / 2; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
   return v;
 }
-__device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFFFFFFu, v); }   // one instruction for integers
 
 // The root is found without sorting.  g(nu) = sum_j max(d_j - nu, 0) is convex, piecewise linear and decreasing, and
 // Newton's step for g(nu) = 1 from a point nu is nu' = (sum of the entries above nu - 1) / (their number): from any
@@ -38,67 +39,68 @@ __device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xFFFF
 // find the set of entries above the root up to rounding.  The last rounds repeat the step in fp64 from that set
 // until it is stable - usually one or two - so the result is the exact piece of the equation: the sums are exact to
 // about 1e-16 relative (the inputs are fp32), and there is one rounding to fp32 at the end.
-// Q = entries per lane (K <= 32 Q).  u may be d.
-template <int Q>
+//
+// L lanes share a vector, sixteen entries each (K <= 16 L), so a warp works on 32 / L vectors at once: a round is a
+// chain of dependent steps (a sum over the group, a division, a comparison), and what the kernel needs is many such
+// chains in flight, not many lanes per chain.  Entry j of a vector sits in lane j % L, slot j / L.  u may be d.
+constexpr int kVecQ = 16;
+template <int L>
 __global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float* d, long long n, int K, float* u) {
-  const int lane = threadIdx.x & 31;
-  const long long stride = (long long)gridDim.x * kVecWarps;
-  long long i = (long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
-  if (i >= n) return;                      // whole warps leave together
-  unsigned exists = 0u;                    // bit q: entry lane + 32 q exists
+  constexpr int G = 32 / L;                // vectors per warp
+  const int lane = threadIdx.x & 31, sl = lane & (L - 1), g = lane / L;
+  const long long stride = (long long)gridDim.x * kVecWarps * G;
+  const long long first = ((long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5)) * G;
+  if (first >= n) return;                  // whole warps leave together
+  unsigned exists = 0u;                    // bit q: entry sl + L q exists
 #pragma unroll
-  for (int q = 0; q < Q; ++q) exists |= (lane + 32 * q < K) ? (1u << q) : 0u;
-  // a warp walks over its vectors with the next one's loads already in flight (the grid is a few blocks per SM)
-  float nxt[Q];
+  for (int q = 0; q < kVecQ; ++q) exists |= (sl + L * q < K) ? (1u << q) : 0u;
+  for (long long base = first; base < n; base += stride) {
+    const bool valid = base + g < n;
+    const long long i = valid ? base + g : n - 1;       // a group without a vector repeats the last one and stores nothing
+    float x[kVecQ];
 #pragma unroll
-  for (int q = 0; q < Q; ++q) nxt[q] = ((exists >> q) & 1u) ? __ldcs(d + i * K + lane + 32 * q) : 0.0f;
-  for (; i < n; i += stride) {
-    float x[Q];
-#pragma unroll
-    for (int q = 0; q < Q; ++q) x[q] = nxt[q];
-    if (i + stride < n) {
-#pragma unroll
-      for (int q = 0; q < Q; ++q)
-        if ((exists >> q) & 1u) nxt[q] = __ldcs(d + (i + stride) * K + lane + 32 * q);
-    }
+    for (int q = 0; q < kVecQ; ++q) x[q] = ((exists >> q) & 1u) ? __ldcs(d + i * K + sl + L * q) : 0.0f;
     unsigned above = exists;               // bit q: entry q of this lane is above nu
     for (int round = 0; round < K; ++round) {          // fp32 rounds
       float s = 0.0f;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) s += ((above >> q) & 1u) ? x[q] : 0.0f;
-      s = warp_sum(s);
-      const int cnt = warp_sum(__popc(above));
+      for (int q = 0; q < kVecQ; ++q) s += ((above >> q) & 1u) ? x[q] : 0.0f;
+      s = group_sum<L>(s);
+      const int cnt = group_sum<L>(__popc(above));
       const float nu32 = (s - 1.0f) / (float)cnt;
       unsigned keep = 0u;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) keep |= (((above >> q) & 1u) && x[q] > nu32) ? (1u << q) : 0u;
-      if (!__any_sync(0xFFFFFFFFu, keep != 0u)) break;   // rounding only: keep the last set that was not empty
-      const bool changed = keep != above;
-      above = keep;
-      if (!__any_sync(0xFFFFFFFFu, changed)) break;
+      for (int q = 0; q < kVecQ; ++q) keep |= (((above >> q) & 1u) && x[q] > nu32) ? (1u << q) : 0u;
+      const bool empty = group_sum<L>(__popc(keep)) == 0;   // rounding only: the group keeps its last set that was not empty
+      const bool changed = !empty && keep != above;
+      if (!empty) above = keep;
+      if (!__any_sync(0xFFFFFFFFu, changed)) break;         // every vector of the warp is through
     }
     double nu = 0.0;
     for (int round = 0; round < K + 2; ++round) {       // fp64 rounds from the set found
       double s = 0.0;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) s += ((above >> q) & 1u) ? (double)x[q] : 0.0;
-      s = warp_sum(s);
-      const int cnt = warp_sum(__popc(above));          // >= 1, see above
+      for (int q = 0; q < kVecQ; ++q) s += ((above >> q) & 1u) ? (double)x[q] : 0.0;
+      s = group_sum<L>(s);
+      const int cnt = group_sum<L>(__popc(above));      // >= 1, see above
       nu = (s - 1.0) / (double)cnt;
       unsigned now = 0u;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) now |= (((exists >> q) & 1u) && (double)x[q] > nu) ? (1u << q) : 0u;
-      const bool changed = now != above;
-      if (!__any_sync(0xFFFFFFFFu, changed) || !__any_sync(0xFFFFFFFFu, now != 0u)) break;   // empty: entries too large for 1 to count
-      above = now;
+      for (int q = 0; q < kVecQ; ++q) now |= (((exists >> q) & 1u) && (double)x[q] > nu) ? (1u << q) : 0u;
+      const bool empty = group_sum<L>(__popc(now)) == 0;    // entries too large for the 1 to count
+      const bool changed = !empty && now != above;
+      if (!empty) above = now;
+      if (!__any_sync(0xFFFFFFFFu, changed)) break;
     }
-    float* ui = u + i * K;
+    if (valid) {
+      float* ui = u + i * K;
 #pragma unroll
-    for (int q = 0; q < Q; ++q)
-      if ((exists >> q) & 1u) {
-        const double r = (double)x[q] - nu;
-        __stcs(ui + lane + 32 * q, (float)(r > 0.0 ? r : 0.0));
-      }
+      for (int q = 0; q < kVecQ; ++q)
+        if ((exists >> q) & 1u) {
+          const double r = (double)x[q] - nu;
+          __stcs(ui + sl + L * q, (float)(r > 0.0 ? r : 0.0));
+        }
+    }
   }
 }
 
@@ -199,11 +201,11 @@ __global__ void __launch_bounds__(256) k_pick_survivors(MaskTable lib, const uns
 }
 
 // Blocks of the vector kernels: enough for eight resident blocks per SM, each warp then walks over its vectors.
-unsigned vec_grid(int64_t n) {
+unsigned vec_grid(int64_t n, int per_warp = 1) {
   static thread_local DeviceSlot slots[kMaxDevices];
   DeviceSlot* dv = device_slot(slots);
   const long long want = (long long)(dv ? dv->sms : 148) * 8;
-  const long long need = (n + kVecWarps - 1) / kVecWarps;
+  const long long need = (n + (long long)kVecWarps * per_warp - 1) / ((long long)kVecWarps * per_warp);
   return (unsigned)(need < want ? need : want);
 }
 
@@ -219,12 +221,12 @@ extern "C" int pat_simplex_project(const float* d, int64_t n, int K, float* u, v
   if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_simplex_project: n=%lld out of range", (long long)n);
   if (!aligned(d, 4) || !aligned(u, 4)) return set_error(PAT_ERR_ALIGN, "pat_simplex_project: buffers must be 4-byte aligned");
   if (n == 0) return PAT_OK;
-  const unsigned grid = vec_grid(n);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (K <= 32) k_simplex_project<1><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
-  else if (K <= 64) k_simplex_project<2><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
-  else if (K <= 128) k_simplex_project<4><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
-  else k_simplex_project<8><<<grid, 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  if (K <= 16) k_simplex_project<1><<<vec_grid(n, 32), 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else if (K <= 32) k_simplex_project<2><<<vec_grid(n, 16), 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else if (K <= 64) k_simplex_project<4><<<vec_grid(n, 8), 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else if (K <= 128) k_simplex_project<8><<<vec_grid(n, 4), 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
+  else k_simplex_project<16><<<vec_grid(n, 2), 32 * kVecWarps, 0, st>>>(d, (long long)n, K, u);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_simplex_project launch");
 }
