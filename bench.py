@@ -35,7 +35,7 @@ DEFAULT_CONFIG = 3
 # DRAM traffic of the convolution path (ncu counters of a small case), written by `bench.py --write-traffic` and
 # valid only for the kernel sources it was captured from
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_conv_f16_img_conv6_b32.json")
-TRAFFIC_SOURCES = ["conv_f16_img.cu", "f16_tile.cuh", "common.cuh"]
+TRAFFIC_SOURCES = ["conv_f16_img.cu", "f16_tile.cuh", "common.cuh", "img_geometry.cuh"]
 
 
 def kernel_source_hash() -> str:

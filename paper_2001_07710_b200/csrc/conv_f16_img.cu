@@ -21,16 +21,16 @@
 //  3. k_reduce_parts adds, in a fixed order, the fp32 partial sums of work items that were cut along the input
 //     channels (the items of a last, mostly idle round; every item when there are fewer items than half the SMs).
 #include <algorithm>
-#include "f16_tile.cuh"
+#include "img_geometry.cuh"
 
 namespace pat {
 namespace img16 {
 using namespace fast16;
+using namespace imggeo;
 
 constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three idle warps (register donors)
 constexpr int W_PRODUCER = NCW;
 constexpr int CBI = kChanTile;             // channels per ring stage (16)
-constexpr int MAXROWS = LY * TR4 + 4;      // two bands, each with a top and a bottom halo row (36)
 constexpr int CHP = MAXROWS * ROWB;        // channel plane pitch (4608)
 constexpr int IMG_BYTES = CBI * CHP;       // 73728
 // Ring slots hold one stage each: the stage image and the kernel-descriptor block of the same 16 channels.
@@ -52,7 +52,7 @@ constexpr int CONSUMER_REGS = 112, OTHER_REGS = 32;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 512;        // 4 consumer warps per lane quarter x 2 filters x 64 columns
 
-struct Params {
+struct Params : ImgGeometry {   // geometry, work items and cut items: see img_geometry.cuh (nct = channel blocks of 16)
   const __half* x;
   __half* y;
   char* images;            // stage images: [region][channel block][IMG_BYTES]
@@ -61,48 +61,12 @@ struct Params {
   const char* dblk;
   const BlobHeader* hdr;
   int* status;
-  int N, H, W, C, F, K, nct;  // nct = channel blocks of 16
-  int Ho, Wo, sub;            // output size; sub = stride - 1: with stride 2 only the results at even rows and columns are written
+  int K;
   long long n_keep;
-  int TY;                  // tile rows per image (ceil(H / 4))
-  int TXe, NI;             // tile columns per region, images side by side
-  int CG, NIG;             // column groups per image, image groups
-  int NG;                  // filter groups (F / 32)
-  int n_regions, n_items;  // n_items = n_regions * NG
-  // Tail balancing: items [0, n_whole) are processed whole, one per block and round.  Each of the n_split items
-  // that would start another, mostly idle round is cut along the input channels into `parts` pieces that run on
-  // different blocks and write fp32 partial sums (`partials`: [piece][32 filters][56 values][32 lanes]);
-  // k_reduce_parts adds them up in a fixed order.  parts == 1: no cutting.
-  int n_whole, n_split, parts;
-  float* partials;
-  FastDiv d_CG, d_TY, d_NG;     // divisions by CG, TY, NG
   unsigned long long wait_ns;   // limit of every wait of the convolution kernel
   int test_skip;           // test hook: the producer never issues the copies of this stage number (-1: none)
   uint16_t masks[256];     // the library (checked against the blob header)
 };
-
-// A region = LY consecutive tile rows (of four pixel rows) x LX column slots.  Tile rows are numbered through all image groups
-// (group g, tile row t -> g * TY + t), so a region may straddle two image groups: it then has two bands,
-// each with its own halo rows.
-struct Region {
-  int cg;           // column group
-  int ig0, ta0, n0; // band 0: image group, first tile row, number of tile rows
-  bool band1;       // band 1 exists (image group ig0 + 1, tile rows 0 .. LY - n0)
-  int nrows;        // image rows in use
-};
-
-__device__ __forceinline__ Region decode_region(const Params& p, int reg) {
-  Region r;
-  const int rb = p.d_CG.div(reg);
-  r.cg = reg - rb * p.CG;
-  const int gt0 = rb * LY;
-  r.ig0 = p.d_TY.div(gt0);
-  r.ta0 = gt0 - r.ig0 * p.TY;
-  r.n0 = min(LY, p.TY - r.ta0);
-  r.band1 = (r.n0 < LY) && (r.ig0 + 1 < p.NIG);
-  r.nrows = r.band1 ? MAXROWS : TR4 * r.n0 + 2;
-  return r;
-}
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -515,9 +479,7 @@ k_conv_f16_img(const Params p) {
 // (cut item, row of the thread tiles): the sums go through shared memory as [448 px][32 channels] and leave as
 // 64-byte runs, like the results of a whole item.  One block per (cut item, row of the thread tiles, half of the
 // tile columns).
-constexpr int MAX_PIECES = 256;            // pieces in flight (the workspace holds that many partial tiles)
-constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
-constexpr int RP_THREADS = 1024, MAX_PARTS = 8, RP_XH = TC / 2;
+constexpr int RP_THREADS = 1024, RP_XH = TC / 2;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");   // launched as a programmatic dependent of the convolution kernel
   if (!blob_matches_block(p)) return;                    // the convolution kernel refused the blob and wrote no partial sums
@@ -572,26 +534,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
 }
 
 // ------------------------------------------------------------------------------------------ host side
-static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
-  p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
-  p.nct = C / CBI;
-  p.TY = std::max((H + TR4 - 1) / TR4, LY / 2);   // a last, partly empty tile row when H is not a multiple of 4; small images take four tile rows
-  const int TX = W < TC ? 1 : W / TC;                // an image narrower than a thread tile takes one tile column
-  p.TXe = TX >= LX ? LX : TX;
-  p.NI = LX / p.TXe;
-  p.CG = TX / p.TXe;
-  p.NIG = (N + p.NI - 1) / p.NI;
-  p.NG = F / FG;
-  const long long row_blocks = ((long long)p.NIG * p.TY + LY - 1) / LY;
-  const long long regions = row_blocks * p.CG;
-  const long long items = regions * p.NG;
-  if (items > 0x7FFFFFFFll || regions * p.nct > 0x7FFFFFFFll) return false;
-  p.n_regions = (int)regions;
-  p.n_items = (int)items;
-  p.n_whole = p.n_items; p.n_split = 0; p.parts = 1; p.partials = nullptr;
-  p.d_CG.set(p.CG); p.d_TY.set(p.TY); p.d_NG.set(p.NG);
-  return true;
-}
+static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) { return imggeo::fill_geometry(p, F, C, N, H, W, CBI); }
 
 }  // namespace img16
 
@@ -608,14 +551,7 @@ int conv_f16_img_debug(int what, long long value) {
 // True when the stage-image kernels cover this layer.
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img16;
-  if (dtype != PAT_F16 || (stride != 1 && stride != 2)) return false;   // stride 2: computed like stride 1, one result in four written
-  const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
-  if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
-  const int TX = W < TC ? 1 : W / TC;
-  if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
-  if (C % kChanTile != 0 || F % FG != 0) return false;
-  Params p;
-  return N >= 1 && fill_geometry(p, F, C, N, H, W);
+  return dtype == PAT_F16 && shape_supported(F, C, N, H, W, stride, kChanTile, CBI);
 }
 
 // Bytes of workspace (the stage images) for a layer the kernels cover; 0 otherwise.
@@ -672,29 +608,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     }
     dv->ready = true;
   }
-  int grid = std::min(p.n_items, sm_count);
-  // fewer work items than half the SMs (small batches): every item is cut along the input channels, so that up to
-  // eight blocks share an item; their partial sums are added by the reduce kernel
-  if (2 * p.n_items <= sm_count) {
-    // a piece keeps at least 32 input channels - below that its partial sums cost more than the idle SMs - unless
-    // the items are so few (a single small image) that the partial sums are a few megabytes in all
-    const int min_channels = p.n_items <= 8 ? CBI : 32;
-    const int parts = std::min(std::min(MAX_PARTS, C / min_channels), std::min(sm_count, MAX_PIECES) / p.n_items);
-    if (parts >= 3) {
-      p.n_whole = 0; p.n_split = p.n_items; p.parts = parts;
-      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nct * IMG_BYTES));
-      grid = p.n_items * parts;
-    }
-  }
-  // the items of a last, mostly idle round are cut into up to eight pieces (see Params)
-  const int left = p.parts > 1 ? 0 : p.n_items % grid;
-  if (left > 0) {
-    const int parts = std::min(std::min(MAX_PARTS, p.nct), std::min(grid, MAX_PIECES) / left);
-    if (parts >= 2) {
-      p.n_whole = p.n_items - left; p.n_split = left; p.parts = parts;
-      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nct * IMG_BYTES));
-    }
-  }
+  const int grid = plan_items(p, sm_count, CBI, reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nct * IMG_BYTES)));
   k_stage_images<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
   // the two kernels that follow are programmatic dependents of their predecessor: the launch itself overlaps the
   // predecessor's tail, the kernels wait for its completion before they touch its results

@@ -10,18 +10,18 @@
 //  * an operation is 32 bytes (four fp32 taps), a window row is four 16-byte loads and plain fp32 multiply-adds;
 //  * the results leave in two rounds (tile rows 0-1, then 2-3): a slot takes one tile row of fp32 results.
 #include <algorithm>
-#include "f16_tile.cuh"
+#include "img_geometry.cuh"
 
 namespace pat {
 namespace img32 {
 using namespace fast16;
+using namespace imggeo;
 
 constexpr int NTHREADS = 640;              // 16 consumer warps, producer warp, three idle warps (register donors)
 constexpr int W_PRODUCER = NCW;
 constexpr int CBI = kChanStageF32;         // channels per ring stage (8)
 constexpr int SEGF = 64;                   // bytes of a segment: 16 px of one channel
 constexpr int ROWF = LX * SEGF;            // 256
-constexpr int MAXROWS = LY * TR4 + 4;      // 36
 constexpr int CHPF = MAXROWS * ROWF;       // channel plane pitch (9216)
 constexpr int IMG_BYTES = CBI * CHPF;      // 73728
 static_assert(ROWF == kImgRowBytesF32 && CHPF == kImgPlaneBytesF32 && NCW == kBlockWarps, "the descriptor blocks are written for this geometry");
@@ -41,7 +41,7 @@ constexpr int CONSUMER_REGS = 112, OTHER_REGS = 32;
 static_assert(NCW * 32 * CONSUMER_REGS + (NTHREADS / 32 - NCW) * 32 * OTHER_REGS <= NTHREADS * LAUNCH_REGS, "register pool of the block");
 constexpr uint32_t TMEM_COLS = 512;
 
-struct Params {
+struct Params : ImgGeometry {   // geometry, work items and cut items: see img_geometry.cuh (nct = stages of 8 channels)
   const float* x;
   float* y;
   char* images;            // stage images: [region][stage of 8 channels][IMG_BYTES]
@@ -50,32 +50,11 @@ struct Params {
   const char* dblk;
   const BlobHeader* hdr;
   int* status;
-  int N, H, W, C, F, K, nst;  // nst = stages of 8 channels
-  int Ho, Wo, sub;            // output size; sub = stride - 1: with stride 2 only the results at even rows and columns are written
+  int K;
   long long n_keep;
-  int TY, TXe, NI, CG, NIG, NG;
-  int n_regions, n_items;
-  int n_whole, n_split, parts;   // cut items: see conv_f16_img.cu
-  float* partials;
   uint16_t masks[256];
 };
 
-struct Region {
-  int cg, ig0, ta0, n0;
-  bool band1;
-  int nrows;
-};
-__device__ __forceinline__ Region decode_region(const Params& p, int reg) {
-  Region r;
-  r.cg = reg % p.CG;
-  const int gt0 = (reg / p.CG) * LY;
-  r.ig0 = gt0 / p.TY;
-  r.ta0 = gt0 % p.TY;
-  r.n0 = min(LY, p.TY - r.ta0);
-  r.band1 = (r.n0 < LY) && (r.ig0 + 1 < p.NIG);
-  r.nrows = r.band1 ? MAXROWS : TR4 * r.n0 + 2;
-  return r;
-}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -91,8 +70,8 @@ constexpr int SI_SMEM = CBI * SI_PITCH;
 __global__ void __launch_bounds__(SI_THREADS) k_stage_images_f32(const Params p) {
   extern __shared__ __align__(16) unsigned char img[];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see conv_f16_img.cu
-  const int st8 = (int)(blockIdx.x % (unsigned)p.nst);
-  const int reg = (int)(blockIdx.x / (unsigned)p.nst);
+  const int st8 = (int)(blockIdx.x % (unsigned)p.nct);
+  const int reg = (int)(blockIdx.x / (unsigned)p.nct);
   const Region r = decode_region(p, reg);
   const int rows0 = TR4 * r.n0 + 2;
   const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
@@ -273,7 +252,7 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 
   const int n_my_whole = (p.n_whole > (int)blockIdx.x) ? (p.n_whole - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const int n_my_items = n_my_whole + ((p.parts > 1 && (int)blockIdx.x < p.n_split * p.parts) ? 1 : 0);
-  const int nst = p.nst;
+  const int nst = p.nct;
   auto item_of = [&](int it_idx) {
     return it_idx < n_my_whole ? (int)blockIdx.x + it_idx * (int)gridDim.x : p.n_whole + (int)blockIdx.x / p.parts;
   };
@@ -554,9 +533,7 @@ k_conv_f32_img(const Params p) {
 // ------------------------------------------------------------------------------------------ cut items
 // Adds the partial sums of the pieces of a cut item (piece 0 first) and writes the results.  One block per
 // (cut item, value of the thread tile); thread = (filter position, lane).
-constexpr int MAX_PIECES = 256;
-constexpr size_t PIECE_FLOATS = (size_t)FG * TR4 * TC * 32;
-constexpr int RP_THREADS = 1024, MAX_PARTS = 8;
+constexpr int RP_THREADS = 1024;
 __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (!blob_matches_block(p)) return;                    // the convolution kernel refused the blob and wrote no partial sums
@@ -581,39 +558,14 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
 }
 
 // ------------------------------------------------------------------------------------------ host side
-static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) {
-  p.N = N; p.H = H; p.W = W; p.C = C; p.F = F;
-  p.nst = C / CBI;
-  p.TY = std::max((H + TR4 - 1) / TR4, LY / 2);   // a last, partly empty tile row when H is not a multiple of 4; small images take four tile rows
-  const int TX = W < TC ? 1 : W / TC;                // an image narrower than a thread tile takes one tile column
-  p.TXe = TX >= LX ? LX : TX;
-  p.NI = LX / p.TXe;
-  p.CG = TX / p.TXe;
-  p.NIG = (N + p.NI - 1) / p.NI;
-  p.NG = F / FG;
-  const long long row_blocks = ((long long)p.NIG * p.TY + LY - 1) / LY;
-  const long long regions = row_blocks * p.CG;
-  const long long items = regions * p.NG;
-  if (items > 0x7FFFFFFFll || regions * p.nst > 0x7FFFFFFFll) return false;
-  p.n_regions = (int)regions;
-  p.n_items = (int)items;
-  p.n_whole = p.n_items; p.n_split = 0; p.parts = 1; p.partials = nullptr;
-  return true;
-}
+static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) { return imggeo::fill_geometry(p, F, C, N, H, W, CBI); }
 
 }  // namespace img32
 
 // True when the fp32 stage-image kernels cover this layer.
 bool conv_f32_img_supported(int F, int C, int dtype, int N, int H, int W, int stride) {
   using namespace img32;
-  if (dtype != PAT_F32 || (stride != 1 && stride != 2)) return false;   // stride 2: computed like stride 1, one result in four written
-  const int TY = std::max((H + TR4 - 1) / TR4, LY / 2);
-  if ((W % TC != 0 && W > TC) || !(TY >= LY - 1 || 2 * TY == LY)) return false;   // a region spans at most two image groups
-  const int TX = W < TC ? 1 : W / TC;
-  if (!(TX == 1 || TX == 2 || TX % 4 == 0)) return false;
-  if (C % kChanTile != 0 || F % FG != 0) return false;
-  Params p;
-  return N >= 1 && fill_geometry(p, F, C, N, H, W);
+  return dtype == PAT_F32 && shape_supported(F, C, N, H, W, stride, kChanTile, CBI);
 }
 
 size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride) {
@@ -621,7 +573,7 @@ size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
   if (!conv_f32_img_supported(F, C, dtype, N, H, W, stride)) return 0;
   Params p;
   if (!fill_geometry(p, F, C, N, H, W)) return 0;
-  return align256((size_t)p.n_regions * p.nst * IMG_BYTES) + MAX_PIECES * PIECE_FLOATS * sizeof(float);
+  return align256((size_t)p.n_regions * p.nct * IMG_BYTES) + MAX_PIECES * PIECE_FLOATS * sizeof(float);
 }
 
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
@@ -669,29 +621,8 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     }
     dv->ready = true;
   }
-  int grid = std::min(p.n_items, sm_count);
-  // fewer work items than half the SMs (small batches): every item is cut along the input channels, so that up to
-  // eight blocks share an item; their partial sums are added by the reduce kernel
-  if (2 * p.n_items <= sm_count) {
-    // a piece keeps at least 32 input channels - below that its partial sums cost more than the idle SMs - unless
-    // the items are so few (a single small image) that the partial sums are a few megabytes in all
-    const int min_channels = p.n_items <= 8 ? CBI : 32;
-    const int parts = std::min(std::min(MAX_PARTS, C / min_channels), std::min(sm_count, MAX_PIECES) / p.n_items);
-    if (parts >= 3) {
-      p.n_whole = 0; p.n_split = p.n_items; p.parts = parts;
-      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nst * IMG_BYTES));
-      grid = p.n_items * parts;
-    }
-  }
-  const int left = p.parts > 1 ? 0 : p.n_items % grid;
-  if (left > 0) {
-    const int parts = std::min(std::min(MAX_PARTS, p.nst), std::min(grid, MAX_PIECES) / left);
-    if (parts >= 2) {
-      p.n_whole = p.n_items - left; p.n_split = left; p.parts = parts;
-      p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nst * IMG_BYTES));
-    }
-  }
-  k_stage_images_f32<<<(unsigned)(p.n_regions * p.nst), SI_THREADS, SI_SMEM, st>>>(p);
+  const int grid = plan_items(p, sm_count, CBI, reinterpret_cast<float*>(static_cast<char*>(workspace) + align256((size_t)p.n_regions * p.nct * IMG_BYTES)));
+  k_stage_images_f32<<<(unsigned)(p.n_regions * p.nct), SI_THREADS, SI_SMEM, st>>>(p);
   cudaLaunchAttribute pdl;
   pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   pdl.val.programmaticStreamSerializationAllowed = 1;
