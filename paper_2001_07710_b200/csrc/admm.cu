@@ -5,23 +5,16 @@
 //   pat_argmax_binarize   the one-hot vector closest to z: 1 at argmax_j z_j
 //   pat_extract_library   "calculate the pattern distribution, remove the patterns with fewest occurrences"
 //
-// The first two stream n x K floats in and out once (8 and 4 - 8 bytes per element): one warp per vector, lanes
-// strided over its entries so that every load and store is a full line.
+// The first two stream n x K floats in and out once (8 and 4 - 8 bytes per element): a vector is shared by the lanes
+// of a warp (or of a group of lanes), strided over its entries so that loads and stores cover whole sectors.
 #include "common.cuh"
 #include "select.cuh"
 
 namespace pat {
 namespace {
 
-constexpr int kVecMaxK = 256;              // entries per vector: eight per lane
-constexpr int kVecPerLane = kVecMaxK / 32;
-constexpr int kVecWarps = 8;               // vectors per block
-
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-  return v;                                // the same bits in every lane: a butterfly adds the same pairs everywhere
-}
+constexpr int kVecMaxK = 256;              // entries per vector
+constexpr int kVecWarps = 8;               // warps per block
 
 // Sums over the L lanes that share a vector (L a power of two, groups aligned): the same bits in every lane of a group.
 template <int L, typename T>
