@@ -79,8 +79,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // with chunk = px >> 3, px = 0..15 <-> image column 14 * (tile column) - 1 + px, and swz(row) = parity of the tile
 // row (counted through both bands) whose window starts in that row's group of four.
 constexpr int SI_THREADS = 256;
-constexpr int SI_PITCH = CHP + 8;          // the two channel octets a warp writes at once fall into different bank halves
-constexpr int SI_SMEM = CBI * SI_PITCH;
+// Channel planes in shared memory: dense (the bulk copies that write them out want 16-byte aligned, contiguous
+// sources), the upper octet 64 bytes further on so that the two channel octets a warp writes at once fall into
+// different bank halves.
+constexpr int SI_SMEM = CBI * CHP + 64;
+__device__ __forceinline__ uint32_t si_plane(int ch) { return (uint32_t)(ch * CHP + (ch >> 3) * 64); }
 __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
   extern __shared__ __align__(16) unsigned char img[];
   // the convolution kernel is launched as a programmatic dependent: its blocks may take over SMs as this grid's
@@ -125,15 +128,20 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
     const uint32_t c[4] = {vb[i].x, vb[i].y, vb[i].z, vb[i].w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j) * SI_PITCH + o) = __byte_perm(a[j], c[j], 0x5410);
-      *reinterpret_cast<uint32_t*>(img + (half * 8 + 2 * j + 1) * SI_PITCH + o) = __byte_perm(a[j], c[j], 0x7632);
+      *reinterpret_cast<uint32_t*>(img + si_plane(half * 8 + 2 * j) + o) = __byte_perm(a[j], c[j], 0x5410);
+      *reinterpret_cast<uint32_t*>(img + si_plane(half * 8 + 2 * j + 1) + o) = __byte_perm(a[j], c[j], 0x7632);
     }
   }
+  // the planes leave by bulk copies (one per channel, issued by sixteen threads): no thread spends load / store
+  // pairs on them, and the block only waits until its shared memory has been read
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stores above, before the copy engine reads them
   __syncthreads();
-  uint2* dst = reinterpret_cast<uint2*>(p.images + (size_t)blockIdx.x * IMG_BYTES);
-  for (int i = threadIdx.x; i < IMG_BYTES / 8; i += SI_THREADS) {
-    const int ch = i / (CHP / 8), w = i % (CHP / 8);
-    dst[i] = *reinterpret_cast<const uint2*>(img + ch * SI_PITCH + w * 8);
+  if (threadIdx.x < CBI) {
+    char* dst = p.images + (size_t)blockIdx.x * IMG_BYTES + (size_t)threadIdx.x * CHP;
+    const uint32_t src = smem_u32(img + si_plane((int)threadIdx.x));
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"((uint32_t)CHP) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
   }
 }
 
