@@ -107,11 +107,15 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images_f32(const Params p)
     *reinterpret_cast<uint32_t*>(img + (quad * 4 + 2) * SI_PITCH + o) = v[i].z;
     *reinterpret_cast<uint32_t*>(img + (quad * 4 + 3) * SI_PITCH + o) = v[i].w;
   }
+  // the planes leave by bulk copies (one per channel; the plane pitch keeps them 16-byte aligned), see conv_f16_img.cu
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
-  uint4* dst = reinterpret_cast<uint4*>(p.images + (size_t)blockIdx.x * IMG_BYTES);
-  for (int i = threadIdx.x; i < IMG_BYTES / 16; i += SI_THREADS) {
-    const int ch = i / (CHPF / 16), w = i % (CHPF / 16);
-    dst[i] = *reinterpret_cast<const uint4*>(img + ch * SI_PITCH + w * 16);
+  if (threadIdx.x < CBI) {
+    char* dst = p.images + (size_t)blockIdx.x * IMG_BYTES + (size_t)threadIdx.x * CHPF;
+    const uint32_t src = smem_u32(img + threadIdx.x * SI_PITCH);
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"((uint32_t)CHPF) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
   }
 }
 
