@@ -97,49 +97,44 @@ __global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float*
   }
 }
 
-// Largest entry of every vector, the lowest index among equal ones; optionally the one-hot vector itself.  A warp
-// takes kArgU vectors per turn and issues all their loads before it looks at any of them: the kernel only streams,
-// and what it needs is bytes in flight.  Q = entries per lane (K <= 32 Q).
-constexpr int kArgU = 4;
-template <int Q>
+// Largest entry of every vector, the lowest index among equal ones; optionally the one-hot vector itself.  As in the
+// projection kernel L lanes share a vector (sixteen entries each, entry j in lane j % L, slot j / L), so a warp has
+// 32 / L vectors in flight and the maximum over a vector takes log2(L) shuffle steps.
+template <int L>
 __global__ void __launch_bounds__(32 * kVecWarps) k_argmax_binarize(const float* __restrict__ z, long long n, int K,
                                                                      unsigned char* __restrict__ index_out,
                                                                      float* __restrict__ onehot_out) {
-  const int lane = threadIdx.x & 31;
-  const long long stride = (long long)gridDim.x * kVecWarps * kArgU;
-  const long long first = ((long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5)) * kArgU;
+  constexpr int G = 32 / L;
+  const int lane = threadIdx.x & 31, sl = lane & (L - 1), g = lane / L;
+  const long long stride = (long long)gridDim.x * kVecWarps * G;
+  const long long first = ((long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5)) * G;
+  if (first >= n) return;                  // whole warps leave together
   for (long long base = first; base < n; base += stride) {
-    float x[kArgU][Q];
+    const bool valid = base + g < n;
+    const long long i = valid ? base + g : n - 1;       // a group without a vector repeats the last one and stores nothing
+    float x[kVecQ];
 #pragma unroll
-    for (int v = 0; v < kArgU; ++v)
+    for (int q = 0; q < kVecQ; ++q) x[q] = (sl + L * q < K) ? __ldcs(z + i * K + sl + L * q) : 0.0f;
+    float best = x[0];                     // entry sl exists: K > 16 (L / 2) >= L > sl for L >= 2, and sl = 0 for L = 1
+    int bj = sl;
 #pragma unroll
-      for (int q = 0; q < Q; ++q) {
-        const int j = lane + 32 * q;
-        x[v][q] = (base + v < n && j < K) ? __ldcs(z + (base + v) * K + j) : 0.0f;
-      }
+    for (int q = 1; q < kVecQ; ++q) {
+      const int j = sl + L * q;
+      if (j < K && x[q] > best) { best = x[q]; bj = j; }   // ascending j inside a lane: the first maximum stays
+    }
 #pragma unroll
-    for (int v = 0; v < kArgU; ++v) {
-      const long long i = base + v;
-      if (i >= n) break;                   // the same decision in every lane
-      float best = 0.0f;
-      int bj = 0x7FFFFFFF;                 // no entry yet
-#pragma unroll
-      for (int q = 0; q < Q; ++q) {
-        const int j = lane + 32 * q;
-        if (j < K && (bj == 0x7FFFFFFF || x[v][q] > best)) { best = x[v][q]; bj = j; }   // ascending j inside a lane: the first maximum stays
-      }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
-        const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
-        if (oj != 0x7FFFFFFF && (bj == 0x7FFFFFFF || ob > best || (ob == best && oj < bj))) { best = ob; bj = oj; }
-      }
-      if (lane == 0) index_out[i] = (unsigned char)bj;
+    for (int off = L / 2; off > 0; off >>= 1) {
+      const float ob = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+      const int oj = __shfl_xor_sync(0xFFFFFFFFu, bj, off);
+      if (ob > best || (ob == best && oj < bj)) { best = ob; bj = oj; }
+    }
+    if (valid) {
+      if (sl == 0) index_out[i] = (unsigned char)bj;
       if (onehot_out) {
         float* oi = onehot_out + i * K;
 #pragma unroll
-        for (int q = 0; q < Q; ++q) {
-          const int j = lane + 32 * q;
+        for (int q = 0; q < kVecQ; ++q) {
+          const int j = sl + L * q;
           if (j < K) __stcs(oi + j, (j == bj) ? 1.0f : 0.0f);
         }
       }
@@ -231,12 +226,13 @@ extern "C" int pat_argmax_binarize(const float* z, int64_t n, int K, uint8_t* in
   if (n < 0 || n > 0x7FFFFFFFll * kVecWarps) return set_error(PAT_ERR_SHAPE, "pat_argmax_binarize: n=%lld out of range", (long long)n);
   if (!aligned(z, 4) || (onehot_out && !aligned(onehot_out, 4))) return set_error(PAT_ERR_ALIGN, "pat_argmax_binarize: buffers must be 4-byte aligned");
   if (n == 0) return PAT_OK;
-  const unsigned grid = vec_grid(n, kArgU);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (K <= 32) k_argmax_binarize<1><<<grid, 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
-  else if (K <= 64) k_argmax_binarize<2><<<grid, 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
-  else if (K <= 128) k_argmax_binarize<4><<<grid, 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
-  else k_argmax_binarize<8><<<grid, 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
+  // the smallest group of lanes that holds the vector (sixteen entries per lane), but never more lanes than entries
+  if (K <= 16) k_argmax_binarize<1><<<vec_grid(n, 32), 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
+  else if (K <= 32) k_argmax_binarize<2><<<vec_grid(n, 16), 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
+  else if (K <= 64) k_argmax_binarize<4><<<vec_grid(n, 8), 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
+  else if (K <= 128) k_argmax_binarize<8><<<vec_grid(n, 4), 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
+  else k_argmax_binarize<16><<<vec_grid(n, 2), 32 * kVecWarps, 0, st>>>(z, (long long)n, K, index_out, onehot_out);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_argmax_binarize launch");
 }
