@@ -26,12 +26,13 @@ __device__ __forceinline__ T group_sum(T v) {
 
 // The root is found without sorting.  g(nu) = sum_j max(d_j - nu, 0) is convex, piecewise linear and decreasing, and
 // Newton's step for g(nu) = 1 from a point nu is nu' = (sum of the entries above nu - 1) / (their number): from any
-// start whose set of entries above it is not empty the steps reach the root in finitely many rounds (after the first
-// step they approach it from below and never pass it), and at the root the set no longer changes.  Most rounds run
-// in fp32, starting with all entries (then every step only drops entries, and the largest one always stays): they
-// find the set of entries above the root up to rounding.  The last rounds repeat the step in fp64 from that set
-// until it is stable - usually one or two - so the result is the exact piece of the equation: the sums are exact to
-// about 1e-16 relative (the inputs are fp32), and there is one rounding to fp32 at the end.
+// start with at least one entry above it the steps reach the root in finitely many rounds (after the first step they
+// approach it from below and never pass it).  The sets {entries above nu} are nested whatever nu is, so two rounds
+// with the same number of entries above nu have the same set, and then nu is the root of that piece: no set has
+// to be stored, a round is one pass "compare, add, count" over the entries.  The rounds run in fp32 from nu = -inf
+// (all entries) until the count repeats, then in fp64 from the fp32 result until the count repeats again - usually
+// two or three rounds - so the final piece and its root are exact: the sums are exact to about 1e-16 relative (the
+// inputs are fp32), and there is one rounding to fp32 at the end.
 //
 // L lanes share a vector, sixteen entries each (K <= 16 L), so a warp works on 32 / L vectors at once: a round is a
 // chain of dependent steps (a sum over the group, a division, a comparison), and what the kernel needs is many such
@@ -44,52 +45,58 @@ __global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float*
   const long long stride = (long long)gridDim.x * kVecWarps * G;
   const long long first = ((long long)blockIdx.x * kVecWarps + (threadIdx.x >> 5)) * G;
   if (first >= n) return;                  // whole warps leave together
-  unsigned exists = 0u;                    // bit q: entry sl + L q exists
-#pragma unroll
-  for (int q = 0; q < kVecQ; ++q) exists |= (sl + L * q < K) ? (1u << q) : 0u;
   for (long long base = first; base < n; base += stride) {
     const bool valid = base + g < n;
     const long long i = valid ? base + g : n - 1;       // a group without a vector repeats the last one and stores nothing
-    float x[kVecQ];
+    float x[kVecQ];                        // slots beyond K hold the lowest float: never above any nu
 #pragma unroll
-    for (int q = 0; q < kVecQ; ++q) x[q] = ((exists >> q) & 1u) ? __ldcs(d + i * K + sl + L * q) : 0.0f;
-    unsigned above = exists;               // bit q: entry q of this lane is above nu
-    for (int round = 0; round < K; ++round) {          // fp32 rounds
+    for (int q = 0; q < kVecQ; ++q) x[q] = (sl + L * q < K) ? __ldcs(d + i * K + sl + L * q) : -3.402823466e38f;
+    float nu32 = -3.402823466e38f;         // every entry of the vector is above it (or equal, if it is that low itself)
+    int before = -1;
+    bool done = false;
+    for (int round = 0; round < K + 2; ++round) {       // fp32 rounds
       float s = 0.0f;
+      int c = 0;
 #pragma unroll
-      for (int q = 0; q < kVecQ; ++q) s += ((above >> q) & 1u) ? x[q] : 0.0f;
+      for (int q = 0; q < kVecQ; ++q) {
+        const bool above = x[q] > nu32;
+        s += above ? x[q] : 0.0f;
+        c += above ? 1 : 0;
+      }
       s = group_sum<L>(s);
-      const int cnt = group_sum<L>(__popc(above));
-      const float nu32 = (s - 1.0f) / (float)cnt;
-      unsigned keep = 0u;
-#pragma unroll
-      for (int q = 0; q < kVecQ; ++q) keep |= (((above >> q) & 1u) && x[q] > nu32) ? (1u << q) : 0u;
-      const bool empty = group_sum<L>(__popc(keep)) == 0;   // rounding only: the group keeps its last set that was not empty
-      const bool changed = !empty && keep != above;
-      if (!empty) above = keep;
-      if (!__any_sync(0xFFFFFFFFu, changed)) break;         // every vector of the warp is through
+      c = group_sum<L>(c);
+      if (!done) {
+        if (c == before || c == 0) done = true;          // the set repeats (or rounding has pushed nu past the largest entry)
+        else { nu32 = (s - 1.0f) / (float)c; before = c; }
+      }
+      if (__all_sync(0xFFFFFFFFu, done)) break;          // every vector of the warp is through
     }
-    double nu = 0.0;
-    for (int round = 0; round < K + 2; ++round) {       // fp64 rounds from the set found
+    double nu = (double)nu32;
+    before = -1;
+    done = false;
+    for (int round = 0; round < K + 3; ++round) {       // fp64 rounds from the fp32 result
       double s = 0.0;
+      int c = 0;
 #pragma unroll
-      for (int q = 0; q < kVecQ; ++q) s += ((above >> q) & 1u) ? (double)x[q] : 0.0;
+      for (int q = 0; q < kVecQ; ++q) {
+        const bool above = (double)x[q] > nu;
+        s += above ? (double)x[q] : 0.0;
+        c += above ? 1 : 0;
+      }
       s = group_sum<L>(s);
-      const int cnt = group_sum<L>(__popc(above));      // >= 1, see above
-      nu = (s - 1.0) / (double)cnt;
-      unsigned now = 0u;
-#pragma unroll
-      for (int q = 0; q < kVecQ; ++q) now |= (((exists >> q) & 1u) && (double)x[q] > nu) ? (1u << q) : 0u;
-      const bool empty = group_sum<L>(__popc(now)) == 0;    // entries too large for the 1 to count
-      const bool changed = !empty && now != above;
-      if (!empty) above = now;
-      if (!__any_sync(0xFFFFFFFFu, changed)) break;
+      c = group_sum<L>(c);
+      if (!done) {
+        if (c == before) done = true;
+        else if (c == 0) { nu = -1.7976931348623157e308; before = -1; }   // past the largest entry: start again from all entries
+        else { nu = (s - 1.0) / (double)c; before = c; }
+      }
+      if (__all_sync(0xFFFFFFFFu, done)) break;
     }
     if (valid) {
       float* ui = u + i * K;
 #pragma unroll
       for (int q = 0; q < kVecQ; ++q)
-        if ((exists >> q) & 1u) {
+        if (sl + L * q < K) {
           const double r = (double)x[q] - nu;
           __stcs(ui + sl + L * q, (float)(r > 0.0 ? r : 0.0));
         }
