@@ -47,6 +47,7 @@ def lib():
         L.orc_simplex_project.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_argmax_binarize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
         L.orc_extract_library.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_relu_maxpool.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p]
         _lib = L
     return _lib
 
@@ -181,3 +182,14 @@ def extract_library(w: np.ndarray, masks: np.ndarray, K_out: int):
     if rc != 0:
         raise ValueError(f"orc_extract_library failed ({rc})")
     return out, counts
+
+
+def relu_maxpool(x: np.ndarray, pool: bool) -> np.ndarray:
+    """max(x, 0) and, if pool, 2x2 max pooling with stride 2, on NHWC x (any float dtype; computed in float64)."""
+    x64 = np.ascontiguousarray(x, dtype=np.float64)
+    N, H, W, Cc = x64.shape
+    y = np.empty((N, H // 2, W // 2, Cc) if pool else (N, H, W, Cc), dtype=np.float64)
+    rc = lib().orc_relu_maxpool(_p(x64), N, H, W, Cc, 1 if pool else 0, _p(y))
+    if rc != 0:
+        raise ValueError(f"orc_relu_maxpool failed ({rc})")
+    return y

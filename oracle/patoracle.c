@@ -28,6 +28,7 @@
  *   orc_extract_library  pinned: for the full 126-mask library the assignment is "the four largest |w|"
  *                        (independent numpy), planted pattern frequencies are recovered; the tie rule and
  *                        the order of the survivors are conventions: "parity unpinned".
+ *   orc_relu_maxpool     pinned: library relu + max_pool2d (float64), hand case.
  */
 #include <math.h>
 #include <stdint.h>
@@ -383,4 +384,30 @@ int orc_extract_library(const float *w, int64_t n, const uint16_t *masks_in, int
         if (before < K_out) masks_out[m++] = masks_in[j];
     }
     return m == K_out ? 0 : 2;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * What stands between two convolution layers of the VGG-16 / ResNet models of Section 7: the
+ * rectifier max(x, 0) and, after some layers, 2x2 max pooling with stride 2 (the models' own
+ * definition, not the paper's).  NHWC, values given as float64; pool = 0: rectifier only,
+ * pool = 1: rectifier, then the maximum over each 2x2 block (H and W even).
+ * ---------------------------------------------------------------------------------------- */
+int orc_relu_maxpool(const double *x, int N, int H, int W, int C, int pool, double *y) {
+    if (pool != 0 && pool != 1) return 1;
+    if (pool && ((H & 1) || (W & 1))) return 1;
+    const int Ho = pool ? H / 2 : H, Wo = pool ? W / 2 : W;
+    for (int n = 0; n < N; ++n)
+        for (int yo = 0; yo < Ho; ++yo)
+            for (int xo = 0; xo < Wo; ++xo)
+                for (int c = 0; c < C; ++c) {
+                    double m = 0.0;                       /* the rectifier's floor */
+                    const int k = pool ? 2 : 1;
+                    for (int dy = 0; dy < k; ++dy)
+                        for (int dx = 0; dx < k; ++dx) {
+                            const double v = x[(((int64_t)n * H + yo * k + dy) * W + xo * k + dx) * C + c];
+                            if (v > m) m = v;
+                        }
+                    y[(((int64_t)n * Ho + yo) * Wo + xo) * C + c] = m;
+                }
+    return 0;
 }

@@ -153,3 +153,20 @@ def test_extraction_tie_rules():
     out, counts = oracle.extract_library(np.zeros((10, 3, 3), dtype=np.float32), masks, 3)
     assert counts[0] == 10 and counts[1:].sum() == 0
     assert list(out) == [int(m) for m in masks[:3]]
+
+
+# ----------------------------------------------------------------------------------------- rectifier and pooling
+def test_relu_maxpool_matches_library_ops():
+    import torch
+    rng = np.random.default_rng(10)
+    x = rng.standard_normal((2, 6, 8, 5))
+    t = torch.from_numpy(x).permute(0, 3, 1, 2)
+    relu = torch.relu(t)
+    assert np.array_equal(oracle.relu_maxpool(x, False), relu.permute(0, 2, 3, 1).numpy())
+    pooled = torch.nn.functional.max_pool2d(relu, 2, 2).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(oracle.relu_maxpool(x, True), pooled)
+    # by hand: one channel, one 2x2 block; all negative -> 0
+    assert oracle.relu_maxpool(np.array([[[[-1.0], [3.0]], [[2.0], [-5.0]]]]), True).tolist() == [[[[3.0]]]]
+    assert oracle.relu_maxpool(np.array([[[[-1.0], [-3.0]], [[-2.0], [-5.0]]]]), True).tolist() == [[[[0.0]]]]
+    with pytest.raises(ValueError):
+        oracle.relu_maxpool(np.zeros((1, 3, 4, 1)), True)
