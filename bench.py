@@ -438,6 +438,15 @@ def admm_primitives(pc, torch, peaks, with_cpu: bool, reps: int = 10):
                                "bytes": "read once, one index byte per vector"},
            "extract_library_126_to_12": {"ms": round(t_ex * 1e3, 4), "kernels_per_s": round(n / t_ex, 0),
                                          "note": "a memset and two launches; 126 mask energies per kernel (fp32, exact fp64 fallback): arithmetic, not memory"}}
+    # the rectifier and 2x2 max pooling after the second VGG-16 layer: 64 x 224 x 224 x 64 fp16 in, a quarter out
+    xa = torch.randn((64, 224, 224, 64), dtype=torch.float16, device="cuda")
+    ya = torch.empty((64, 112, 112, 64), dtype=torch.float16, device="cuda")
+    t_rp = timed(lambda: pc.pat_relu_maxpool(xa, "f16", True, ya))
+    by = (xa.numel() + ya.numel()) * 2.0
+    res["relu_maxpool_vgg_conv2_output"] = {"ms": round(t_rp * 1e3, 4), "GB/s": round(by / t_rp / 1e9, 1),
+                                            "roofline": {"bound": "hbm", "peak": hbm, "frac": round(by / t_rp / 1e9 / hbm, 4)},
+                                            "bytes": "input read once, output written once (514 MB)"}
+    del xa, ya
     if with_cpu:
         import oracle
         m = 8192                                      # a bounded sample of the same vectors / kernels

@@ -202,6 +202,17 @@ uint64_t pat_launch_count(void);
  * The paper has no counterpart (it reports end-to-end latencies, Section 7.2). */
 int pat_measure_fma_peak(int kind, void *scratch, size_t scratch_bytes, double *tflops_out, void *stream);
 
+/* What stands between two convolution layers of the models the paper evaluates (Section 7: VGG-16, ResNet-50; their
+ * own definition, the paper adds nothing to it): the rectifier max(x, 0) and, with pool = 1, 2x2 max pooling with
+ * stride 2 after it.
+ *   x      dev in  NHWC [N][H][W][C], dtype PAT_F32 or PAT_F16, finite values
+ *   y      dev out NHWC [N][H][W][C] (pool = 0; may be x itself) or [N][H/2][W/2][C] (pool = 1; H and W even, y must
+ *          not overlap x)
+ * One pass over the data; 16-byte accesses when C * (element size) is a multiple of 16 and both buffers are 16-byte
+ * aligned, element by element otherwise.  Asynchronous on `stream`; allocates nothing.
+ * Errors: PAT_ERR_INVALID_ARG, PAT_ERR_DTYPE, PAT_ERR_SHAPE (odd H or W with pool = 1), PAT_ERR_ALIGN, PAT_ERR_CUDA. */
+int pat_relu_maxpool(const void *x, int dtype, int N, int H, int W, int C, int pool, void *y, void *stream);
+
 /* ---- Primitives of the pattern-selection ADMM and of the library extraction (training side; the loop around them,
  * the loss and the data are not part of this library).  All pointers are device pointers unless marked host. ---- */
 

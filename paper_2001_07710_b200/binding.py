@@ -25,7 +25,7 @@ EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
            "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels",
            "pat_conv3x3_workspace", "pat_conv3x3_ws", "pat_debug_set", "pat_measure_fma_peak",
-           "pat_simplex_project", "pat_argmax_binarize", "pat_extract_library"]
+           "pat_simplex_project", "pat_argmax_binarize", "pat_extract_library", "pat_relu_maxpool"]
 
 
 class PatError(RuntimeError):
@@ -68,6 +68,7 @@ def load() -> C.CDLL:
     L.pat_simplex_project.argtypes = [vp, i64, i32, vp, vp]
     L.pat_argmax_binarize.argtypes = [vp, i64, i32, vp, vp, vp]
     L.pat_extract_library.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp]
+    L.pat_relu_maxpool.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp]
     _lib = L
     return L
 
@@ -239,6 +240,15 @@ def pat_extract_library(w: torch.Tensor, masks, K_out: int, masks_out: Optional[
     _check(load().pat_extract_library(_ptr(w), n, m.ctypes.data, len(m), int(K_out), _ptr(masks_out), _ptr(counts),
                                       _stream(stream)))
     return masks_out, counts
+
+
+def pat_relu_maxpool(x: torch.Tensor, dtype, pool: bool, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """x: cuda NHWC.  Returns max(x, 0), 2x2 max-pooled with stride 2 when pool is set."""
+    N, H, W, Cc = (int(v) for v in x.shape)
+    if y is None:
+        y = torch.empty((N, H // 2, W // 2, Cc) if pool else (N, H, W, Cc), dtype=x.dtype, device=x.device)
+    _check(load().pat_relu_maxpool(_ptr(x), _DT[dtype], N, H, W, Cc, 1 if pool else 0, _ptr(y), _stream(stream)))
+    return y
 
 
 def pat_debug_set(what: int, value: int) -> None:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpatconv.so")
-SOURCES = ["api.cu", "project.cu", "pack.cu", "conv_generic.cu", "conv_dense_mma.cu", "conv_f16_fast.cu", "conv_f16_img.cu", "conv_f32_img.cu", "conv_api.cu", "fma_peak.cu", "admm.cu"]
+SOURCES = ["api.cu", "project.cu", "pack.cu", "conv_generic.cu", "conv_dense_mma.cu", "conv_f16_fast.cu", "conv_f16_img.cu", "conv_f32_img.cu", "conv_api.cu", "fma_peak.cu", "admm.cu", "activation.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
 

@@ -124,3 +124,32 @@ def test_library_extraction_schedule_and_ties():
     assert np.array_equal(pid.cpu().numpy(), pid_o)
     with pytest.raises(pc.PatError):
         pc.pat_extract_library(wg, masks_g, 5)             # more than the library holds
+
+
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+@pytest.mark.parametrize("shape", [(2, 8, 12, 64), (1, 14, 14, 24), (3, 6, 10, 5), (1, 2, 2, 1), (2, 56, 56, 128)])
+@pytest.mark.parametrize("pool", [False, True])
+def test_relu_maxpool_matches_oracle(dtype, shape, pool):
+    """The rectifier and 2x2 max pooling between layers: the maximum of stored values is exact, so the comparison is too."""
+    rng = np.random.default_rng(sum(shape) + pool)
+    npdt, tdt = (np.float16, torch.float16) if dtype == "f16" else (np.float32, torch.float32)
+    x = rng.standard_normal(shape).astype(npdt)
+    ref = oracle.relu_maxpool(x, pool)
+    N, H, W, Cc = shape
+    n_out = ref.size
+    buf = torch.full((n_out + 64,), 7.0, dtype=tdt, device="cuda")
+    y = buf[32:32 + n_out].view(ref.shape)
+    pc.pat_relu_maxpool(torch.from_numpy(x).cuda(), dtype, pool, y)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy().astype(np.float64), ref)
+    assert bool((buf[:32] == 7.0).all()) and bool((buf[32 + n_out:] == 7.0).all())
+    assert pc.pat_query_status() == 0
+
+
+def test_relu_maxpool_refuses_odd_sizes_and_runs_in_place():
+    x = torch.randn((1, 5, 6, 8), device="cuda")
+    with pytest.raises(pc.PatError):
+        pc.pat_relu_maxpool(x, "f32", True)
+    ref = oracle.relu_maxpool(x.cpu().numpy(), False)
+    pc.pat_relu_maxpool(x, "f32", False, x)
+    assert np.array_equal(x.cpu().numpy().astype(np.float64), ref)
