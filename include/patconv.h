@@ -171,6 +171,15 @@ int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K,
                    int dtype, const void *x, void *y, int N, int H, int W, int stride,
                    void *workspace, size_t workspace_bytes, void *stream);
 
+/* pat_conv3x3_ws with the rectifier that follows the layer in the models of Section 7 fused into its epilogue
+ * (the graph-level fusion of Section 6.2): act = 1 writes max(result, 0), act = 0 is pat_conv3x3_ws.  The workspace
+ * kernels apply it to the fp32 sums before they are rounded and stored, at no extra pass over the output; a layer
+ * they do not cover runs the plain convolution and then pat_relu_maxpool in place (same result).  Arguments, errors
+ * and workspace as for pat_conv3x3_ws; PAT_ERR_INVALID_ARG for any other `act`. */
+int pat_conv3x3_ws_act(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
+                       int dtype, const void *x, void *y, int N, int H, int W, int stride, int act,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
 /* Dense 3x3 convolution for layers that are not pruned: the first layer of the VGG-16 of Section 7
  * (C = 3 input channels), which stays dense when the other twelve are pattern-pruned.
  *   w   dev, [F][C][3][3] fp32 (converted to the activation type on the fly)

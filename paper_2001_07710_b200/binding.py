@@ -25,7 +25,7 @@ EXPORTS = ["pat_strerror", "pat_last_error", "pat_library_builtin", "pat_project
            "pat_pack_size", "pat_pack", "pat_blob_layout", "pat_unpack", "pat_conv3x3", "pat_conv3x3_dense",
            "pat_query_status", "pat_launch_count", "pat_project_static", "pat_project_static_max_kernels",
            "pat_conv3x3_workspace", "pat_conv3x3_ws", "pat_debug_set", "pat_measure_fma_peak",
-           "pat_simplex_project", "pat_argmax_binarize", "pat_extract_library", "pat_relu_maxpool"]
+           "pat_simplex_project", "pat_argmax_binarize", "pat_extract_library", "pat_relu_maxpool", "pat_conv3x3_ws_act"]
 
 
 class PatError(RuntimeError):
@@ -69,6 +69,7 @@ def load() -> C.CDLL:
     L.pat_argmax_binarize.argtypes = [vp, i64, i32, vp, vp, vp]
     L.pat_extract_library.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp]
     L.pat_relu_maxpool.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp]
+    L.pat_conv3x3_ws_act.argtypes = [vp, i32, i32, vp, i32, i64, i32, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
     _lib = L
     return L
 
@@ -157,7 +158,7 @@ def pat_conv3x3_workspace(F: int, Cc: int, dtype, N: int, H: int, W: int, stride
 
 def pat_conv3x3(blob: torch.Tensor, F: int, Cc: int, masks, n_keep: int, dtype, x: torch.Tensor,
                 stride: int = 1, y: Optional[torch.Tensor] = None, stream=None,
-                workspace: Optional[torch.Tensor] = None, use_workspace: bool = True) -> torch.Tensor:
+                workspace: Optional[torch.Tensor] = None, use_workspace: bool = True, relu: bool = False) -> torch.Tensor:
     """x: cuda NHWC [N,H,W,C] in the blob's dtype.  Returns y NHWC [N,Ho,Wo,F].
 
     Calls pat_conv3x3_ws with `workspace` (a cuda uint8 tensor, allocated here when None and the layer wants
@@ -167,6 +168,13 @@ def pat_conv3x3(blob: torch.Tensor, F: int, Cc: int, masks, n_keep: int, dtype, 
     if y is None:
         y = torch.empty((N, (H - 1) // stride + 1, (W - 1) // stride + 1, F), dtype=x.dtype, device=x.device)
     need = pat_conv3x3_workspace(F, Cc, dtype, N, H, W, stride) if use_workspace else 0
+    if relu:
+        # the rectifier fused into the epilogue (pat_conv3x3_ws_act; layers without workspace kernels: convolution + rectifier)
+        if workspace is None:
+            workspace = torch.empty(max(pat_conv3x3_workspace(F, Cc, dtype, N, H, W, stride), 256), dtype=torch.uint8, device=x.device)
+        _check(load().pat_conv3x3_ws_act(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
+                                         N, H, W, int(stride), 1, _ptr(workspace), int(workspace.numel()), _stream(stream)))
+        return y
     if need == 0:
         _check(load().pat_conv3x3(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
                                   N, H, W, int(stride), _stream(stream)))

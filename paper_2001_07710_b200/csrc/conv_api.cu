@@ -10,11 +10,11 @@ int conv_f16_fast(const void* blob, int F, int C, const uint16_t* masks, int K, 
 bool conv_f16_img_supported(int F, int C, int dtype, int N, int H, int W, int stride);
 size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
+                 const void* x, void* y, int N, int H, int W, int stride, int relu, void* workspace, cudaStream_t st);
 int conv_f16_img_debug(int what, long long value);
 size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int stride);
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st);
+                 const void* x, void* y, int N, int H, int W, int stride, int relu, void* workspace, cudaStream_t st);
 }
 
 using namespace pat;
@@ -51,15 +51,29 @@ extern "C" size_t pat_conv3x3_workspace(int F, int C, int dtype, int N, int H, i
   return dtype == PAT_F32 ? conv_f32_img_workspace(F, C, dtype, N, H, W, stride) : conv_f16_img_workspace(F, C, dtype, N, H, W, stride);
 }
 
-extern "C" int pat_conv3x3_ws(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                              int dtype, const void* x, void* y, int N, int H, int W, int stride,
-                              void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int pat_relu_maxpool(const void* x, int dtype, int N, int H, int W, int C, int pool, void* y, void* stream);
+
+extern "C" int pat_conv3x3_ws_act(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                                  int dtype, const void* x, void* y, int N, int H, int W, int stride, int act,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+  if (act != 0 && act != 1) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3_ws_act: act %d (0: none, 1: rectifier)", act);
   if (int rc = check_conv_args(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride)) return rc;
   const size_t need = pat_conv3x3_workspace(F, C, dtype, N, H, W, stride);
-  if (need == 0) return pat_conv3x3(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, stream);
+  if (need == 0) {
+    // a layer the workspace kernels do not cover: the plain convolution, then the rectifier in place
+    if (int rc = pat_conv3x3(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, stream)) return rc;
+    if (!act) return PAT_OK;
+    return pat_relu_maxpool(y, dtype, N, (H - 1) / stride + 1, (W - 1) / stride + 1, F, 0, y, stream);
+  }
   if (!workspace || workspace_bytes < need)
     return set_error(PAT_ERR_WORKSPACE, "pat_conv3x3_ws: workspace has %zu bytes, needs %zu", workspace_bytes, need);
   if (!aligned(workspace, 256)) return set_error(PAT_ERR_ALIGN, "pat_conv3x3_ws: workspace must be 256-byte aligned");
-  if (dtype == PAT_F32) return conv_f32_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, workspace, reinterpret_cast<cudaStream_t>(stream));
-  return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, workspace, reinterpret_cast<cudaStream_t>(stream));
+  if (dtype == PAT_F32) return conv_f32_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, act, workspace, reinterpret_cast<cudaStream_t>(stream));
+  return conv_f16_img(blob, F, C, masks, K, n_keep, x, y, N, H, W, stride, act, workspace, reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pat_conv3x3_ws(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
+                              int dtype, const void* x, void* y, int N, int H, int W, int stride,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+  return pat_conv3x3_ws_act(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, 0, workspace, workspace_bytes, stream);
 }

@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
 // In a real stage a consumer warp runs the operations of its list in the stage's descriptor block: the kernels of the
 // filter whose tile it holds, a swap of the two accumulator tiles through tensor memory if its other filter has
 // kernels in this stage, and those kernels; the next stage starts with the tile it then holds.
-template <bool SPARSE, int NCODES, bool GENERIC>
+template <bool SPARSE, int NCODES, bool GENERIC, bool RELU>
 __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
   constexpr int NS = SPARSE ? 3 : 2;
   constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
@@ -376,6 +376,12 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           const uint32_t cp = ol + (cur ? cposB : cposA);
+          if constexpr (RELU) {              // the fused rectifier: a kernel of its own, so that the plain one pays nothing
+#pragma unroll
+            for (int y = 0; y < TR4; ++y)
+#pragma unroll
+              for (int x = 0; x < TC; ++x) acc[y][x] = fmaxf(acc[y][x], 0.0f);
+          }
 #pragma unroll
           for (int y = 0; y < TR4; ++y)
 #pragma unroll
@@ -462,8 +468,8 @@ __device__ __forceinline__ bool blob_matches_block(const Params& p) {
 }
 
 // NCODES / GENERIC: the pattern codes the kernel carries code for (see one_kernel4); the host picks the smallest
-// set that covers the library.
-template <int NCODES, bool GENERIC>
+// set that covers the library.  RELU: results below zero are written as zero.
+template <int NCODES, bool GENERIC, bool RELU>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f16_img(const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -478,8 +484,8 @@ k_conv_f16_img(const Params p) {
   // everything below reads the stage images or writes the output: the stage-image grid must be complete
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // ring geometry by the size of the largest descriptor block (see MAX_NS above)
-  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC>(p, smem);
-  else conv_body<false, NCODES, GENERIC>(p, smem);
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC, RELU>(p, smem);
+  else conv_body<false, NCODES, GENERIC, RELU>(p, smem);
 }
 
 // ------------------------------------------------------------------------------------------ cut items
@@ -517,7 +523,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
 #pragma unroll
     for (int q = 0; q < MAX_PARTS; ++q) sum += v[i][q];       // piece 0 first
     const int cpos = (__ldg(p.xfilt + g * FG + slot) & (FG - 1)) * 2;
-    *reinterpret_cast<__half*>(stage + (lane * TC + x) * OUT_PITCH + cpos) = __float2half_rn(sum);
+    *reinterpret_cast<__half*>(stage + (lane * TC + x) * OUT_PITCH + cpos) = __float2half_rn(p.relu ? fmaxf(sum, 0.0f) : sum);
   }
   __syncthreads();
   const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
@@ -572,7 +578,7 @@ size_t conv_f16_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
 }
 
 int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st) {
+                 const void* x, void* y, int N, int H, int W, int stride, int relu, void* workspace, cudaStream_t st) {
   using namespace img16;
   const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F16);
   const char* b = static_cast<const char*>(blob);
@@ -589,7 +595,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
   p.wait_ns = g_wait_ns; p.test_skip = g_test_skip;
-  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
+  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1; p.relu = relu;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   // the smallest set of compiled pattern codes that covers the library
@@ -599,7 +605,8 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     variant = std::max(variant, code == kGenericCode ? 2 : (code >= 6 ? 1 : 0));
   }
   using KernelFn = void (*)(const Params);
-  static const KernelFn kernels[3] = {k_conv_f16_img<6, false>, k_conv_f16_img<kNumCodes, false>, k_conv_f16_img<kNumCodes, true>};
+  static const KernelFn kernels[6] = {k_conv_f16_img<6, false, false>, k_conv_f16_img<kNumCodes, false, false>, k_conv_f16_img<kNumCodes, true, false>,
+                                      k_conv_f16_img<6, false, true>, k_conv_f16_img<kNumCodes, false, true>, k_conv_f16_img<kNumCodes, true, true>};
 
   static thread_local DeviceSlot slots[kMaxDevices];
   DeviceSlot* dv = device_slot(slots);
@@ -626,7 +633,7 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   cudaLaunchConfig_t cfg = {};
   cfg.stream = st; cfg.attrs = &pdl; cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM_BYTES;
-  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant], p), "pat_conv3x3 launch")) return rc;
+  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant + (relu ? 3 : 0)], p), "pat_conv3x3 launch")) return rc;
   count_launches(2);
   if (p.parts > 1) {
     cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * 2)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;

@@ -430,6 +430,12 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           const uint32_t cp = ol + (cur ? cposB : cposA);
+          if (p.relu) {                      // the fused rectifier (a tile parked between the rounds is clamped twice: harmless)
+#pragma unroll
+            for (int y = 0; y < TR4; ++y)
+#pragma unroll
+              for (int x = 0; x < TC; ++x) acc[y][x] = fmaxf(acc[y][x], 0.0f);
+          }
 #pragma unroll
           for (int x = 0; x < TC; ++x) {
             sts32(ob0 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[2][x] : acc[0][x]));
@@ -558,7 +564,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
   const int n_img = ig * p.NI + ni;
   const int row = TR4 * ty + v / TC, col = (it.cg * p.TXe + tx) * TC + v % TC;
   if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || row >= p.H || col >= p.W || ((row | col) & p.sub) != 0) return;
-  p.y[(((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo + (col >> p.sub)) * p.F + __ldg(p.xfilt + g * FG + slot)] = sum;
+  p.y[(((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo + (col >> p.sub)) * p.F + __ldg(p.xfilt + g * FG + slot)] = p.relu ? fmaxf(sum, 0.0f) : sum;
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -581,7 +587,7 @@ size_t conv_f32_img_workspace(int F, int C, int dtype, int N, int H, int W, int 
 }
 
 int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
-                 const void* x, void* y, int N, int H, int W, int stride, void* workspace, cudaStream_t st) {
+                 const void* x, void* y, int N, int H, int W, int stride, int relu, void* workspace, cudaStream_t st) {
   using namespace img32;
   const BlobLayout L = blob_layout(F, C, K, n_keep, PAT_F32);
   const char* b = static_cast<const char*>(blob);
@@ -597,7 +603,7 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.status = status_word();
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
-  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
+  p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1; p.relu = relu;
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   int variant = 0;

@@ -474,3 +474,30 @@ def test_bounded_wait_runs_out_and_is_reported():
     y = pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", xt, 1)
     assert pc.pat_query_status() == 0
     check_close(y.float().cpu().numpy(), oracle.conv3x3(stored_weights(wm_o, "f16"), x, 1), "f16")
+
+
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+@pytest.mark.parametrize("case", [(3, 56, 56, 32, 64, 8, 1, 4, 1), (5, 14, 14, 64, 32, 8, 1, 2, 1), (2, 28, 28, 16, 32, 12, 1, 1, 2),
+                                  (24, 28, 56, 64, 64, 8, 1, 8, 1), (1, 28, 28, 64, 64, 8, 1, 8, 1), (2, 23, 17, 24, 40, 8, 1, 2, 1)])
+def test_conv_with_fused_rectifier(case, dtype):
+    """pat_conv3x3_ws_act: max(conv, 0) written by the convolution's own epilogue (whole items, cut items whose sums
+    pass through the reduce kernel, a small batch that is cut entirely, stride 2, and a shape the workspace kernels do
+    not cover: convolution, then the rectifier in place) - every element against the oracle's relu(conv)."""
+    N, H, W, C, F, K, num, den, stride = case
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 5)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = np.maximum(oracle.conv3x3(stored_weights(wm_o, dtype), x, stride), 0.0)
+    assert (ref == 0).mean() > 0.2                      # the rectifier has something to do
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    y = pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, torch.from_numpy(x).cuda(), stride, relu=True)
+    assert pc.pat_query_status() == 0
+    out = y.float().cpu().numpy()
+    assert tuple(out.shape) == ref.shape and (out >= 0).all()
+    check_close(out, ref, dtype)
+    # where the reference is clearly negative before the rectifier the output is exactly zero
+    pre = oracle.conv3x3(stored_weights(wm_o, dtype), x, stride)
+    assert (out[pre < -1e-2] == 0).all()
