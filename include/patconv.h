@@ -174,8 +174,14 @@ int pat_conv3x3_ws(const void *blob, int F, int C, const uint16_t *masks, int K,
 /* pat_conv3x3_ws with the rectifier that follows the layer in the models of Section 7 fused into its epilogue
  * (the graph-level fusion of Section 6.2): act = 1 writes max(result, 0), act = 0 is pat_conv3x3_ws.  The workspace
  * kernels apply it to the fp32 sums before they are rounded and stored, at no extra pass over the output; a layer
- * they do not cover runs the plain convolution and then pat_relu_maxpool in place (same result).  Arguments, errors
- * and workspace as for pat_conv3x3_ws; PAT_ERR_INVALID_ARG for any other `act`. */
+ * they do not cover runs the plain convolution and then pat_relu_maxpool in place (same result).
+ * act = 2 fuses the 2 x 2 max pooling that follows five of the thirteen layers of the VGG-16 of Section 7 as well:
+ * y is then NHWC [N][H/2][W/2][F] and holds max(0, the four results of each 2 x 2 block) - the values of
+ * pat_relu_maxpool(pool = 1) on the output of act = 0, bit for bit (rounding is monotone) - and the full-size
+ * output is never written.  act = 2 needs stride 1, even H and W and a layer the workspace kernels cover
+ * (pat_conv3x3_workspace(...) > 0): PAT_ERR_SHAPE otherwise, nothing launched; such a layer takes act = 1 and a
+ * separate pat_relu_maxpool.  Other arguments, errors and workspace as for pat_conv3x3_ws; PAT_ERR_INVALID_ARG for
+ * any other `act`. */
 int pat_conv3x3_ws_act(const void *blob, int F, int C, const uint16_t *masks, int K, int64_t n_keep,
                        int dtype, const void *x, void *y, int N, int H, int W, int stride, int act,
                        void *workspace, size_t workspace_bytes, void *stream);

@@ -158,22 +158,25 @@ def pat_conv3x3_workspace(F: int, Cc: int, dtype, N: int, H: int, W: int, stride
 
 def pat_conv3x3(blob: torch.Tensor, F: int, Cc: int, masks, n_keep: int, dtype, x: torch.Tensor,
                 stride: int = 1, y: Optional[torch.Tensor] = None, stream=None,
-                workspace: Optional[torch.Tensor] = None, use_workspace: bool = True, relu: bool = False) -> torch.Tensor:
-    """x: cuda NHWC [N,H,W,C] in the blob's dtype.  Returns y NHWC [N,Ho,Wo,F].
+                workspace: Optional[torch.Tensor] = None, use_workspace: bool = True, relu: bool = False,
+                pool: bool = False) -> torch.Tensor:
+    """x: cuda NHWC [N,H,W,C] in the blob's dtype.  Returns y NHWC [N,Ho,Wo,F]; relu / pool: pat_conv3x3_ws_act with
+    act = 1 (rectifier) or act = 2 (rectifier and 2 x 2 max pooling: y is [N,H/2,W/2,F]).
 
     Calls pat_conv3x3_ws with `workspace` (a cuda uint8 tensor, allocated here when None and the layer wants
     one); use_workspace=False calls the entry point without workspace, pat_conv3x3."""
     m = _masks(masks)
     N, H, W = int(x.shape[0]), int(x.shape[1]), int(x.shape[2])
     if y is None:
-        y = torch.empty((N, (H - 1) // stride + 1, (W - 1) // stride + 1, F), dtype=x.dtype, device=x.device)
+        Ho, Wo = ((H // 2, W // 2) if pool else ((H - 1) // stride + 1, (W - 1) // stride + 1))
+        y = torch.empty((N, Ho, Wo, F), dtype=x.dtype, device=x.device)
     need = pat_conv3x3_workspace(F, Cc, dtype, N, H, W, stride) if use_workspace else 0
-    if relu:
+    if relu or pool:
         # the rectifier fused into the epilogue (pat_conv3x3_ws_act; layers without workspace kernels: convolution + rectifier)
         if workspace is None:
             workspace = torch.empty(max(pat_conv3x3_workspace(F, Cc, dtype, N, H, W, stride), 256), dtype=torch.uint8, device=x.device)
         _check(load().pat_conv3x3_ws_act(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),
-                                         N, H, W, int(stride), 1, _ptr(workspace), int(workspace.numel()), _stream(stream)))
+                                         N, H, W, int(stride), 2 if pool else 1, _ptr(workspace), int(workspace.numel()), _stream(stream)))
         return y
     if need == 0:
         _check(load().pat_conv3x3(_ptr(blob), F, Cc, m.ctypes.data, len(m), int(n_keep), _DT[dtype], _ptr(x), _ptr(y),

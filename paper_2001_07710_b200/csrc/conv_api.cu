@@ -56,9 +56,14 @@ extern "C" int pat_relu_maxpool(const void* x, int dtype, int N, int H, int W, i
 extern "C" int pat_conv3x3_ws_act(const void* blob, int F, int C, const uint16_t* masks, int K, int64_t n_keep,
                                   int dtype, const void* x, void* y, int N, int H, int W, int stride, int act,
                                   void* workspace, size_t workspace_bytes, void* stream) {
-  if (act != 0 && act != 1) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3_ws_act: act %d (0: none, 1: rectifier)", act);
+  if (act < 0 || act > 2) return set_error(PAT_ERR_INVALID_ARG, "pat_conv3x3_ws_act: act %d (0: none, 1: rectifier, 2: rectifier and 2 x 2 max pooling)", act);
   if (int rc = check_conv_args(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride)) return rc;
   const size_t need = pat_conv3x3_workspace(F, C, dtype, N, H, W, stride);
+  // pooling happens inside a thread tile of the workspace kernels: no other kernel writes a pooled image (y is too
+  // small for the full-size result, so there is no two-pass substitute without memory of the library's own)
+  if (act == 2 && (need == 0 || stride != 1 || (H & 1) || (W & 1)))
+    return set_error(PAT_ERR_SHAPE, "pat_conv3x3_ws_act: act 2 needs a layer the workspace kernels cover, stride 1, even H and W "
+                                    "(otherwise: act 1, then pat_relu_maxpool)");
   if (need == 0) {
     // a layer the workspace kernels do not cover: the plain convolution, then the rectifier in place
     if (int rc = pat_conv3x3(blob, F, C, masks, K, n_keep, dtype, x, y, N, H, W, stride, stream)) return rc;

@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(SI_THREADS) k_stage_images(const Params p) {
 // In a real stage a consumer warp runs the operations of its list in the stage's descriptor block: the kernels of the
 // filter whose tile it holds, a swap of the two accumulator tiles through tensor memory if its other filter has
 // kernels in this stage, and those kernels; the next stage starts with the tile it then holds.
-template <bool SPARSE, int NCODES, bool GENERIC, bool RELU>
+template <bool SPARSE, int NCODES, bool GENERIC, int ACT>
 __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) {
   constexpr int NS = SPARSE ? 3 : 2;
   constexpr uint32_t SLOT = (uint32_t)IMG_BYTES + (uint32_t)(SPARSE ? DBLK3 : DBLK2);
@@ -376,17 +376,31 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           const uint32_t cp = ol + (cur ? cposB : cposA);
-          if constexpr (RELU) {              // the fused rectifier: a kernel of its own, so that the plain one pays nothing
+          if constexpr (ACT == 1) {          // the fused rectifier: a kernel of its own, so that the plain one pays nothing
 #pragma unroll
             for (int y = 0; y < TR4; ++y)
 #pragma unroll
               for (int x = 0; x < TC; ++x) acc[y][x] = fmaxf(acc[y][x], 0.0f);
           }
+          if constexpr (ACT == 2) {
+            // rectifier and 2 x 2 max pooling: a thread tile starts at an even row and column, so every pooling window
+            // lies inside one lane's registers; the 2 x 7 pooled values take the first output stage (rounding is
+            // monotone: the maximum of the fp32 sums rounds to the maximum of the rounded results)
 #pragma unroll
-          for (int y = 0; y < TR4; ++y)
+            for (int yy = 0; yy < TR4 / 2; ++yy)
 #pragma unroll
-            for (int x = 0; x < TC; ++x)
-              sts16((y < 2 ? ob0 : ob1) + (uint32_t)((y & 1) * OUT_ROW + x * OUT_PITCH) + cp, __half_as_ushort(__float2half_rn(acc[y][x])));
+              for (int xx = 0; xx < TC / 2; ++xx) {
+                const float m = fmaxf(fmaxf(fmaxf(acc[2 * yy][2 * xx], acc[2 * yy][2 * xx + 1]),
+                                            fmaxf(acc[2 * yy + 1][2 * xx], acc[2 * yy + 1][2 * xx + 1])), 0.0f);
+                sts16(ob0 + (uint32_t)(yy * OUT_ROW + xx * OUT_PITCH) + cp, __half_as_ushort(__float2half_rn(m)));
+              }
+          } else {
+#pragma unroll
+            for (int y = 0; y < TR4; ++y)
+#pragma unroll
+              for (int x = 0; x < TC; ++x)
+                sts16((y < 2 ? ob0 : ob1) + (uint32_t)((y & 1) * OUT_ROW + x * OUT_PITCH) + cp, __half_as_ushort(__float2half_rn(acc[y][x])));
+          }
           if (half == 0) {
             cur ^= 1u;
             fetch(cur, acc);
@@ -416,6 +430,22 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           const int row0 = TR4 * ty, colp = col0 + (lane >> 2);
           __half* dst = p.y + (size_t)n_img * p.Ho * p.Wo * p.F + g_out * FG + (lane & 3) * 8;
           const uint32_t src = sl + (uint32_t)(t * TC) * OUT_PITCH + (uint32_t)(t >> 4) * 4u;
+          if constexpr (ACT == 2) {
+            // pooled tile: 2 rows x 7 pixels, each pixel one 64-byte run of the image of half the height and width
+            const int prow0 = row0 >> 1, pcol = (col0 >> 1) + (lane >> 2);
+            uint4 pv[TR4 / 2];
+#pragma unroll
+            for (int yy = 0; yy < TR4 / 2; ++yy)
+              if (lane < 4 * (TC / 2)) {
+                const uint32_t a = ob0 + src + (uint32_t)(yy * OUT_ROW);
+                pv[yy].x = lds32(a); pv[yy].y = lds32(a + 4); pv[yy].z = lds32(a + 8); pv[yy].w = lds32(a + 12);
+              }
+#pragma unroll
+            for (int yy = 0; yy < TR4 / 2; ++yy)
+              if (lane < 4 * (TC / 2) && prow0 + yy < p.Ho && pcol < p.Wo)
+                *reinterpret_cast<uint4*>(dst + ((size_t)(prow0 + yy) * p.Wo + pcol) * p.F) = pv[yy];
+            continue;
+          }
           uint4 v[TR4][2];
 #pragma unroll
           for (int y = 0; y < TR4; ++y)
@@ -468,8 +498,9 @@ __device__ __forceinline__ bool blob_matches_block(const Params& p) {
 }
 
 // NCODES / GENERIC: the pattern codes the kernel carries code for (see one_kernel4); the host picks the smallest
-// set that covers the library.  RELU: results below zero are written as zero.
-template <int NCODES, bool GENERIC, bool RELU>
+// set that covers the library.  ACT: 1 - results below zero are written as zero; 2 - that, then the maximum of every
+// 2 x 2 block of results is written (the pooled image has half the height and width).
+template <int NCODES, bool GENERIC, int ACT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_conv_f16_img(const Params p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -484,8 +515,8 @@ k_conv_f16_img(const Params p) {
   // everything below reads the stage images or writes the output: the stage-image grid must be complete
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // ring geometry by the size of the largest descriptor block (see MAX_NS above)
-  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC, RELU>(p, smem);
-  else conv_body<false, NCODES, GENERIC, RELU>(p, smem);
+  if (bh->max_block_entries + 1 <= MAXE3) conv_body<true, NCODES, GENERIC, ACT>(p, smem);
+  else conv_body<false, NCODES, GENERIC, ACT>(p, smem);
 }
 
 // ------------------------------------------------------------------------------------------ cut items
@@ -547,6 +578,55 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts(const Params p) {
   }
 }
 
+// The same for a call with rectifier and 2 x 2 max pooling: one block per (cut item, pooled row of the thread
+// tiles); the four sums of a pooling window are formed piece by piece in the same fixed order, then clamped and
+// compared.  The pooled values go through shared memory as [32 tiles x 7 px][32 channels] and leave as 64-byte runs.
+__global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_pool(const Params p) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!blob_matches_block(p)) return;
+  __shared__ __align__(16) unsigned char stage[OUT_ROW];
+  constexpr int PX = TC / 2;                                  // pooled pixels of a tile row
+  const int yy = (int)blockIdx.x % (TR4 / 2), li = (int)blockIdx.x / (TR4 / 2);
+  const int item = p.n_whole + li;
+  const int g = p.d_NG.mod(item);
+  const Region it = decode_region(p, p.d_NG.div(item));
+  const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS;
+  static_assert(FG * PX * 32 % RP_THREADS == 0, "elements per thread");
+#pragma unroll 1
+  for (int i = 0; i < FG * PX * 32 / RP_THREADS; ++i) {
+    const int idx = (int)threadIdx.x + i * RP_THREADS;
+    const int lane = idx & 31, xx = (idx >> 5) % PX, slot = idx / (32 * PX);
+    float m = 0.0f;                                           // the rectifier's floor
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int y = 2 * yy + (w >> 1), x = 2 * xx + (w & 1);
+      const size_t e = ((size_t)slot * (TR4 * TC) + (size_t)(y * TC + x)) * 32 + lane;
+      float sum = 0.0f;
+      for (int q = 0; q < p.parts; ++q) sum += __ldg(src + (size_t)q * PIECE_FLOATS + e);   // piece 0 first
+      m = fmaxf(m, sum);
+    }
+    const int cpos = (__ldg(p.xfilt + g * FG + slot) & (FG - 1)) * 2;
+    *reinterpret_cast<__half*>(stage + (lane * TC + xx) * OUT_PITCH + cpos) = __float2half_rn(m);
+  }
+  __syncthreads();
+  const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+  const int t = threadIdx.x >> 5, lane = threadIdx.x & 31;    // one warp per thread tile
+  const int ly = t >> 2, lx = t & 3;
+  const int b = (ly < it.n0) ? 0 : 1;
+  const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+  const int ig = it.ig0 + b;
+  const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+  const int n_img = ig * p.NI + ni;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) return;
+  const int prow = (TR4 / 2) * ty + yy, pcol = ((it.cg * p.TXe + tx) * TC >> 1) + (lane >> 2);
+  if (lane < 4 * PX && prow < p.Ho && pcol < p.Wo) {
+    const int j = lane & 3;
+    const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage + (t * TC + (lane >> 2)) * OUT_PITCH + j * 16);
+    __half* dst = p.y + (((size_t)n_img * p.Ho + prow) * p.Wo + pcol) * p.F + g * FG + j * 8;
+    *reinterpret_cast<uint4*>(dst) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+  }
+}
+
 // ------------------------------------------------------------------------------------------ host side
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) { return imggeo::fill_geometry(p, F, C, N, H, W, CBI); }
 
@@ -596,6 +676,10 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   p.K = K; p.n_keep = n_keep;
   p.wait_ns = g_wait_ns; p.test_skip = g_test_skip;
   p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1; p.relu = relu;
+  if (relu == 2) {   // rectifier and 2 x 2 max pooling: the pooled image is written
+    if (stride != 1 || (H & 1) || (W & 1)) return set_error(PAT_ERR_SHAPE, "pat_conv3x3_ws_act: pooling needs stride 1 and even H and W");
+    p.Ho = H / 2; p.Wo = W / 2;
+  }
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   // the smallest set of compiled pattern codes that covers the library
@@ -605,8 +689,9 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
     variant = std::max(variant, code == kGenericCode ? 2 : (code >= 6 ? 1 : 0));
   }
   using KernelFn = void (*)(const Params);
-  static const KernelFn kernels[6] = {k_conv_f16_img<6, false, false>, k_conv_f16_img<kNumCodes, false, false>, k_conv_f16_img<kNumCodes, true, false>,
-                                      k_conv_f16_img<6, false, true>, k_conv_f16_img<kNumCodes, false, true>, k_conv_f16_img<kNumCodes, true, true>};
+  static const KernelFn kernels[9] = {k_conv_f16_img<6, false, 0>, k_conv_f16_img<kNumCodes, false, 0>, k_conv_f16_img<kNumCodes, true, 0>,
+                                      k_conv_f16_img<6, false, 1>, k_conv_f16_img<kNumCodes, false, 1>, k_conv_f16_img<kNumCodes, true, 1>,
+                                      k_conv_f16_img<6, false, 2>, k_conv_f16_img<kNumCodes, false, 2>, k_conv_f16_img<kNumCodes, true, 2>};
 
   static thread_local DeviceSlot slots[kMaxDevices];
   DeviceSlot* dv = device_slot(slots);
@@ -633,11 +718,11 @@ int conv_f16_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   cudaLaunchConfig_t cfg = {};
   cfg.stream = st; cfg.attrs = &pdl; cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM_BYTES;
-  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant + (relu ? 3 : 0)], p), "pat_conv3x3 launch")) return rc;
+  if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[variant + 3 * relu], p), "pat_conv3x3 launch")) return rc;
   count_launches(2);
   if (p.parts > 1) {
-    cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * 2)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
-    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, k_reduce_parts, p), "pat_conv3x3 launch")) return rc;
+    cfg.gridDim = dim3((unsigned)(relu == 2 ? p.n_split * (TR4 / 2) : p.n_split * TR4 * 2)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
+    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, relu == 2 ? k_reduce_parts_pool : k_reduce_parts, p), "pat_conv3x3 launch")) return rc;
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");

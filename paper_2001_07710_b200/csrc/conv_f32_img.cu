@@ -436,10 +436,21 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
 #pragma unroll
               for (int x = 0; x < TC; ++x) acc[y][x] = fmaxf(acc[y][x], 0.0f);
           }
+          if (p.relu == 2) {
+            // rectifier and 2 x 2 max pooling: a thread tile starts at an even row and column, so the pooling windows
+            // of this round's two rows lie in this lane's registers; the seven pooled values take the first slot
 #pragma unroll
-          for (int x = 0; x < TC; ++x) {
-            sts32(ob0 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[2][x] : acc[0][x]));
-            sts32(ob1 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[3][x] : acc[1][x]));
+            for (int xx = 0; xx < TC / 2; ++xx) {
+              const float top = round ? fmaxf(acc[2][2 * xx], acc[2][2 * xx + 1]) : fmaxf(acc[0][2 * xx], acc[0][2 * xx + 1]);
+              const float bot = round ? fmaxf(acc[3][2 * xx], acc[3][2 * xx + 1]) : fmaxf(acc[1][2 * xx], acc[1][2 * xx + 1]);
+              sts32(ob0 + (uint32_t)(xx * OUT_PITCH) + cp, __float_as_uint(fmaxf(fmaxf(top, bot), 0.0f)));
+            }
+          } else {
+#pragma unroll
+            for (int x = 0; x < TC; ++x) {
+              sts32(ob0 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[2][x] : acc[0][x]));
+              sts32(ob1 + (uint32_t)(x * OUT_PITCH) + cp, __float_as_uint(round ? acc[3][x] : acc[1][x]));
+            }
           }
           if (half == 0) {
             if (round == 0) park(cur, acc);     // its rows 2-3 are still to come
@@ -464,6 +475,23 @@ __device__ __forceinline__ void conv_body(const Params& p, unsigned char* smem) 
           if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N)) continue;
           const int col0 = (it.cg * p.TXe + tx) * TC;
           const uint32_t src = slc + (uint32_t)(t * TC) * OUT_PITCH + (uint32_t)(t >> 4) * 4u;
+          if (p.relu == 2) {
+            // this round's pooled row of the tile: seven pixels of 128 bytes in the image of half the height and width
+            const int prow = (TR4 / 2) * ty + round, pcol = (col0 >> 1) + (lane >> 3);
+            float* dst = p.y + ((size_t)n_img * p.Ho + prow) * p.Wo * p.F + g_out * FG + (lane & 7) * 4;
+            uint4 pv[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              if (4 * i + (lane >> 3) < TC / 2) {
+                const uint32_t a = ob0 + src + (uint32_t)(4 * i) * OUT_PITCH;
+                pv[i].x = lds32(a); pv[i].y = lds32(a + 4); pv[i].z = lds32(a + 8); pv[i].w = lds32(a + 12);
+              }
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              if (4 * i + (lane >> 3) < TC / 2 && prow < p.Ho && pcol + 4 * i < p.Wo)
+                *reinterpret_cast<uint4*>(dst + (size_t)(pcol + 4 * i) * p.F) = pv[i];
+            continue;
+          }
 #pragma unroll
           for (int yy = 0; yy < 2; ++yy) {
             const int row = TR4 * ty + 2 * round + yy;
@@ -567,6 +595,39 @@ __global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_f32(const Params p)
   p.y[(((size_t)n_img * p.Ho + (row >> p.sub)) * p.Wo + (col >> p.sub)) * p.F + __ldg(p.xfilt + g * FG + slot)] = p.relu ? fmaxf(sum, 0.0f) : sum;
 }
 
+// The same for a call with rectifier and 2 x 2 max pooling: one block per (cut item, pooled value of the thread
+// tile); the four sums of the pooling window are formed piece by piece in the same fixed order, then clamped and compared.
+__global__ void __launch_bounds__(RP_THREADS) k_reduce_parts_pool_f32(const Params p) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!blob_matches_block(p)) return;
+  constexpr int PV = (TR4 / 2) * (TC / 2);
+  const int v = (int)blockIdx.x % PV, li = (int)blockIdx.x / PV;
+  const int yy = v / (TC / 2), xx = v % (TC / 2);
+  const int item = p.n_whole + li;
+  const int g = item % p.NG;
+  const Region it = decode_region(p, item / p.NG);
+  const int lane = threadIdx.x & 31, slot = threadIdx.x >> 5;
+  const float* src = p.partials + (size_t)li * p.parts * PIECE_FLOATS + (size_t)slot * (TR4 * TC) * 32 + lane;
+  float m = 0.0f;                                          // the rectifier's floor
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const float* s = src + (size_t)((2 * yy + (w >> 1)) * TC + 2 * xx + (w & 1)) * 32;
+    float sum = 0.0f;
+    for (int q = 0; q < p.parts; ++q) sum += __ldg(s + (size_t)q * PIECE_FLOATS);   // piece 0 first
+    m = fmaxf(m, sum);
+  }
+  const int txe_shift = (p.TXe == 4) ? 2 : (p.TXe == 2 ? 1 : 0);
+  const int ly = lane >> 2, lx = lane & 3;
+  const int b = (ly < it.n0) ? 0 : 1;
+  const int ni = lx >> txe_shift, tx = lx & (p.TXe - 1);
+  const int ig = it.ig0 + b;
+  const int ty = b ? (ly - it.n0) : (it.ta0 + ly);
+  const int n_img = ig * p.NI + ni;
+  const int prow = (TR4 / 2) * ty + yy, pcol = ((it.cg * p.TXe + tx) * TC >> 1) + xx;
+  if (!((b == 0 || it.band1) && ig < p.NIG && n_img < p.N) || prow >= p.Ho || pcol >= p.Wo) return;
+  p.y[(((size_t)n_img * p.Ho + prow) * p.Wo + pcol) * p.F + __ldg(p.xfilt + g * FG + slot)] = m;
+}
+
 // ------------------------------------------------------------------------------------------ host side
 static bool fill_geometry(Params& p, int F, int C, int N, int H, int W) { return imggeo::fill_geometry(p, F, C, N, H, W, CBI); }
 
@@ -604,6 +665,10 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   if (!p.status) return set_error(PAT_ERR_CUDA, "pat_conv3x3: cannot resolve the status word");
   p.K = K; p.n_keep = n_keep;
   p.sub = stride - 1; p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1; p.relu = relu;
+  if (relu == 2) {   // rectifier and 2 x 2 max pooling: the pooled image is written
+    if (stride != 1 || (H & 1) || (W & 1)) return set_error(PAT_ERR_SHAPE, "pat_conv3x3_ws_act: pooling needs stride 1 and even H and W");
+    p.Ho = H / 2; p.Wo = W / 2;
+  }
   for (int j = 0; j < 256; ++j) p.masks[j] = (j < K) ? masks[j] : (uint16_t)0;
 
   int variant = 0;
@@ -642,8 +707,8 @@ int conv_f32_img(const void* blob, int F, int C, const uint16_t* masks, int K, i
   if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernels[3 * p.sub + variant], p), "pat_conv3x3 launch")) return rc;
   count_launches(2);
   if (p.parts > 1) {
-    cfg.gridDim = dim3((unsigned)(p.n_split * TR4 * TC)); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
-    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, k_reduce_parts_f32, p), "pat_conv3x3 launch")) return rc;
+    cfg.gridDim = dim3((unsigned)(p.n_split * (relu == 2 ? (TR4 / 2) * (TC / 2) : TR4 * TC))); cfg.blockDim = dim3(RP_THREADS); cfg.dynamicSmemBytes = 0;
+    if (int rc = check_cuda(cudaLaunchKernelEx(&cfg, relu == 2 ? k_reduce_parts_pool_f32 : k_reduce_parts_f32, p), "pat_conv3x3 launch")) return rc;
     count_launches(1);
   }
   return check_cuda(cudaGetLastError(), "pat_conv3x3 launch");

@@ -20,7 +20,8 @@ struct ImgGeometry {
   int N, H, W, C, F;
   int nct;                 // ring stages per work item: C / (channels of a stage)
   int Ho, Wo, sub;         // output size; sub = stride - 1: with stride 2 only the results at even rows and columns are written
-  int relu;                // 1: results below zero are written as zero (the rectifier that follows the layer, fused)
+  int relu;                // 1: results below zero are written as zero (the rectifier that follows the layer, fused);
+                           // 2: that, then 2 x 2 max pooling (Ho, Wo are then the pooled sizes H / 2, W / 2)
   int TY;                  // tile rows per image (ceil(H / 4), at least four)
   int TXe, NI;             // tile columns per region, images side by side
   int CG, NIG;             // column groups per image, image groups

@@ -501,3 +501,51 @@ def test_conv_with_fused_rectifier(case, dtype):
     # where the reference is clearly negative before the rectifier the output is exactly zero
     pre = oracle.conv3x3(stored_weights(wm_o, dtype), x, stride)
     assert (out[pre < -1e-2] == 0).all()
+
+
+@pytest.mark.parametrize("dtype", ["f16", "f32"])
+@pytest.mark.parametrize("case", [(3, 56, 56, 32, 64, 8, 1, 4), (5, 14, 14, 64, 32, 8, 1, 2), (24, 28, 56, 64, 64, 8, 1, 8),
+                                  (1, 28, 28, 64, 64, 8, 1, 8), (9, 8, 8, 16, 32, 12, 1, 1), (2, 30, 28, 32, 32, 4, 1, 2)])
+def test_conv_with_fused_rectifier_and_pooling(case, dtype):
+    """pat_conv3x3_ws_act(act = 2): the pooled image max(0, 2 x 2 block of conv) written by the convolution's own
+    epilogue (whole items, cut items through the pooling reduce kernel, a batch that is cut entirely, 14 x 14 images
+    whose last tile row is half empty, images narrower than a thread tile, a height that is no multiple of 4) -
+    every element against the oracle's relu_maxpool(conv), and bit for bit against the two-pass result of the
+    library itself (same sums, monotone rounding)."""
+    N, H, W, C, F, K, num, den = case
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 11)
+    w = workloads.make_weights(rng, F, C)
+    x = store(workloads.make_inputs(rng, N, H, W, C), dtype)
+    masks = oracle.library(K)
+    n_keep = F * C * num // den
+    pid_o, wm_o, _ = oracle.project(w, masks, n_keep)
+    ref = oracle.relu_maxpool(oracle.conv3x3(stored_weights(wm_o, dtype), x, 1), True)
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, dtype)
+    xt = torch.from_numpy(x).cuda()
+    assert pc.pat_conv3x3_workspace(F, C, dtype, N, H, W, 1) > 0
+    y = torch.full((N, H // 2, W // 2, F), float("nan"), dtype=xt.dtype, device="cuda")
+    pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, xt, 1, y=y, pool=True)
+    assert pc.pat_query_status() == 0
+    out = y.float().cpu().numpy()
+    assert tuple(out.shape) == ref.shape and np.isfinite(out).all() and (out >= 0).all()
+    check_close(out, ref, dtype)
+    two_pass = pc.pat_relu_maxpool(pc.pat_conv3x3(blob, F, C, masks, n_keep, dtype, xt, 1), dtype, True)
+    assert torch.equal(two_pass, y)
+
+
+def test_fused_pooling_refuses_what_it_cannot_pool():
+    """act = 2 with stride 2, an odd height, or a layer without workspace kernels: PAT_ERR_SHAPE, nothing written."""
+    F, C, K = 32, 16, 8
+    masks = oracle.library(K)
+    w = _weights(9, F, C)
+    n_keep = F * C // 2
+    pid, wm, blob = gpu_project_pack(w, masks, n_keep, "f16")
+    for (N, H, W, stride) in [(1, 28, 28, 2), (1, 15, 14, 1), (1, 24, 46, 1)]:
+        x = torch.zeros((N, H, W, C), dtype=torch.float16, device="cuda")
+        y = torch.full((N, H // 2, W // 2, F), 7.0, dtype=torch.float16, device="cuda")
+        with pytest.raises(pc.PatError) as e:
+            pc.pat_conv3x3(blob, F, C, masks, n_keep, "f16", x, stride, y=y, pool=True)
+        assert e.value.code == 2                                        # PAT_ERR_SHAPE
+        torch.cuda.synchronize()
+        assert float(y.min()) == 7.0
+    assert pc.pat_query_status() == 0
