@@ -381,6 +381,8 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if world == 1 and cfg.number == 3 and not args.no_other_configs:
+        out["fused_pooling"] = fused_pooling(pc, torch, layers, masks, dtype, cws, N)
     if world == 1 and not args.no_other_configs and args.batch is None and args.layers is None:
         # the other four configurations: short measurements of their own, after the main timed region
         out["other_configs"] = {str(c): quick_config(pc, torch, c, peaks) for c in range(5) if c != cfg.number}
@@ -392,6 +394,43 @@ def run_ours(args):
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def fused_pooling(pc, torch, layers, masks, dtype, cws, N, reps: int = 5):
+    """The five layers of the VGG-16 stack that are followed by the rectifier and 2x2 max pooling: the convolution
+    with both fused into its epilogue (pat_conv3x3_ws_act, act = 2: the pooled image is the only output) next to the
+    convolution followed by pat_relu_maxpool as a pass of its own.  Plain launches on one stream, CUDA events,
+    two warm-up calls; the inputs and packed weights are those of the step (already resident)."""
+    res = {}
+    for st in layers:
+        L = st["L"]
+        if L.dense or L.name not in ("conv2", "conv4", "conv7", "conv10", "conv13"):
+            continue
+        yp = torch.empty((N, L.H // 2, L.W // 2, L.F), dtype=st["y"].dtype, device="cuda")
+
+        def two_pass():
+            pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], 1, y=st["y"], workspace=cws)
+            pc.pat_relu_maxpool(st["y"], dtype, True, yp)
+
+        def fused():
+            pc.pat_conv3x3(st["blob"], L.F, L.C, masks[L.K], L.n_keep, dtype, st["x"], 1, y=yp, workspace=cws, pool=True)
+
+        t = []
+        for fn in (two_pass, fused):
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            t.append(e0.elapsed_time(e1) / reps * 1e3)
+        res[L.name] = {"conv_then_relu_maxpool_us": round(t[0], 1), "fused_us": round(t[1], 1), "speedup": round(t[0] / t[1], 3)}
+        del yp
+    assert pc.pat_query_status() == 0
+    return res
 
 
 def admm_primitives(pc, torch, peaks, with_cpu: bool, reps: int = 10):

@@ -20,6 +20,7 @@ from helpers import check_close, read_blob
 pytestmark = pytest.mark.gpu
 
 N_RANDOM = 3000
+POOLED_LAYERS = ("conv2", "conv4", "conv7", "conv10", "conv13")   # Section 7's VGG-16: pooling after these
 WHOLE_IMAGE_MACS = 2.5e9      # dense 9 * C * F * Ho * Wo of one image: about a second of the oracle on 16 cores
 
 
@@ -70,10 +71,19 @@ def _check_layer(cfg, L):
     ref = oracle.conv3x3_at(wst, xs, coords, L.stride)
     out = y[coords[:, 0], coords[:, 1], coords[:, 2], coords[:, 3]].float().cpu().numpy()
     check_close(out, ref, dtype)
+    # the layers of the VGG-16 stack that 2x2 max pooling follows: the pooled image written by the convolution's own
+    # epilogue equals, bit for bit and over the whole batch, the pooling pass run on the full-size output
+    pooled = None
+    if not L.dense and cfg.number in (1, 3) and L.name in POOLED_LAYERS:
+        pooled = pc.pat_conv3x3(blob, L.F, L.C, masks, L.n_keep, dtype, xt, L.stride, pool=True)
+        assert pc.pat_query_status() == 0
+        assert torch.equal(pooled, pc.pat_relu_maxpool(y, dtype, True))
     if _whole(L):
         for n in sorted({0, cfg.N // 2, cfg.N - 1}):
             ref_img = oracle.conv3x3(wst, xs[n:n + 1], L.stride)
             check_close(y[n:n + 1].float().cpu().numpy(), ref_img, dtype)
+            if pooled is not None:
+                check_close(pooled[n:n + 1].float().cpu().numpy(), oracle.relu_maxpool(ref_img, True), dtype)
 
 
 def _layers(cfg_no):
