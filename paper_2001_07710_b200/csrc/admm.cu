@@ -29,8 +29,8 @@ __device__ __forceinline__ T group_sum(T v) {
 // start with at least one entry above it the steps reach the root in finitely many rounds (after the first step they
 // approach it from below and never pass it).  The sets {entries above nu} are nested whatever nu is, so two rounds
 // with the same number of entries above nu have the same set, and then nu is the root of that piece: no set has
-// to be stored, a round is one pass "compare, add, count" over the entries.  The rounds run in fp32 from nu = -inf
-// (all entries) until the count repeats, then in fp64 from the fp32 result until the count repeats again - usually
+// to be stored, a round is one pass "compare, add, count" over the entries.  The rounds run in fp32 from a lower
+// bound of the root (see the kernel) until the count repeats, then in fp64 from the fp32 result until the count repeats again - usually
 // two or three rounds - so the final piece and its root are exact: the sums are exact to about 1e-16 relative (the
 // inputs are fp32), and there is one rounding to fp32 at the end.
 //
@@ -39,7 +39,7 @@ __device__ __forceinline__ T group_sum(T v) {
 // chains in flight, not many lanes per chain.  Entry j of a vector sits in lane j % L, slot j / L.  u may be d.
 constexpr int kVecQ = 16;
 template <int L>
-__global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float* d, long long n, int K, float* u) {
+__global__ void __launch_bounds__(32 * kVecWarps, 5) k_simplex_project(const float* d, long long n, int K, float* u) {
   constexpr int G = 32 / L;                // vectors per warp
   const int lane = threadIdx.x & 31, sl = lane & (L - 1), g = lane / L;
   const long long stride = (long long)gridDim.x * kVecWarps * G;
@@ -49,57 +49,67 @@ __global__ void __launch_bounds__(32 * kVecWarps) k_simplex_project(const float*
     const bool valid = base + g < n;
     const long long i = valid ? base + g : n - 1;       // a group without a vector repeats the last one and stores nothing
     float x[kVecQ];                        // slots beyond K hold the lowest float: never above any nu
+    const float* di = d + i * K + sl;
+    const int nq = (K - sl + L - 1) / L;   // this lane's entries: slots 0 .. nq - 1
 #pragma unroll
-    for (int q = 0; q < kVecQ; ++q) x[q] = (sl + L * q < K) ? __ldcs(d + i * K + sl + L * q) : -3.402823466e38f;
-    float nu32 = -3.402823466e38f;         // every entry of the vector is above it (or equal, if it is that low itself)
-    int before = -1;
+    for (int q = 0; q < kVecQ; ++q) x[q] = (q < nq) ? __ldcs(di + L * q) : -3.402823466e38f;
+    // Start: for any set S of entries (sum of S - 1) / |S| is at most the root (the root is the largest such value,
+    // taken over the sets of the k largest entries), so the largest entry of every lane gives a lower bound that lies
+    // close below the root when few entries are active, and at least one entry is above it (the root is below the largest
+    // entry).  Rounding may lift it past the root: the first Newton step from there lands below the root again.
+    float top = x[0];
+#pragma unroll
+    for (int q = 1; q < kVecQ; ++q) top = fmaxf(top, x[q]);
+    float nu32 = (group_sum<L>(top) - 1.0f) / (float)L;
+    if (!(nu32 > -3.402823466e38f)) nu32 = -3.402823466e38f;   // overflow of the sum (or a NaN): start below every entry
+    // Counts are kept as floats (exact up to 2^24): a pass is then one comparison and two predicated additions per entry.
+    float before = -1.0f;
     bool done = false;
     for (int round = 0; round < K + 2; ++round) {       // fp32 rounds
-      float s = 0.0f;
-      int c = 0;
+      float s = 0.0f, c = 0.0f;
 #pragma unroll
-      for (int q = 0; q < kVecQ; ++q) {
-        const bool above = x[q] > nu32;
-        s += above ? x[q] : 0.0f;
-        c += above ? 1 : 0;
-      }
+      for (int q = 0; q < kVecQ; ++q)
+        if (x[q] > nu32) { s += x[q]; c += 1.0f; }
       s = group_sum<L>(s);
       c = group_sum<L>(c);
       if (!done) {
-        if (c == before || c == 0) done = true;          // the set repeats (or rounding has pushed nu past the largest entry)
-        else { nu32 = (s - 1.0f) / (float)c; before = c; }
+        if (c == before || c == 0.0f) done = true;       // the set repeats (or rounding has pushed nu past the largest entry)
+        else { nu32 = (s - 1.0f) / c; before = c; }
       }
       if (__all_sync(0xFFFFFFFFu, done)) break;          // every vector of the warp is through
     }
+    // Exact rounds.  A float x is above a double nu exactly when it is above nu rounded down to a float, so the sets are
+    // formed by fp32 comparisons; only the sum of a set is taken in fp64.  A round: count the entries above the
+    // current threshold; the same count as before means the same set, whose root nu already is; otherwise its exact
+    // sum gives the next nu.  After the fp32 rounds the first set is usually the final one: one fp64 sum, two counts.
     double nu = (double)nu32;
-    before = -1;
+    float thr = nu32;
+    before = -1.0f;
     done = false;
-    for (int round = 0; round < K + 3; ++round) {       // fp64 rounds from the fp32 result
-      double s = 0.0;
-      int c = 0;
-#pragma unroll
-      for (int q = 0; q < kVecQ; ++q) {
-        const bool above = (double)x[q] > nu;
-        s += above ? (double)x[q] : 0.0;
-        c += above ? 1 : 0;
-      }
-      s = group_sum<L>(s);
-      c = group_sum<L>(c);
-      if (!done) {
-        if (c == before) done = true;
-        else if (c == 0) { nu = -1.7976931348623157e308; before = -1; }   // past the largest entry: start again from all entries
-        else { nu = (s - 1.0) / (double)c; before = c; }
-      }
-      if (__all_sync(0xFFFFFFFFu, done)) break;
-    }
-    if (valid) {
-      float* ui = u + i * K;
+    for (int round = 0; round < K + 4; ++round) {
+      float c = 0.0f;
 #pragma unroll
       for (int q = 0; q < kVecQ; ++q)
-        if (sl + L * q < K) {
-          const double r = (double)x[q] - nu;
-          __stcs(ui + sl + L * q, (float)(r > 0.0 ? r : 0.0));
-        }
+        if (x[q] > thr) c += 1.0f;
+      c = group_sum<L>(c);
+      if (!done && c == before) done = true;
+      if (__all_sync(0xFFFFFFFFu, done)) break;
+      double s = 0.0;
+#pragma unroll
+      for (int q = 0; q < kVecQ; ++q)
+        if (x[q] > thr) s += (double)x[q];
+      s = group_sum<L>(s);
+      if (!done) {
+        if (c == 0.0f) { thr = -3.402823466e38f; before = -1.0f; }   // past the largest entry: start again from all entries (not the padding)
+        else { nu = (s - 1.0) / (double)c; thr = __double2float_rd(nu); before = c; }
+      }
+    }
+    if (valid) {
+      float* ui = u + i * K + sl;
+      // x - nu in fp64 is exact up to one rounding; an entry at or below the threshold is not above nu
+#pragma unroll
+      for (int q = 0; q < kVecQ; ++q)
+        if (q < nq) __stcs(ui + L * q, x[q] > thr ? (float)((double)x[q] - nu) : 0.0f);
     }
   }
 }
