@@ -45,6 +45,10 @@ __device__ __forceinline__ int channel_of(int jt, int col) {
   return (jt < 4 ? 0 : 32) + 8 * (col >> 1) + 2 * (jt & 3) + (col & 1);
 }
 
+// WORDS (W even): the window is moved as aligned 4-byte words.  The first half of a staged row is then the half in
+// front of pixel x0 - 1 (that pixel starts at an odd half index of the image whenever W and x0 are even), pixel
+// boundaries of the window's edges fall on word boundaries, and a row of the window is 52 consecutive words.
+template <bool WORDS>
 __global__ void __launch_bounds__(NTHREADS, 4) k_conv_dense_c3_mma(const Args a) {
   __shared__ __align__(16) __half tile[(TH + 2) * ROWP];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -64,17 +68,32 @@ __global__ void __launch_bounds__(NTHREADS, 4) k_conv_dense_c3_mma(const Args a)
     }
 
   // the input window of a tile travels through registers: the next tile's loads are in flight while this one is computed
-  constexpr int WIN = (TH + 2) * (TW + 2) * 3, PER_THREAD = (WIN + NTHREADS - 1) / NTHREADS;
-  __half win[PER_THREAD];
+  // (staged rows start one half early in both variants: half 0 of a row is unused, pixel x0 - 1 begins at half 1)
+  constexpr int RW = ROWP / 2;             // words per staged row (52)
+  constexpr int WIN = WORDS ? (TH + 2) * RW : (TH + 2) * (TW + 2) * 3, PER_THREAD = (WIN + NTHREADS - 1) / NTHREADS;
+  static_assert(ROWP % 2 == 0 && ROWP >= (TW + 2) * 3 + 2, "a staged row holds the unused first half, 34 pixels and a last half");
+  uint32_t win[PER_THREAD];                // WORDS: a word each; otherwise one half each
   auto load_window = [&](long long tl) {
     const int tx = (int)(tl % a.tiles_x), ty = (int)((tl / a.tiles_x) % a.tiles_y), n = (int)(tl / ((long long)a.tiles_x * a.tiles_y));
 #pragma unroll
     for (int q = 0; q < PER_THREAD; ++q) {
       const int i = (int)threadIdx.x + q * NTHREADS;
-      const int row = i / ((TW + 2) * 3), rem = i % ((TW + 2) * 3);
-      const int yy = ty * TH - 1 + row, xx = tx * TW - 1 + rem / 3;
-      win[q] = __float2half_rn(0.0f);
-      if (i < WIN && yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) win[q] = a.x[(((size_t)n * a.H + yy) * a.W + xx) * 3 + rem % 3];
+      win[q] = 0u;
+      if constexpr (WORDS) {
+        // word j of a row = halves 2 j - 1, 2 j of the window row; both belong to pixels on the same side of the
+        // image's edge (or one of them is an unused half), so the pixel of half 2 j decides (half 101 for the last word)
+        const int row = i / RW, j = i % RW;
+        const int yy = ty * TH - 1 + row, xx = tx * TW - 1 + (j == RW - 1 ? TW + 1 : (2 * j) / 3);
+        if (i < WIN && yy >= 0 && yy < a.H && xx >= 0 && xx < a.W) {
+          const long long h0 = (((long long)n * a.H + yy) * a.W + tx * TW - 1) * 3 - 1;   // even: the row's first word
+          win[q] = __ldg(reinterpret_cast<const uint32_t*>(a.x + h0) + j);
+        }
+      } else {
+        const int row = i / ((TW + 2) * 3), rem = i % ((TW + 2) * 3);
+        const int yy = ty * TH - 1 + row, xx = tx * TW - 1 + rem / 3;
+        if (i < WIN && yy >= 0 && yy < a.H && xx >= 0 && xx < a.W)
+          win[q] = __half_as_ushort(a.x[(((size_t)n * a.H + yy) * a.W + xx) * 3 + rem % 3]);
+      }
     }
   };
   if ((long long)blockIdx.x < a.n_tiles) load_window(blockIdx.x);
@@ -85,7 +104,11 @@ __global__ void __launch_bounds__(NTHREADS, 4) k_conv_dense_c3_mma(const Args a)
 #pragma unroll
     for (int q = 0; q < PER_THREAD; ++q) {
       const int i = (int)threadIdx.x + q * NTHREADS;
-      if (i < WIN) tile[(i / ((TW + 2) * 3)) * ROWP + i % ((TW + 2) * 3)] = win[q];
+      if constexpr (WORDS) {
+        if (i < WIN) reinterpret_cast<uint32_t*>(tile)[i] = win[q];
+      } else {
+        if (i < WIN) tile[(i / ((TW + 2) * 3)) * ROWP + 1 + i % ((TW + 2) * 3)] = __ushort_as_half((unsigned short)win[q]);
+      }
     }
     __syncthreads();
     if (tl + gridDim.x < a.n_tiles) load_window(tl + gridDim.x);
@@ -99,7 +122,7 @@ __global__ void __launch_bounds__(NTHREADS, 4) k_conv_dense_c3_mma(const Args a)
 #pragma unroll
       for (int r = 0; r < 3; ++r) {
         // A[m][k] = tile[ry + r][(px0 + m) * 3 + k] for k < 9, zero above
-        const __half* rowp = tile + (ry + r) * ROWP + px0 * 3;
+        const __half* rowp = tile + (ry + r) * ROWP + 1 + px0 * 3;
         const __half z = __float2half_rn(0.0f);
         uint32_t af[4];
         af[0] = pack2(rowp[g * 3 + 2 * t], rowp[g * 3 + 2 * t + 1]);
@@ -149,7 +172,8 @@ int conv_dense_c3_mma(const float* w, const void* x, void* y, int N, int H, int 
   const int sm_count = dv->sms;
   const long long want = (long long)sm_count * 8;         // eight resident blocks of four warps per SM
   const unsigned grid = (unsigned)(a.n_tiles < want ? a.n_tiles : want);
-  k_conv_dense_c3_mma<<<grid, NTHREADS, 0, st>>>(a);
+  if (W % 2 == 0) k_conv_dense_c3_mma<true><<<grid, NTHREADS, 0, st>>>(a);
+  else k_conv_dense_c3_mma<false><<<grid, NTHREADS, 0, st>>>(a);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "pat_conv3x3_dense launch");
 }

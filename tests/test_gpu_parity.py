@@ -379,7 +379,8 @@ def test_conv_tuned_f16_arbitrary_library():
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
-@pytest.mark.parametrize("N,H,W,C,F,stride", [(2, 40, 70, 3, 64, 1), (1, 9, 9, 1, 8, 1), (2, 17, 33, 3, 40, 2), (1, 16, 16, 16, 32, 1)])
+@pytest.mark.parametrize("N,H,W,C,F,stride", [(2, 40, 70, 3, 64, 1), (1, 9, 9, 1, 8, 1), (2, 17, 33, 3, 40, 2), (1, 16, 16, 16, 32, 1),
+                                             (2, 10, 37, 3, 64, 1), (1, 8, 32, 3, 64, 1), (3, 5, 64, 3, 64, 1)])
 def test_dense_conv_matches_oracle(N, H, W, C, F, stride, dtype):
     rng = np.random.default_rng(N * 1000 + H)
     w = workloads.make_weights(rng, F, C)
