@@ -167,6 +167,14 @@ def run_ours(args):
 
     cfg = workloads.configs()[args.config]
     N = cfg.N if args.batch is None else args.batch
+    if args.strong and world > 1:
+        # strong scaling: the configuration's batch is cut into contiguous slices, one per rank (no data-path
+        # collective: images are independent); every rank draws the tensors of a batch of its slice's size
+        from paper_2001_07710_b200.sharding import shard_batch
+        lo, hi = shard_batch(N, world, rank)
+        if hi == lo:
+            raise SystemExit("bench.py --strong: more ranks than images in the batch")
+        N = hi - lo
     dtype = cfg.dtype
     tdt = torch.float16 if dtype == "f16" else torch.float32
     elem = 2 if dtype == "f16" else 4
@@ -359,7 +367,7 @@ def run_ours(args):
                f"inputs and outputs of a step ({touched / 1e6:.1f} MB) are not much larger than the 126 MB L2: no flush between steps, warm-cache numbers")
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "strong" if (args.strong and world > 1) else "weak",
         "vs_baseline": None, "dtype": "f16 storage, f32 accumulate" if dtype == "f16" else "f32", "data": "synthetic",
         "config": {"workload": f"config {cfg.number}: {cfg.name}", "batch_per_gpu": N,
                    "layers": len(layers), "step": "project + pack + conv for every layer" + ("" if args.no_overlap else ", projection / packing of each layer on a stream of its own")
@@ -713,6 +721,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="workload number (3 = VGG-16 batch 64 fp16 storage)")
+    ap.add_argument("--strong", action="store_true", help="with N > 1 ranks: shard the configuration's batch over the ranks (strong scaling) instead of one whole batch per rank")
     ap.add_argument("--batch", type=int, default=None, help="override the batch size (profiling small cases)")
     ap.add_argument("--layers", default=None, help="comma-separated layer names: run only these (profiling one layer)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
