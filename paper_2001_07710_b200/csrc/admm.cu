@@ -73,11 +73,15 @@ __global__ void __launch_bounds__(32 * kVecWarps, 5) k_simplex_project(const flo
       s = group_sum<L>(s);
       c = group_sum<L>(c);
       if (!done) {
-        if (c == before || c == 0.0f) done = true;       // the set repeats (or rounding has pushed nu past the largest entry)
+        if (c == before || c == 0.0f) { done = true; before = c; }   // the set repeats (or rounding has pushed nu past the largest entry)
         else { nu32 = (s - 1.0f) / c; before = c; }
       }
       if (__all_sync(0xFFFFFFFFu, done)) break;          // every vector of the warp is through
     }
+    // `before` is now the number of entries above nu32 (when the rounds ended because the count repeated); if that holds
+    // for every vector of the warp the first exact round needs no counting pass
+    const float known = done ? before : 0.0f;
+    const bool skip_first_count = __all_sync(0xFFFFFFFFu, known > 0.0f);
     // Exact rounds.  A float x is above a double nu exactly when it is above nu rounded down to a float, so the sets are
     // formed by fp32 comparisons; only the sum of a set is taken in fp64.  A round: count the entries above the
     // current threshold; the same count as before means the same set, whose root nu already is; otherwise its exact
@@ -87,11 +91,14 @@ __global__ void __launch_bounds__(32 * kVecWarps, 5) k_simplex_project(const flo
     before = -1.0f;
     done = false;
     for (int round = 0; round < K + 4; ++round) {
-      float c = 0.0f;
+      float c = known;
+      if (round > 0 || !skip_first_count) {
+        c = 0.0f;
 #pragma unroll
-      for (int q = 0; q < kVecQ; ++q)
-        if (x[q] > thr) c += 1.0f;
-      c = group_sum<L>(c);
+        for (int q = 0; q < kVecQ; ++q)
+          if (x[q] > thr) c += 1.0f;
+        c = group_sum<L>(c);
+      }
       if (!done && c == before) done = true;
       if (__all_sync(0xFFFFFFFFu, done)) break;
       double s = 0.0;
